@@ -1,0 +1,235 @@
+/*
+ * mpgemmfi -- fault-injected mixed-precision GEMM with in-kernel exponent-only
+ * detection/correction, for NVIDIA B200 (sm_100a).
+ *
+ * C ABI. Every matrix pointer is a caller-owned DEVICE pointer that must stay
+ * valid until the work queued on `stream` has completed. All entry points are
+ * asynchronous and stream-ordered; none of them synchronises, and none allocates
+ * device memory. Return value: MPGEMMFI_OK (0) or a negative MPGEMMFI_ERR_*.
+ * Problems found on the device (a site outside the matrices, a wait that ran into
+ * its time limit) never trap: they set bits in the status word of the flags header
+ * (or the trial record) and the offending site is skipped.
+ *
+ * Operation (paper Section II-B, IV-C): D = A x B with A (M x K) and B (K x N) in a
+ * low-precision format -- FP16 (1/5/10), BF16 (1/8/7) or TF32 (1/8/10 held in a
+ * 32-bit word, Section II-A) -- products accumulated into FP32, FP32 output.
+ *
+ * Layouts: A is M x K row-major (K contiguous). B is passed K-major as Bt[N][K]
+ * (row j of Bt is column j of B). C is M x N row-major FP32. FP16/BF16 elements
+ * are 2 bytes, TF32 elements are 4-byte FP32 words whose low 13 bits are zero.
+ * A and Bt must be 16-byte aligned and K * element_size a multiple of 16 bytes.
+ */
+#ifndef MPGEMMFI_H
+#define MPGEMMFI_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* `stream` is a cudaStream_t passed as an opaque pointer (NULL = default stream). */
+typedef void *mpgemmfi_stream;
+
+enum {
+    MPGEMMFI_FP16 = 0,
+    MPGEMMFI_BF16 = 1,
+    MPGEMMFI_TF32 = 2
+};
+
+/*
+ * Fault-site kinds. The paper's own fault is MPGEMMFI_SITE_TERM: bit flips in the
+ * result of one multiplication, carried into the running sum by the write-back
+ * of Eq. 1-2 (Section III-E, Section IV-A/IV-C). The other kinds place the same
+ * XOR on an operand element, on a running accumulator, or on an output element.
+ */
+enum {
+    MPGEMMFI_SITE_A = 0,    /* operand A[row, k]: storage bits ^= mask before the multiply   */
+    MPGEMMFI_SITE_B = 1,    /* operand B[k, col] (= Bt[col, k])                               */
+    MPGEMMFI_SITE_ACC = 2,  /* accumulator of C[row, col] after k elements were accumulated   */
+    MPGEMMFI_SITE_OUT = 3,  /* output element C[row, col] before the output check             */
+    MPGEMMFI_SITE_TERM = 4  /* product a[row,k]*b[k,col]: p' = p ^ mask; acc = (acc - p) + p' */
+};
+
+/*
+ * One entry of the fault-site descriptor table (32 bytes).
+ *   A / B : xor_mask addresses the operand's storage bits: bits 0..15 for FP16 and
+ *           BF16; for TF32 mask bit b (0..18) addresses bit b+13 of the FP32 word.
+ *   ACC   : k = number of k elements accumulated before the flip; must be a multiple
+ *           of mpgemmfi_kstep(dtype), or equal to K; 0 < k <= K. 32-bit mask.
+ *   TERM  : k = index of the term; the write-back is applied at the accumulator
+ *           boundary that ends the k-step containing k. If a product-level check is
+ *           selected it is applied to p' first (Section VI-B). 32-bit mask.
+ *   OUT   : 32-bit mask on the FP32 output word.
+ * Sites are applied in table order. `trial` is carried through for the caller.
+ */
+typedef struct {
+    uint32_t kind;
+    uint32_t row;
+    uint32_t col;
+    uint32_t k;
+    uint32_t xor_mask;
+    uint32_t trial;
+    uint32_t pad[2];
+} mpgemmfi_site;
+
+/*
+ * detect_mode: bits 1:0 select the technique (Section VI-A), bit 4 enables the
+ * correction (applied only where the detection fires, Section VI-B).
+ *   BOUNDCHECK : exponent MSB = 1 together with any of the next three exponent bits
+ *                ("1eeexxxx", some e = 1, i.e. |v| >= 131072, Table III); correction
+ *                clears the three e bits. Applied to TERM products and to every
+ *                output element; only this technique produces output flags.
+ *   RANGE_MAX  : faulty product exponent > e1 + e2 + 1; correction replaces it by
+ *                that bound. Applied to TERM products only.
+ *   RANGE_FLIP : same detection; correction clears the 1s of the exponent from its
+ *                rightmost bit until it is <= the bound. TERM products only.
+ */
+enum {
+    MPGEMMFI_DETECT_NONE = 0,
+    MPGEMMFI_DETECT_BOUNDCHECK = 1,
+    MPGEMMFI_DETECT_RANGE_MAX = 2,
+    MPGEMMFI_DETECT_RANGE_FLIP = 3,
+    MPGEMMFI_DETECT_TECHNIQUE_MASK = 3,
+    MPGEMMFI_CORRECT = 16
+};
+
+enum {
+    MPGEMMFI_OK = 0,
+    MPGEMMFI_ERR_ARG = -1,        /* null pointer, non-positive size, n_faults out of range */
+    MPGEMMFI_ERR_DTYPE = -2,
+    MPGEMMFI_ERR_ALIGN = -3,      /* pointer or row pitch not 16-byte aligned */
+    MPGEMMFI_ERR_SITE = -4,       /* mpgemmfi_validate_sites: a site is out of range */
+    MPGEMMFI_ERR_WORKSPACE = -5,  /* workspace too small or misaligned */
+    MPGEMMFI_ERR_ARCH = -6,       /* current device is not sm_100 */
+    MPGEMMFI_ERR_CUDA = -7        /* a CUDA runtime/driver call failed; see mpgemmfi_last_cuda_error() */
+};
+
+#define MPGEMMFI_MAX_FAULTS 4096      /* sites per mpgemmfi_gemm call */
+#define MPGEMMFI_HEADER_WORDS 16
+
+/* status word of the flags header */
+#define MPGEMMFI_STATUS_SITE_SKIPPED 1u  /* at least one site was invalid and skipped */
+#define MPGEMMFI_STATUS_WAIT_LIMIT 2u    /* a device-side wait ran into its time limit; results invalid */
+
+/*
+ * flags_out layout (uint32 words):
+ *   [0 .. 16)            header: [0] status, [1] n_detected, [2] n_corrected,
+ *                        [3] sites applied, [4] sites skipped, rest reserved (0)
+ *   [16 .. 16+4*n_faults) site log, one entry per table entry (the paper logs the sum
+ *                        before and after injection the same way, Section V-B):
+ *                        {before_bits, after_bits, final_bits, status}
+ *                          A/B : operand storage word before / after the XOR, final = after
+ *                          ACC : accumulator bits before / after, final = after
+ *                          TERM: product bits before / after the XOR, final = after the
+ *                                product-level check; status bit 2 = detected
+ *                          OUT : output bits before / after, final = after the output check
+ *                        status: 1 applied, 2 skipped (invalid), bit 2 detected (TERM)
+ *   [16+4*n_faults ..)   bitmap, M rows of ceil(N/32) words: bit (j mod 32) of word
+ *                        i*ceil(N/32) + j/32 is 1 iff C[i,j] was detected (and corrected
+ *                        when correction is on). Bits beyond column N-1 are 0.
+ */
+typedef struct {
+    uint32_t before_bits;
+    uint32_t after_bits;
+    uint32_t final_bits;
+    uint32_t status;
+} mpgemmfi_site_log;
+
+/*
+ * One record per campaign trial (48 bytes). A trial is one site applied alone to
+ * the clean GEMM ("a single fault is injected in each trial", Section IV-A).
+ *   status        bit0 changed (some affected element's final bits differ from the
+ *                 clean ones: the complement of the paper's "zero difference",
+ *                 Section V-B), bit1 detected, bit2 corrected, bit8 invalid site
+ *   primary_index OUT/ACC/TERM: row*N+col; A: row*K+k; B: col*K+k
+ *   before/after  the word the mask was applied to, before and after the XOR
+ *   final_bits    OUT/ACC/TERM: the output element after the check; A/B: = after_bits
+ *   n_affected    output elements re-evaluated (1, N for an A site, M for a B site)
+ *   n_detected    how many of them the output check flagged
+ *   idx_hash      sum over flagged elements of (row*N+col+1) * 0x9E3779B97F4A7C15 mod 2^64
+ *   first_detected smallest flagged row*N+col, 0xFFFFFFFF if none
+ *   max_abs_dev   max over affected elements of |final - clean| (FP32; NaN counts as +inf)
+ */
+typedef struct {
+    uint32_t status;
+    uint32_t kind;
+    uint32_t primary_index;
+    uint32_t before_bits;
+    uint32_t after_bits;
+    uint32_t final_bits;
+    uint32_t n_affected;
+    uint32_t n_detected;
+    uint64_t idx_hash;
+    uint32_t first_detected;
+    float max_abs_dev;
+} mpgemmfi_trial_record;
+
+/*
+ * Fault-injected GEMM with the fused check (Sections II-B, III-E, IV-C, VI-A).
+ *   A, Bt, C     device pointers, layouts above; C is written in full.
+ *   fault_sites  device pointer to n_faults entries (may be NULL when n_faults = 0);
+ *                0 <= n_faults <= MPGEMMFI_MAX_FAULTS.
+ *   flags_out    device pointer to mpgemmfi_flags_bytes(M, N, n_faults) bytes, 16-byte
+ *                aligned, written in full; may be NULL only when n_faults = 0 and the
+ *                technique is NONE (plain GEMM, nothing to report).
+ * Errors: ERR_ARG, ERR_DTYPE, ERR_ALIGN, ERR_ARCH, ERR_CUDA.
+ */
+int mpgemmfi_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C,
+                  const mpgemmfi_site *fault_sites, int n_faults, int detect_mode,
+                  uint32_t *flags_out, mpgemmfi_stream stream);
+
+/*
+ * Injection campaign: ONE clean GEMM, then every trial is evaluated on the output
+ * elements it can reach (Section IV-A: one fault per trial; Eq. 1-2 for how a
+ * faulty term enters a finished sum).
+ *   C_clean     device, M x N, written: the fault-free, unchecked product.
+ *   sites       device, n_trials entries, one site per trial.
+ *   records     device, n_trials records, written in full.
+ *   workspace   device scratch of at least mpgemmfi_campaign_workspace_bytes(...)
+ *               bytes, 256-byte aligned; contents undefined afterwards.
+ * OUT trials flip the clean element. ACC and TERM trials recompute their element's
+ * dot product in k order on the FP32 ALUs with the site active (and once without it,
+ * which is the trial's clean reference). A and B trials apply, to every element of the
+ * affected row or column, c' = (c - a*b) + a'*b with the clean and the faulty operand
+ * (the write-back form of Eq. 1-2 applied to a finished sum). Every re-evaluated
+ * element then goes through the output check of detect_mode.
+ * Errors: as mpgemmfi_gemm, plus ERR_WORKSPACE.
+ */
+int mpgemmfi_campaign(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C_clean,
+                      const mpgemmfi_site *sites, int n_trials, int detect_mode,
+                      mpgemmfi_trial_record *records, void *workspace, size_t workspace_bytes,
+                      mpgemmfi_stream stream);
+
+/* k elements between two accumulator boundaries: 64 (FP16, BF16), 32 (TF32); 0 for a bad dtype. */
+int mpgemmfi_kstep(int dtype);
+
+/* bytes of the flags_out buffer for an M x N output and n_faults sites */
+size_t mpgemmfi_flags_bytes(int M, int N, int n_faults);
+
+/* offset, in uint32 words, of the bitmap inside flags_out */
+size_t mpgemmfi_flags_bitmap_offset(int n_faults);
+
+size_t mpgemmfi_campaign_workspace_bytes(int dtype, int M, int N, int K, int n_trials);
+
+/*
+ * Host-side check of a HOST copy of a site table: returns MPGEMMFI_OK, or
+ * MPGEMMFI_ERR_SITE and stores the index of the first bad entry in *first_bad
+ * (if non-NULL). The device applies the same rules and skips bad entries.
+ */
+int mpgemmfi_validate_sites(const mpgemmfi_site *host_sites, int n, int dtype, int M, int N, int K,
+                            int *first_bad);
+
+const char *mpgemmfi_strerror(int code);
+
+/* cudaError_t value of the last failed CUDA call seen by this library (0 if none) */
+int mpgemmfi_last_cuda_error(void);
+
+/* major*10000 + minor*100 + patch */
+int mpgemmfi_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MPGEMMFI_H */

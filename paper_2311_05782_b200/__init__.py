@@ -1,0 +1,19 @@
+"""B200-native fault-injected mixed-precision GEMM (MPGemmFI hot path).
+
+Thin binding over the C ABI declared in include/mpgemmfi.h: the functions here
+have the same names as the library's entry points and only marshal arguments.
+All arithmetic runs in the CUDA kernels; there is no CPU fallback, and loading
+fails loudly when the CUDA library is missing.
+"""
+from .binding import (  # noqa: F401
+    FP16, BF16, TF32,
+    SITE_A, SITE_B, SITE_ACC, SITE_OUT, SITE_TERM,
+    DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP, CORRECT,
+    STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT, MAX_FAULTS, HEADER_WORDS,
+    SITE_DTYPE, SITE_LOG_DTYPE, RECORD_DTYPE,
+    MpgemmfiError, library_path, load_library, exported_symbols,
+    mpgemmfi_gemm, mpgemmfi_campaign, mpgemmfi_kstep, mpgemmfi_flags_bytes,
+    mpgemmfi_flags_bitmap_offset, mpgemmfi_campaign_workspace_bytes,
+    mpgemmfi_validate_sites, mpgemmfi_strerror, mpgemmfi_last_cuda_error, mpgemmfi_version,
+    gemm, campaign, split_flags,
+)

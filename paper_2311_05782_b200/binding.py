@@ -1,0 +1,230 @@
+"""ctypes binding of libmpgemmfi.so.
+
+`mpgemmfi_*` functions mirror the C ABI one to one (raw pointers and sizes).
+`gemm` and `campaign` are convenience wrappers that take torch CUDA tensors,
+allocate the output buffers with torch and pass `data_ptr()`s and the current
+stream; they do no arithmetic.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+FP16, BF16, TF32 = 0, 1, 2
+SITE_A, SITE_B, SITE_ACC, SITE_OUT, SITE_TERM = 0, 1, 2, 3, 4
+DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP = 0, 1, 2, 3
+CORRECT = 16
+STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT = 1, 2
+MAX_FAULTS = 4096
+HEADER_WORDS = 16
+
+SITE_DTYPE = np.dtype([("kind", "<u4"), ("row", "<u4"), ("col", "<u4"), ("k", "<u4"),
+                       ("xor_mask", "<u4"), ("trial", "<u4"), ("pad0", "<u4"), ("pad1", "<u4")])
+SITE_LOG_DTYPE = np.dtype([("before_bits", "<u4"), ("after_bits", "<u4"), ("final_bits", "<u4"), ("status", "<u4")])
+RECORD_DTYPE = np.dtype([("status", "<u4"), ("kind", "<u4"), ("primary_index", "<u4"), ("before_bits", "<u4"),
+                         ("after_bits", "<u4"), ("final_bits", "<u4"), ("n_affected", "<u4"), ("n_detected", "<u4"),
+                         ("idx_hash", "<u8"), ("first_detected", "<u4"), ("max_abs_dev", "<f4")])
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libmpgemmfi.so")
+_lib = None
+
+_SYMBOLS = [
+    "mpgemmfi_gemm", "mpgemmfi_campaign", "mpgemmfi_kstep", "mpgemmfi_flags_bytes",
+    "mpgemmfi_flags_bitmap_offset", "mpgemmfi_campaign_workspace_bytes", "mpgemmfi_validate_sites",
+    "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version",
+]
+
+
+class MpgemmfiError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        detail = ""
+        if code == -7:
+            detail = f" (cudaError {mpgemmfi_last_cuda_error()})"
+        super().__init__(f"{where}: {mpgemmfi_strerror(code)} [{code}]{detail}")
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def exported_symbols():
+    """Names every build of the library must export (the declarations of include/mpgemmfi.h)."""
+    return list(_SYMBOLS)
+
+
+def load_library():
+    """Load libmpgemmfi.so; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2311_05782_b200.build`")
+    L = C.CDLL(_LIB_PATH)
+    vp, i, sz = C.c_void_p, C.c_int, C.c_size_t
+    L.mpgemmfi_gemm.restype = i
+    L.mpgemmfi_gemm.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp]
+    L.mpgemmfi_campaign.restype = i
+    L.mpgemmfi_campaign.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp, sz, vp]
+    L.mpgemmfi_kstep.restype = i
+    L.mpgemmfi_kstep.argtypes = [i]
+    L.mpgemmfi_flags_bytes.restype = sz
+    L.mpgemmfi_flags_bytes.argtypes = [i, i, i]
+    L.mpgemmfi_flags_bitmap_offset.restype = sz
+    L.mpgemmfi_flags_bitmap_offset.argtypes = [i]
+    L.mpgemmfi_campaign_workspace_bytes.restype = sz
+    L.mpgemmfi_campaign_workspace_bytes.argtypes = [i, i, i, i, i]
+    L.mpgemmfi_validate_sites.restype = i
+    L.mpgemmfi_validate_sites.argtypes = [vp, i, i, i, i, i, C.POINTER(C.c_int)]
+    L.mpgemmfi_strerror.restype = C.c_char_p
+    L.mpgemmfi_strerror.argtypes = [i]
+    L.mpgemmfi_last_cuda_error.restype = i
+    L.mpgemmfi_version.restype = i
+    _lib = L
+    return L
+
+
+# ---------------------------------------------------------------- raw C ABI
+
+def mpgemmfi_gemm(dtype, M, N, K, A, Bt, C_out, fault_sites, n_faults, detect_mode, flags_out, stream):
+    """Raw call: every matrix argument is a device address (int), `stream` a cudaStream_t handle (int)."""
+    return load_library().mpgemmfi_gemm(dtype, M, N, K, A, Bt, C_out, fault_sites, n_faults, detect_mode,
+                                        flags_out, stream)
+
+
+def mpgemmfi_campaign(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mode, records, workspace,
+                      workspace_bytes, stream):
+    return load_library().mpgemmfi_campaign(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mode, records,
+                                            workspace, workspace_bytes, stream)
+
+
+def mpgemmfi_kstep(dtype):
+    return load_library().mpgemmfi_kstep(dtype)
+
+
+def mpgemmfi_flags_bytes(M, N, n_faults):
+    return load_library().mpgemmfi_flags_bytes(M, N, n_faults)
+
+
+def mpgemmfi_flags_bitmap_offset(n_faults):
+    return load_library().mpgemmfi_flags_bitmap_offset(n_faults)
+
+
+def mpgemmfi_campaign_workspace_bytes(dtype, M, N, K, n_trials):
+    return load_library().mpgemmfi_campaign_workspace_bytes(dtype, M, N, K, n_trials)
+
+
+def mpgemmfi_validate_sites(host_sites: np.ndarray, dtype, M, N, K):
+    """Returns (code, first_bad_index). host_sites: numpy array of 32-byte site entries."""
+    s = np.ascontiguousarray(host_sites)
+    assert s.dtype.itemsize == 32
+    bad = C.c_int(-1)
+    rc = load_library().mpgemmfi_validate_sites(s.ctypes.data_as(C.c_void_p), len(s), dtype, M, N, K, C.byref(bad))
+    return rc, bad.value
+
+
+def mpgemmfi_strerror(code):
+    return load_library().mpgemmfi_strerror(code).decode()
+
+
+def mpgemmfi_last_cuda_error():
+    return load_library().mpgemmfi_last_cuda_error()
+
+
+def mpgemmfi_version():
+    return load_library().mpgemmfi_version()
+
+
+# ---------------------------------------------------------------- torch-tensor convenience wrappers
+
+def _torch():
+    import torch
+    return torch
+
+
+def _check_operand(t, dtype, name):
+    torch = _torch()
+    want = torch.int32 if dtype == TF32 else torch.int16
+    ok = {TF32: (torch.int32, torch.float32), FP16: (torch.int16, torch.float16),
+          BF16: (torch.int16, torch.bfloat16)}[dtype]
+    if not t.is_cuda or not t.is_contiguous() or t.dim() != 2 or t.dtype not in ok:
+        raise ValueError(f"{name}: expected a contiguous 2-D CUDA tensor of dtype in {ok} (storage {want})")
+
+
+def _sites_tensor(sites, device):
+    """numpy structured array (or None) -> int32 CUDA tensor [n, 8]; tensors pass through."""
+    torch = _torch()
+    if sites is None:
+        return None, 0
+    if isinstance(sites, np.ndarray):
+        s = np.ascontiguousarray(sites)
+        assert s.dtype.itemsize == 32
+        if len(s) == 0:
+            return None, 0
+        t = torch.from_numpy(s.view(np.int32).reshape(len(s), 8)).to(device)
+        return t, len(s)
+    assert sites.is_cuda and sites.is_contiguous() and sites.dtype == torch.int32 and sites.shape[-1] == 8
+    return (sites, sites.shape[0]) if sites.shape[0] else (None, 0)
+
+
+def gemm(dtype, A, Bt, sites=None, detect_mode=DETECT_NONE, C_out=None, flags_out=None, stream=None):
+    """Fault-injected GEMM on CUDA tensors. Returns (C, flags) where flags is the raw uint32 buffer
+    (as an int32 tensor) laid out as documented in include/mpgemmfi.h; see split_flags()."""
+    torch = _torch()
+    _check_operand(A, dtype, "A")
+    _check_operand(Bt, dtype, "Bt")
+    M, K = A.shape
+    N, K2 = Bt.shape
+    if K != K2:
+        raise ValueError("A and Bt disagree on K")
+    st, n_faults = _sites_tensor(sites, A.device)
+    if C_out is None:
+        C_out = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    if flags_out is None:
+        flags_out = torch.empty(mpgemmfi_flags_bytes(M, N, n_faults) // 4, dtype=torch.int32, device=A.device)
+    stream_h = (torch.cuda.current_stream(A.device) if stream is None else stream).cuda_stream
+    rc = mpgemmfi_gemm(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), C_out.data_ptr(),
+                       st.data_ptr() if st is not None else None, n_faults, detect_mode,
+                       flags_out.data_ptr(), stream_h)
+    if rc != 0:
+        raise MpgemmfiError(rc, "mpgemmfi_gemm")
+    return C_out, flags_out
+
+
+def split_flags(flags, M, N, n_faults):
+    """Copy a flags buffer to the host and split it into (header[16], site_log[n_faults], bitmap[M, ceil(N/32)])."""
+    raw = flags.cpu().numpy().view(np.uint32)
+    off = HEADER_WORDS + 4 * n_faults
+    hdr = raw[:HEADER_WORDS].copy()
+    log = raw[HEADER_WORDS:off].copy().view(SITE_LOG_DTYPE)
+    wpr = (N + 31) // 32
+    bitmap = raw[off:off + M * wpr].reshape(M, wpr).copy()
+    return hdr, log, bitmap
+
+
+def campaign(dtype, A, Bt, sites, detect_mode=DETECT_NONE, C_clean=None, records=None, workspace=None, stream=None):
+    """Injection campaign on CUDA tensors. Returns (C_clean, records) with records an int32 tensor [n_trials, 12]
+    (view the host copy as RECORD_DTYPE)."""
+    torch = _torch()
+    _check_operand(A, dtype, "A")
+    _check_operand(Bt, dtype, "Bt")
+    M, K = A.shape
+    N, _ = Bt.shape
+    st, n_trials = _sites_tensor(sites, A.device)
+    if C_clean is None:
+        C_clean = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    if records is None:
+        records = torch.empty((max(n_trials, 1), 12), dtype=torch.int32, device=A.device)
+    ws_bytes = mpgemmfi_campaign_workspace_bytes(dtype, M, N, K, n_trials)
+    if workspace is None:
+        workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=A.device)
+    stream_h = (torch.cuda.current_stream(A.device) if stream is None else stream).cuda_stream
+    rc = mpgemmfi_campaign(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), C_clean.data_ptr(),
+                           st.data_ptr() if st is not None else None, n_trials, detect_mode,
+                           records.data_ptr(), workspace.data_ptr(), workspace.numel(), stream_h)
+    if rc != 0:
+        raise MpgemmfiError(rc, "mpgemmfi_campaign")
+    return C_clean, records[:n_trials]

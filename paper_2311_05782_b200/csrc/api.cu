@@ -1,0 +1,242 @@
+// C ABI of the library: argument checks, tensor-map encoding, kernel launches.
+#include <cstdint>
+#include <cstring>
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "../../include/mpgemmfi.h"
+#include "campaign.cuh"
+#include "checks.cuh"
+#include "gemm_sm100.cuh"
+
+namespace {
+
+int g_last_cuda_error = 0;
+
+int cuda_fail(cudaError_t e)
+{
+    g_last_cuda_error = (int)e;
+    return MPGEMMFI_ERR_CUDA;
+}
+
+struct DeviceInfo {
+    bool known = false;
+    int major = 0;
+    int num_sms = 0;
+};
+
+// properties of the current device, looked up once per device
+int device_info(DeviceInfo &out)
+{
+    static DeviceInfo cache[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= 64) return MPGEMMFI_ERR_ARG;
+    if (!cache[dev].known) {
+        e = cudaDeviceGetAttribute(&cache[dev].major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) return cuda_fail(e);
+        e = cudaDeviceGetAttribute(&cache[dev].num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail(e);
+        cache[dev].known = true;
+    }
+    out = cache[dev];
+    return MPGEMMFI_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// rows x K matrix, K contiguous; box = one 128-byte row segment x box_rows rows, 128-byte swizzle,
+// out-of-range elements read as zero
+int encode_operand_map(CUtensorMap *map, int dtype, const void *base, int rows, int K, int box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return cuda_fail(cudaErrorUnknown);
+    const int es = mpg::esize_of(dtype);
+    const CUtensorMapDataType dt = dtype == MPGEMMFI_FP16   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                   : dtype == MPGEMMFI_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                                            : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * (cuuint64_t)es};
+    const cuuint32_t box[2] = {(cuuint32_t)(128 / es), (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, dt, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return MPGEMMFI_ERR_CUDA; }
+    return MPGEMMFI_OK;
+}
+
+// widest tile that still gives every SM a tile; narrow outputs get narrow tiles
+int choose_bn(int M, int N, int num_sms)
+{
+    const int tiles_m = (M + 127) / 128;
+    const int cands[3] = {256, 128, 64};
+    for (int i = 0; i < 3; ++i) {
+        const int bn = cands[i];
+        if (i < 2 && N <= bn / 2) continue;                 // tile twice as wide as the matrix
+        if (tiles_m * ((N + bn - 1) / bn) >= num_sms || i == 2) return bn;
+    }
+    return 64;
+}
+
+int check_common(int dtype, int M, int N, int K, const void *A, const void *Bt, const void *C)
+{
+    if (dtype != MPGEMMFI_FP16 && dtype != MPGEMMFI_BF16 && dtype != MPGEMMFI_TF32) return MPGEMMFI_ERR_DTYPE;
+    if (M <= 0 || N <= 0 || K <= 0 || !A || !Bt || !C) return MPGEMMFI_ERR_ARG;
+    if ((unsigned long long)M * (unsigned long long)N >= 0xFFFFFFFFull) return MPGEMMFI_ERR_ARG;
+    const int es = mpg::esize_of(dtype);
+    if (((uintptr_t)A & 15) || ((uintptr_t)Bt & 15) || ((uintptr_t)C & 3) || ((size_t)K * es) % 16) return MPGEMMFI_ERR_ALIGN;
+    return MPGEMMFI_OK;
+}
+
+int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C, const mpgemmfi_site *sites,
+             int n_faults, int detect_mode, uint32_t *flags, cudaStream_t stream, const DeviceInfo &di)
+{
+    const int bn = choose_bn(M, N, di.num_sms);
+    CUtensorMap tm_a, tm_b;
+    int rc = encode_operand_map(&tm_a, dtype, A, M, K, 128);
+    if (rc) return rc;
+    rc = encode_operand_map(&tm_b, dtype, Bt, N, K, bn);
+    if (rc) return rc;
+
+    mpg::GemmParams p;
+    p.dtype = dtype; p.M = M; p.N = N; p.K = K;
+    p.detect_mode = detect_mode; p.n_faults = n_faults;
+    p.tiles_m = (M + 127) / 128; p.tiles_n = (N + bn - 1) / bn;
+    p.num_tiles = p.tiles_m * p.tiles_n;
+    const int ks = mpg::kstep_of(dtype);
+    p.num_kt = (K + ks - 1) / ks;
+    p.wpr = (N + 31) / 32;
+    p.c_vec_ok = (N % 4 == 0) && (((uintptr_t)C & 15) == 0);
+    p.A = A; p.Bt = Bt; p.C = C; p.sites = sites; p.flags = flags;
+
+    if (flags) {
+        const cudaError_t e = cudaMemsetAsync(flags, 0, sizeof(uint32_t) * (MPGEMMFI_HEADER_WORDS + 4 * (size_t)n_faults), stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    const int grid = p.num_tiles < di.num_sms ? p.num_tiles : di.num_sms;
+    const cudaError_t e = mpg::launch_gemm(bn, tm_a, tm_b, p, grid, stream);
+    return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
+}
+
+}  // namespace
+
+extern "C" {
+
+int mpgemmfi_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C,
+                  const mpgemmfi_site *fault_sites, int n_faults, int detect_mode, uint32_t *flags_out,
+                  mpgemmfi_stream stream)
+{
+    int rc = check_common(dtype, M, N, K, A, Bt, C);
+    if (rc) return rc;
+    if (n_faults < 0 || n_faults > MPGEMMFI_MAX_FAULTS || (n_faults > 0 && !fault_sites)) return MPGEMMFI_ERR_ARG;
+    if (detect_mode & ~(MPGEMMFI_DETECT_TECHNIQUE_MASK | MPGEMMFI_CORRECT)) return MPGEMMFI_ERR_ARG;
+    if (!flags_out && (n_faults > 0 || (detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK))) return MPGEMMFI_ERR_ARG;
+    if (((uintptr_t)fault_sites & 15) || ((uintptr_t)flags_out & 15)) return MPGEMMFI_ERR_ALIGN;
+    DeviceInfo di;
+    rc = device_info(di);
+    if (rc) return rc;
+    if (di.major != 10) return MPGEMMFI_ERR_ARCH;
+    return run_gemm(dtype, M, N, K, A, Bt, C, fault_sites, n_faults, detect_mode, flags_out,
+                    static_cast<cudaStream_t>(stream), di);
+}
+
+int mpgemmfi_campaign(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C_clean,
+                      const mpgemmfi_site *sites, int n_trials, int detect_mode, mpgemmfi_trial_record *records,
+                      void *workspace, size_t workspace_bytes, mpgemmfi_stream stream)
+{
+    int rc = check_common(dtype, M, N, K, A, Bt, C_clean);
+    if (rc) return rc;
+    if (n_trials < 0 || (n_trials > 0 && (!sites || !records))) return MPGEMMFI_ERR_ARG;
+    if (detect_mode & ~(MPGEMMFI_DETECT_TECHNIQUE_MASK | MPGEMMFI_CORRECT)) return MPGEMMFI_ERR_ARG;
+    if (((uintptr_t)sites & 15) || ((uintptr_t)records & 7)) return MPGEMMFI_ERR_ALIGN;
+    if (!workspace || ((uintptr_t)workspace & 255) ||
+        workspace_bytes < mpgemmfi_campaign_workspace_bytes(dtype, M, N, K, n_trials))
+        return MPGEMMFI_ERR_WORKSPACE;
+    DeviceInfo di;
+    rc = device_info(di);
+    if (rc) return rc;
+    if (di.major != 10) return MPGEMMFI_ERR_ARCH;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the clean product, shared by every trial
+    rc = run_gemm(dtype, M, N, K, A, Bt, C_clean, nullptr, 0, MPGEMMFI_DETECT_NONE, nullptr, st, di);
+    if (rc) return rc;
+    mpg::CampaignParams p;
+    p.dtype = dtype; p.M = M; p.N = N; p.K = K; p.detect_mode = detect_mode; p.n_trials = n_trials;
+    p.A = A; p.Bt = Bt; p.C = C_clean; p.sites = sites; p.records = records;
+    mpg::campaign_bind_schedule(p, workspace);
+    const cudaError_t e = mpg::launch_campaign_trials(p, di.num_sms, st);
+    return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
+}
+
+int mpgemmfi_kstep(int dtype)
+{
+    if (dtype != MPGEMMFI_FP16 && dtype != MPGEMMFI_BF16 && dtype != MPGEMMFI_TF32) return 0;
+    return mpg::kstep_of(dtype);
+}
+
+size_t mpgemmfi_flags_bitmap_offset(int n_faults)
+{
+    return MPGEMMFI_HEADER_WORDS + 4 * (size_t)(n_faults > 0 ? n_faults : 0);
+}
+
+size_t mpgemmfi_flags_bytes(int M, int N, int n_faults)
+{
+    if (M <= 0 || N <= 0) return 0;
+    return sizeof(uint32_t) * (mpgemmfi_flags_bitmap_offset(n_faults) + (size_t)M * (size_t)((N + 31) / 32));
+}
+
+size_t mpgemmfi_campaign_workspace_bytes(int dtype, int M, int N, int K, int n_trials)
+{
+    (void)dtype; (void)M; (void)N; (void)K;
+    return mpg::campaign_schedule_bytes(n_trials);
+}
+
+int mpgemmfi_validate_sites(const mpgemmfi_site *host_sites, int n, int dtype, int M, int N, int K, int *first_bad)
+{
+    if (dtype != MPGEMMFI_FP16 && dtype != MPGEMMFI_BF16 && dtype != MPGEMMFI_TF32) return MPGEMMFI_ERR_DTYPE;
+    if (n < 0 || (n > 0 && !host_sites) || M <= 0 || N <= 0 || K <= 0) return MPGEMMFI_ERR_ARG;
+    for (int i = 0; i < n; ++i)
+        if (!mpg::site_valid(host_sites[i], dtype, M, N, K)) {
+            if (first_bad) *first_bad = i;
+            return MPGEMMFI_ERR_SITE;
+        }
+    return MPGEMMFI_OK;
+}
+
+const char *mpgemmfi_strerror(int code)
+{
+    switch (code) {
+    case MPGEMMFI_OK: return "ok";
+    case MPGEMMFI_ERR_ARG: return "invalid argument";
+    case MPGEMMFI_ERR_DTYPE: return "unknown dtype";
+    case MPGEMMFI_ERR_ALIGN: return "pointer or row pitch not 16-byte aligned";
+    case MPGEMMFI_ERR_SITE: return "fault site out of range";
+    case MPGEMMFI_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case MPGEMMFI_ERR_ARCH: return "device is not sm_100";
+    case MPGEMMFI_ERR_CUDA: return "CUDA call failed";
+    default: return "unknown error";
+    }
+}
+
+int mpgemmfi_last_cuda_error(void) { return g_last_cuda_error; }
+
+int mpgemmfi_version(void) { return 100; }
+
+}  // extern "C"

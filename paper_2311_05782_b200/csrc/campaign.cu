@@ -1,0 +1,265 @@
+// Injection campaign: per-trial evaluation kernels that run after ONE clean GEMM.
+//
+// Every trial is one fault site applied alone. Only the output elements the site can reach
+// are evaluated:
+//   OUT        flip the clean element
+//   ACC, TERM  redo the element's dot product in k order on the FP32 ALUs, once clean and
+//              once with the site active (the clean pass is the trial's reference)
+//   A, B       c' = (c - a*b) + a'*b for every element of the affected row / column
+//              (the write-back of Eq. 1-2 applied to a finished sum)
+// and every evaluated element goes through the output check.
+//
+// Scratch (the "schedule"): three compacted lists of trial indices (A sites, B sites,
+// single-element sites) plus their counters, so that each evaluation kernel walks only its
+// own kind of trial.
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "campaign.cuh"
+#include "checks.cuh"
+
+namespace mpg {
+
+namespace {
+
+constexpr unsigned long long HASH_MUL = 0x9E3779B97F4A7C15ull;
+constexpr int VEC_THREADS = 256;
+
+struct Stats {
+    uint32_t n_det;
+    uint32_t first;
+    uint32_t maxdev_bits;   // non-negative floats order like their bit patterns
+    uint32_t changed;
+    unsigned long long hash;
+};
+
+__device__ __forceinline__ void stats_init(Stats &s)
+{
+    s.n_det = 0; s.first = 0xFFFFFFFFu; s.maxdev_bits = 0; s.changed = 0; s.hash = 0ull;
+}
+
+// run the output check on one evaluated element and fold it into the trial's statistics
+__device__ __forceinline__ uint32_t stats_account(Stats &s, int detect_mode, uint32_t value_bits, uint32_t clean_bits,
+                                                  uint32_t lin)
+{
+    bool det;
+    const uint32_t fin = output_check(detect_mode, value_bits, det);
+    if (det) {
+        s.n_det++;
+        s.hash += ((unsigned long long)lin + 1ull) * HASH_MUL;
+        s.first = min(s.first, lin);
+    }
+    if (fin != clean_bits) s.changed = 1;
+    float dev = fabsf(__fsub_rn(bits_f32(fin), bits_f32(clean_bits)));
+    if (dev != dev) dev = __uint_as_float(0x7F800000u);      // NaN deviation counts as +inf
+    s.maxdev_bits = max(s.maxdev_bits, f32_bits(dev));
+    return fin;
+}
+
+__device__ __forceinline__ void stats_warp_reduce(Stats &s)
+{
+    s.n_det = __reduce_add_sync(0xFFFFFFFFu, s.n_det);
+    s.first = __reduce_min_sync(0xFFFFFFFFu, s.first);
+    s.maxdev_bits = __reduce_max_sync(0xFFFFFFFFu, s.maxdev_bits);
+    s.changed = __reduce_or_sync(0xFFFFFFFFu, s.changed);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s.hash += __shfl_xor_sync(0xFFFFFFFFu, s.hash, o);
+}
+
+__device__ __forceinline__ uint32_t status_bits(const Stats &s, int detect_mode)
+{
+    const bool corr = (detect_mode & MPGEMMFI_CORRECT) &&
+                      (detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK) == MPGEMMFI_DETECT_BOUNDCHECK;
+    return (s.changed ? 1u : 0u) | (s.n_det ? 2u : 0u) | ((s.n_det && corr) ? 4u : 0u);
+}
+
+// ---------------------------------------------------------------- schedule
+
+__global__ void schedule_kernel(CampaignParams p)
+{
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= p.n_trials) return;
+    const mpgemmfi_site s = load_site(p.sites, t);
+    mpgemmfi_trial_record r;
+    r.status = 0; r.kind = s.kind; r.primary_index = 0; r.before_bits = 0; r.after_bits = 0; r.final_bits = 0;
+    r.n_affected = 0; r.n_detected = 0; r.idx_hash = 0ull; r.first_detected = 0xFFFFFFFFu; r.max_abs_dev = 0.0f;
+    if (!site_valid(s, p.dtype, p.M, p.N, p.K)) {
+        r.status = 1u << 8;
+    } else if (s.kind == MPGEMMFI_SITE_A || s.kind == MPGEMMFI_SITE_B) {
+        const bool is_a = s.kind == MPGEMMFI_SITE_A;
+        const size_t pos = (size_t)(is_a ? s.row : s.col) * p.K + s.k;
+        const uint32_t before = load_operand(p.dtype, is_a ? p.A : p.Bt, pos);
+        const uint32_t after = flip_operand(p.dtype, before, s.xor_mask);
+        r.primary_index = (uint32_t)pos; r.before_bits = before; r.after_bits = after; r.final_bits = after;
+        r.n_affected = is_a ? (uint32_t)p.N : (uint32_t)p.M;
+        uint32_t *cnt = p.counters + (is_a ? 0 : 1);
+        uint32_t *list = is_a ? p.list_a : p.list_b;
+        list[atomicAdd(cnt, 1u)] = (uint32_t)t;
+    } else {
+        r.primary_index = s.row * (uint32_t)p.N + s.col;
+        r.n_affected = 1;
+        p.list_e[atomicAdd(p.counters + 2, 1u)] = (uint32_t)t;
+    }
+    p.records[t] = r;
+}
+
+// ---------------------------------------------------------------- single-element trials (one warp each)
+
+__global__ void __launch_bounds__(256) element_kernel(CampaignParams p)
+{
+    const int lane = threadIdx.x & 31;
+    const uint32_t warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t n_warps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t count = p.counters[2];
+    const uint32_t ks = (uint32_t)kstep_of(p.dtype);
+    for (uint32_t w = warp_global; w < count; w += n_warps) {
+        const uint32_t t = p.list_e[w];
+        const mpgemmfi_site s = load_site(p.sites, t);
+        const uint32_t lin = s.row * (uint32_t)p.N + s.col;
+        uint32_t before, after, value_bits, clean_bits;
+        if (s.kind == MPGEMMFI_SITE_OUT) {
+            clean_bits = f32_bits(p.C[lin]);
+            before = clean_bits;
+            after = before ^ s.xor_mask;
+            value_bits = after;
+        } else {
+            // where the site takes effect, in accumulated k elements
+            uint32_t kb;
+            float re2 = 0.0f, a_site = 0.0f, b_site = 0.0f;
+            if (s.kind == MPGEMMFI_SITE_ACC) kb = s.k;
+            else {
+                kb = min((uint32_t)p.K, (s.k / ks + 1u) * ks);
+                a_site = widen_operand(p.dtype, load_operand(p.dtype, p.A, (size_t)s.row * p.K + s.k));
+                b_site = widen_operand(p.dtype, load_operand(p.dtype, p.Bt, (size_t)s.col * p.K + s.k));
+                re2 = __fmul_rn(a_site, b_site);
+            }
+            float acc_c = 0.0f, acc_f = 0.0f;
+            before = 0; after = 0;
+            for (uint32_t k0 = 0; k0 < (uint32_t)p.K; k0 += 32) {
+                const uint32_t k = k0 + lane;
+                float prod = 0.0f;
+                if (k < (uint32_t)p.K) {
+                    const float a = widen_operand(p.dtype, load_operand(p.dtype, p.A, (size_t)s.row * p.K + k));
+                    const float b = widen_operand(p.dtype, load_operand(p.dtype, p.Bt, (size_t)s.col * p.K + k));
+                    prod = __fmul_rn(a, b);
+                }
+                const uint32_t n_here = min(32u, (uint32_t)p.K - k0);
+                for (uint32_t j = 0; j < n_here; ++j) {
+                    const float pj = __shfl_sync(0xFFFFFFFFu, prod, j);
+                    acc_c = __fadd_rn(acc_c, pj);
+                    acc_f = __fadd_rn(acc_f, pj);
+                    if (k0 + j + 1 == kb) {
+                        if (s.kind == MPGEMMFI_SITE_ACC) {
+                            before = f32_bits(acc_f);
+                            after = before ^ s.xor_mask;
+                            acc_f = bits_f32(after);
+                        } else {
+                            before = f32_bits(re2);
+                            after = before ^ s.xor_mask;
+                            bool det;
+                            const uint32_t fin = product_check(p.detect_mode, after, f32_bits(a_site), f32_bits(b_site), det);
+                            acc_f = __fadd_rn(__fsub_rn(acc_f, re2), bits_f32(fin));
+                        }
+                    }
+                }
+            }
+            clean_bits = f32_bits(acc_c);
+            value_bits = f32_bits(acc_f);
+        }
+        if (lane == 0) {
+            Stats st;
+            stats_init(st);
+            const uint32_t fin = stats_account(st, p.detect_mode, value_bits, clean_bits, lin);
+            mpgemmfi_trial_record *r = &p.records[t];
+            r->before_bits = before; r->after_bits = after; r->final_bits = fin;
+            r->n_detected = st.n_det; r->idx_hash = st.hash; r->first_detected = st.first;
+            r->max_abs_dev = bits_f32(st.maxdev_bits);
+            r->status = status_bits(st, p.detect_mode);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- operand trials (one CTA each)
+
+// which = 0: A-site trials (row i fixed, walk the N columns); which = 1: B-site trials
+// (column j fixed, walk the M rows).
+__global__ void __launch_bounds__(VEC_THREADS) vector_kernel(CampaignParams p, int which)
+{
+    __shared__ Stats warp_stats[VEC_THREADS / 32];
+    const uint32_t count = p.counters[which];
+    const uint32_t *list = which == 0 ? p.list_a : p.list_b;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (uint32_t w = blockIdx.x; w < count; w += gridDim.x) {
+        const uint32_t t = list[w];
+        const mpgemmfi_site s = load_site(p.sites, t);
+        const bool is_a = which == 0;
+        const size_t pos = (size_t)(is_a ? s.row : s.col) * p.K + s.k;
+        const uint32_t w_clean = load_operand(p.dtype, is_a ? p.A : p.Bt, pos);
+        const float x = widen_operand(p.dtype, w_clean);
+        const float xf = widen_operand(p.dtype, flip_operand(p.dtype, w_clean, s.xor_mask));
+        const uint32_t n_other = is_a ? (uint32_t)p.N : (uint32_t)p.M;
+        const void *other = is_a ? p.Bt : p.A;
+        Stats st;
+        stats_init(st);
+        for (uint32_t o = threadIdx.x; o < n_other; o += VEC_THREADS) {
+            const float y = widen_operand(p.dtype, load_operand(p.dtype, other, (size_t)o * p.K + s.k));
+            const uint32_t lin = is_a ? s.row * (uint32_t)p.N + o : o * (uint32_t)p.N + s.col;
+            const float c = p.C[lin];
+            const float rep = __fsub_rn(c, __fmul_rn(x, y));        // Eq. 1 on the finished sum
+            const float cf = __fadd_rn(rep, __fmul_rn(xf, y));      // Eq. 2
+            stats_account(st, p.detect_mode, f32_bits(cf), f32_bits(c), lin);
+        }
+        stats_warp_reduce(st);
+        if (lane == 0) warp_stats[warp] = st;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            Stats tot = warp_stats[0];
+            for (int i = 1; i < VEC_THREADS / 32; ++i) {
+                tot.n_det += warp_stats[i].n_det;
+                tot.first = min(tot.first, warp_stats[i].first);
+                tot.maxdev_bits = max(tot.maxdev_bits, warp_stats[i].maxdev_bits);
+                tot.changed |= warp_stats[i].changed;
+                tot.hash += warp_stats[i].hash;
+            }
+            mpgemmfi_trial_record *r = &p.records[t];
+            r->n_detected = tot.n_det; r->idx_hash = tot.hash; r->first_detected = tot.first;
+            r->max_abs_dev = bits_f32(tot.maxdev_bits);
+            r->status = status_bits(tot, p.detect_mode);
+        }
+        __syncthreads();
+    }
+}
+
+}  // namespace
+
+size_t campaign_schedule_bytes(int n_trials)
+{
+    const size_t lists = 3 * sizeof(uint32_t) * (size_t)(n_trials > 0 ? n_trials : 0);
+    return (256 + lists + 255) / 256 * 256;
+}
+
+void campaign_bind_schedule(CampaignParams &p, void *scratch)
+{
+    uint32_t *w = static_cast<uint32_t *>(scratch);
+    p.counters = w;
+    p.list_a = w + 64;
+    p.list_b = p.list_a + p.n_trials;
+    p.list_e = p.list_b + p.n_trials;
+}
+
+cudaError_t launch_campaign_trials(const CampaignParams &p, int num_sms, cudaStream_t stream)
+{
+    if (p.n_trials <= 0) return cudaSuccess;
+    cudaError_t e = cudaMemsetAsync(p.counters, 0, 256, stream);
+    if (e != cudaSuccess) return e;
+    schedule_kernel<<<(p.n_trials + 255) / 256, 256, 0, stream>>>(p);
+    const int max_ctas = num_sms * 8;
+    const int grid_e = min((p.n_trials + 7) / 8, max_ctas);
+    element_kernel<<<grid_e, 256, 0, stream>>>(p);
+    const int grid_v = min(p.n_trials, max_ctas);
+    vector_kernel<<<grid_v, VEC_THREADS, 0, stream>>>(p, 0);
+    vector_kernel<<<grid_v, VEC_THREADS, 0, stream>>>(p, 1);
+    return cudaGetLastError();
+}
+
+}  // namespace mpg

@@ -1,0 +1,82 @@
+"""GPU parity: mpgemmfi_campaign through the C ABI against the oracle's incremental trial evaluation."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2311_05782_b200 as mpg
+import synth
+from parity import check_campaign_against_oracle, run_gpu_campaign, run_gpu_gemm, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,shape,trials", [
+    ("c1", (256, 256, 256), 64),
+    ("c2", (384, 640, 512), 128),
+    ("c3a", (512, 384, 256), 256),
+    ("c3b", (512, 256, 512), 256),
+    ("c4", (256, 384, 544), 128),
+    ("c5", (3000, 64, 576), 300),
+])
+def test_campaign_records_on_config_mixes(name, shape, trials):
+    M, N, K = shape
+    w = synth.make_workload(name, M, N, K, trials=trials)
+    check_campaign_against_oracle(w.dtype, w.A, w.Bt, w.sites, w.detect_mode, max_fragile=2)
+
+
+@pytest.mark.parametrize("tech", [orc.T_NONE, orc.T_BOUND, orc.T_RMAX, orc.T_RFLIP])
+@pytest.mark.parametrize("nbits", [1, 2, 4])
+def test_campaign_term_trials(tech, nbits):
+    """The paper's own fault (1, 2 or 4 bits of one product, Section IV-C) under each technique."""
+    M, N, K = 256, 256, 256
+    A, Bt = synth.make_operands("c2", M, N, K)
+    sites = synth.make_sites("term", orc.BF16, M, N, K, 256, 77 + nbits, nbits=nbits)
+    check_campaign_against_oracle(orc.BF16, A, Bt, sites, tech | orc.CORRECT)
+    check_campaign_against_oracle(orc.BF16, A, Bt, sites, tech)
+
+
+def test_campaign_record_matches_single_site_gemm():
+    """Consistency inside the CUDA path: a trial's record against mpgemmfi_gemm run with that one site."""
+    w = synth.make_workload("c5", 1024, 64, 576, trials=60)
+    Cc, rec = run_gpu_campaign(w.dtype, w.A, w.Bt, w.sites, w.detect_mode)
+    for t in range(0, 60, 3):
+        s = w.sites[t:t + 1]
+        Cg, hdr, log, bm = run_gpu_gemm(w.dtype, w.A, w.Bt, s, w.detect_mode)
+        kind = int(s["kind"][0])
+        if kind == orc.KIND_OUT:
+            assert rec[t]["before_bits"] == log["before_bits"][0] and rec[t]["after_bits"] == log["after_bits"][0]
+            assert rec[t]["final_bits"] == log["final_bits"][0]
+            assert rec[t]["n_detected"] == hdr[1]
+        elif kind in (orc.KIND_A, orc.KIND_B):
+            assert rec[t]["before_bits"] == log["before_bits"][0] and rec[t]["after_bits"] == log["after_bits"][0]
+            assert abs(int(rec[t]["n_detected"]) - int(hdr[1])) <= 1
+        else:
+            assert abs(int(rec[t]["n_detected"]) - int(hdr[1])) <= 1
+
+
+def test_campaign_edge_cases():
+    A, Bt = synth.make_operands("c1", 128, 128, 64)
+    a, b = to_dev(A, orc.FP16), to_dev(Bt, orc.FP16)
+    # no trials: only the clean product is written
+    Cc, rec = mpg.campaign(orc.FP16, a, b, None, orc.T_BOUND)
+    torch.cuda.synchronize()
+    Co, *_ = orc.gemm(orc.FP16, A, Bt)
+    assert np.allclose(Cc.cpu().numpy(), Co, atol=1e-5) and rec.shape[0] == 0
+    # invalid sites are reported in the record, valid ones still evaluated
+    s = np.zeros(3, dtype=orc.SITE)
+    s["kind"] = [orc.KIND_OUT, orc.KIND_ACC, 9]
+    s["row"] = [500, 1, 0]; s["k"] = [0, 33, 0]; s["xor_mask"] = 1 << 30
+    _, rec = run_gpu_campaign(orc.FP16, A, Bt, s, orc.T_BOUND)
+    assert all(r["status"] & 0x100 for r in rec)
+    # workspace too small / misaligned
+    c = torch.empty((128, 128), dtype=torch.float32, device="cuda")
+    r = torch.empty((4, 12), dtype=torch.int32, device="cuda")
+    ws = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    st = torch.from_numpy(s.view(np.int32).reshape(3, 8)).cuda()
+    cs = torch.cuda.current_stream().cuda_stream
+    assert mpg.mpgemmfi_campaign(0, 128, 128, 64, a.data_ptr(), b.data_ptr(), c.data_ptr(), st.data_ptr(), 3, 1,
+                                 r.data_ptr(), ws.data_ptr(), 16, cs) == -5
+    assert mpg.mpgemmfi_campaign(0, 128, 128, 64, a.data_ptr(), b.data_ptr(), c.data_ptr(), st.data_ptr(), 3, 1,
+                                 r.data_ptr(), ws.data_ptr() + 8, 2048, cs) == -5
+    torch.cuda.synchronize()

@@ -1,0 +1,213 @@
+"""GPU parity: mpgemmfi_gemm through the C ABI against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2311_05782_b200 as mpg
+import synth
+from parity import (check_gemm_against_oracle, run_gpu_gemm, to_dev, close, TOL)
+
+pytestmark = pytest.mark.gpu
+
+DTYPES = [orc.FP16, orc.BF16, orc.TF32]
+
+
+def site(kind, row=0, col=0, k=0, mask=0):
+    s = np.zeros(1, dtype=orc.SITE)
+    s["kind"], s["row"], s["col"], s["k"], s["xor_mask"] = kind, row, col, k, mask
+    return s
+
+
+def rand_operands(dtype, M, N, K, seed, scale=1.0):
+    rng = np.random.default_rng(seed)
+    a = (rng.standard_normal((M, K)) * scale).astype(np.float32)
+    b = (rng.standard_normal((N, K)) * scale).astype(np.float32)
+    return synth.round_to_storage(a, dtype), synth.round_to_storage(b, dtype)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_exact_integer_gemm_single_tile(dtype):
+    """Small integers: the tensor-core result must be exactly the integer product (layout, swizzle, descriptors)."""
+    M, N, K = 128, 256, 128
+    rng = np.random.default_rng(11)
+    a = rng.integers(-4, 5, size=(M, K)).astype(np.float32)
+    b = rng.integers(-4, 5, size=(N, K)).astype(np.float32)
+    A, Bt = synth.round_to_storage(a, dtype), synth.round_to_storage(b, dtype)
+    Cg, hdr, log, bm = run_gpu_gemm(dtype, A, Bt, None, orc.T_BOUND)
+    ref = a.astype(np.int64) @ b.astype(np.int64).T
+    assert np.array_equal(Cg.astype(np.int64), ref)
+    assert hdr[0] == 0 and hdr[1] == 0 and not bm.any()
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", [(128, 64, 64), (300, 200, 136), (1000, 520, 72), (257, 129, 8 * 33), (64, 1040, 512)])
+def test_clean_gemm_with_ragged_tiles(dtype, shape):
+    M, N, K = shape
+    A, Bt = rand_operands(dtype, M, N, K, 12)
+    check_gemm_against_oracle(dtype, A, Bt, None, orc.T_BOUND | orc.CORRECT)
+
+
+def test_plain_gemm_without_flags_buffer():
+    A, Bt = rand_operands(orc.BF16, 256, 256, 256, 13)
+    Cg = torch.empty((256, 256), dtype=torch.float32, device="cuda")
+    rc = mpg.mpgemmfi_gemm(orc.BF16, 256, 256, 256, to_dev(A, orc.BF16).data_ptr(), to_dev(Bt, orc.BF16).data_ptr(),
+                           Cg.data_ptr(), None, 0, 0, None, torch.cuda.current_stream().cuda_stream)
+    assert rc == 0
+    torch.cuda.synchronize()
+    Co, *_ = orc.gemm(orc.BF16, A, Bt)
+    assert close(Cg.cpu().numpy(), Co, TOL * orc.absprod(orc.BF16, A, Bt)).all()
+
+
+def test_argument_errors_are_reported_not_launched():
+    A, Bt = rand_operands(orc.BF16, 128, 128, 64, 14)
+    a, b = to_dev(A, orc.BF16), to_dev(Bt, orc.BF16)
+    c = torch.empty((128, 128), dtype=torch.float32, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    f = torch.empty(mpg.mpgemmfi_flags_bytes(128, 128, 0) // 4, dtype=torch.int32, device="cuda")
+    assert mpg.mpgemmfi_gemm(7, 128, 128, 64, a.data_ptr(), b.data_ptr(), c.data_ptr(), None, 0, 0, f.data_ptr(), st) == -2
+    assert mpg.mpgemmfi_gemm(1, 0, 128, 64, a.data_ptr(), b.data_ptr(), c.data_ptr(), None, 0, 0, f.data_ptr(), st) == -1
+    assert mpg.mpgemmfi_gemm(1, 128, 128, 64, a.data_ptr() + 2, b.data_ptr(), c.data_ptr(), None, 0, 0, f.data_ptr(), st) == -3
+    assert mpg.mpgemmfi_gemm(1, 128, 128, 60, a.data_ptr(), b.data_ptr(), c.data_ptr(), None, 0, 0, f.data_ptr(), st) == -3
+    assert mpg.mpgemmfi_gemm(1, 128, 128, 64, a.data_ptr(), b.data_ptr(), c.data_ptr(), None, 1, 0, f.data_ptr(), st) == -1
+    assert mpg.mpgemmfi_gemm(1, 128, 128, 64, a.data_ptr(), b.data_ptr(), c.data_ptr(), None, 0, 1, None, st) == -1
+    torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_every_bit_of_one_output_element(dtype):
+    M, N, K = 256, 256, 128
+    A, Bt = rand_operands(dtype, M, N, K, 15)
+    sites = np.concatenate([site(orc.KIND_OUT, 200 + (b % 3), 7 * b + 1, 0, 1 << b) for b in range(32)])
+    check_gemm_against_oracle(dtype, A, Bt, sites, orc.T_BOUND)
+    check_gemm_against_oracle(dtype, A, Bt, sites, orc.T_BOUND | orc.CORRECT)
+    check_gemm_against_oracle(dtype, A, Bt, sites, orc.T_NONE)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_operand_sites_corners_and_every_bit(dtype):
+    M, N, K = 384, 512, 192
+    A, Bt = rand_operands(dtype, M, N, K, 16, scale=0.25)
+    width = 19 if dtype == orc.TF32 else 16
+    parts = []
+    for b in range(width):
+        parts.append(site(orc.KIND_A, (37 * b) % M, 0, (11 * b) % K, 1 << b))
+        parts.append(site(orc.KIND_B, 0, (53 * b) % N, (13 * b + 5) % K, 1 << b))
+    parts += [site(orc.KIND_A, 0, 0, 0, 1 << (width - 2)), site(orc.KIND_A, M - 1, 0, K - 1, 1 << (width - 2)),
+              site(orc.KIND_B, 0, 0, 0, 1 << (width - 2)), site(orc.KIND_B, 0, N - 1, K - 1, 1 << (width - 2)),
+              site(orc.KIND_A, 5, 0, 70, 0x3), site(orc.KIND_A, 5, 0, 70, 0x3)]      # the last two cancel
+    sites = np.concatenate(parts)
+    check_gemm_against_oracle(dtype, A, Bt, sites, orc.T_BOUND | orc.CORRECT, max_fragile=0)
+    check_gemm_against_oracle(dtype, A, Bt, sites, orc.T_BOUND)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_accumulator_sites_at_every_boundary(dtype):
+    kt = synth.kstep(dtype)
+    M, N, K = 256, 320, 5 * kt + kt // 2          # ragged last k-step: the boundary k = K is allowed
+    A, Bt = rand_operands(dtype, M, N, K, 17)
+    parts = []
+    for b in range(1, 6):
+        parts.append(site(orc.KIND_ACC, (61 * b) % M, (97 * b) % N, b * kt, 1 << (20 + b)))
+    parts.append(site(orc.KIND_ACC, 255, 319, K, 1 << 30))
+    parts.append(site(orc.KIND_ACC, 0, 0, kt, 3 << 29))
+    parts.append(site(orc.KIND_ACC, 130, 300, 2 * kt, 1 << 31))
+    parts.append(site(orc.KIND_ACC, 130, 300, 4 * kt, 1 << 22))      # same element, two boundaries
+    parts.append(site(orc.KIND_ACC, 3, 3, kt + 1, 1 << 30))           # not on a boundary: skipped on the GPU
+    sites = np.concatenate(parts)
+    # the oracle accepts any k; give it only what the GPU interface admits, then check the skip separately
+    Cg, hdr, log, bm = run_gpu_gemm(dtype, A, Bt, sites, orc.T_BOUND)
+    assert hdr[4] == 1 and hdr[0] & mpg.STATUS_SITE_SKIPPED and log["status"][-1] == 2
+    check_gemm_against_oracle(dtype, A, Bt, sites[:-1], orc.T_BOUND, max_fragile=1)
+    check_gemm_against_oracle(dtype, A, Bt, sites[:-1], orc.T_BOUND | orc.CORRECT, max_fragile=1)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("tech", [orc.T_NONE, orc.T_BOUND, orc.T_RMAX, orc.T_RFLIP])
+def test_term_sites_with_each_technique(dtype, tech):
+    kt = synth.kstep(dtype)
+    M, N, K = 128, 192, 3 * kt
+    A, Bt = rand_operands(dtype, M, N, K, 18)
+    rng = np.random.default_rng(19)
+    parts = []
+    for n in range(24):
+        nb = (1, 2, 4)[n % 3]
+        start = int(rng.integers(0, 33 - nb))
+        parts.append(site(orc.KIND_TERM, int(rng.integers(0, M)), int(rng.integers(0, N)), int(rng.integers(0, K)),
+                          ((1 << nb) - 1) << start))
+    parts.append(site(orc.KIND_TERM, 127, 191, K - 1, 1 << 30))
+    parts.append(site(orc.KIND_TERM, 0, 0, 0, 1 << 30))
+    sites = np.concatenate(parts)
+    for corr in (0, orc.CORRECT):
+        check_gemm_against_oracle(dtype, A, Bt, sites, tech | corr, max_fragile=0)
+
+
+def test_term_site_sees_a_faulty_operand():
+    kt = 64
+    A, Bt = rand_operands(orc.BF16, 128, 128, 2 * kt, 20)
+    sites = np.concatenate([site(orc.KIND_A, 9, 0, 70, 1 << 14), site(orc.KIND_TERM, 9, 17, 70, 1 << 3),
+                            site(orc.KIND_B, 0, 40, 5, 1 << 15), site(orc.KIND_TERM, 77, 40, 5, 1 << 29)])
+    check_gemm_against_oracle(orc.BF16, A, Bt, sites, orc.T_RMAX | orc.CORRECT)
+    check_gemm_against_oracle(orc.BF16, A, Bt, sites, orc.T_BOUND | orc.CORRECT)
+
+
+def test_boundcheck_over_all_256_exponents():
+    """Outputs on every FP32 exponent: products 2^(i-64) * 2^(j-32) * (1 + j/64), and all 256 exponents via OUT sites."""
+    M, N, K = 128, 64, 64
+    a = np.zeros((M, K), dtype=np.float32)
+    b = np.zeros((N, K), dtype=np.float32)
+    a[:, 0] = np.ldexp(1.0, np.arange(M) - 64)
+    b[:, 0] = np.ldexp(1.0 + np.arange(N) / 64.0, np.arange(N) - 32)
+    A, Bt = synth.round_to_storage(a, orc.BF16), synth.round_to_storage(b, orc.BF16)
+    Cg, hdr, log, bm = run_gpu_gemm(orc.BF16, A, Bt, None, orc.T_BOUND)
+    assert hdr[1] == (np.abs(Cg) >= 131072.0).sum() > 500
+    check_gemm_against_oracle(orc.BF16, A, Bt, None, orc.T_BOUND)
+    check_gemm_against_oracle(orc.BF16, A, Bt, None, orc.T_BOUND | orc.CORRECT)
+    z = np.zeros((128, 64), dtype=np.uint16)
+    zb = np.zeros((64, 64), dtype=np.uint16)
+    sites = np.concatenate([site(orc.KIND_OUT, e % 128, e // 4, 0, (e << 23) | (0x155555 if e % 2 else 0))
+                            for e in range(256)])
+    check_gemm_against_oracle(orc.BF16, z, zb, sites, orc.T_BOUND)
+    check_gemm_against_oracle(orc.BF16, z, zb, sites, orc.T_BOUND | orc.CORRECT)
+
+
+def test_many_sites_on_one_element_and_determinism():
+    A, Bt = rand_operands(orc.FP16, 128, 128, 128, 21)
+    sites = np.concatenate([site(orc.KIND_OUT, 5, 6, 0, 1 << 30), site(orc.KIND_OUT, 5, 6, 0, 1 << 29),
+                            site(orc.KIND_ACC, 5, 6, 64, 1 << 31), site(orc.KIND_TERM, 5, 6, 100, 1 << 25),
+                            site(orc.KIND_OUT, 5, 6, 0, 1 << 30)])
+    check_gemm_against_oracle(orc.FP16, A, Bt, sites, orc.T_BOUND | orc.CORRECT, max_fragile=1)
+    r1 = run_gpu_gemm(orc.FP16, A, Bt, sites, orc.T_BOUND)
+    r2 = run_gpu_gemm(orc.FP16, A, Bt, sites, orc.T_BOUND)
+    for x, y in zip(r1, r2):
+        assert np.array_equal(np.asarray(x).view(np.uint8), np.asarray(y).view(np.uint8))
+
+
+def test_injection_disabled_equals_empty_table_bitwise():
+    A, Bt = rand_operands(orc.BF16, 512, 512, 512, 22)
+    c0, *_ = run_gpu_gemm(orc.BF16, A, Bt, None, orc.T_NONE)
+    c1, hdr, log, bm = run_gpu_gemm(orc.BF16, A, Bt, site(orc.KIND_OUT, 9999, 0, 0, 1), orc.T_BOUND)
+    assert np.array_equal(c0.view(np.uint32), c1.view(np.uint32)) and hdr[4] == 1 and hdr[3] == 0
+
+
+@pytest.mark.parametrize("name,shape,trials", [
+    ("c1", (256, 256, 256), 64),
+    ("c2", (512, 768, 512), 96),
+    ("c3a", (640, 512, 256), 128),
+    ("c3b", (640, 256, 512), 128),
+    ("c4", (384, 512, 256), 96),
+    ("c5", (2048, 64, 576), 128),
+])
+def test_config_tables_in_one_gemm(name, shape, trials):
+    """The configs' site mixes at reduced sizes, all sites of the table applied in one call."""
+    M, N, K = shape
+    w = synth.make_workload(name, M, N, K, trials=trials)
+    check_gemm_against_oracle(w.dtype, w.A, w.Bt, w.sites, w.detect_mode, max_fragile=1)
+
+
+def test_maximum_site_count():
+    w = synth.make_workload("c5", 1024, 64, 192, trials=mpg.MAX_FAULTS, mix="out")
+    check_gemm_against_oracle(w.dtype, w.A, w.Bt, w.sites, w.detect_mode, max_fragile=2)
+    a, b = to_dev(w.A, w.dtype), to_dev(w.Bt, w.dtype)
+    with pytest.raises(mpg.MpgemmfiError):
+        mpg.gemm(w.dtype, a, b, np.zeros(mpg.MAX_FAULTS + 1, dtype=orc.SITE), 0)

@@ -1,0 +1,54 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every declared symbol, and its host helpers work."""
+import ctypes
+import os
+import re
+
+import numpy as np
+
+import paper_2311_05782_b200 as mpg
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "mpgemmfi.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mpgemmfi_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2311_05782_b200.build import build
+    lib = ctypes.CDLL(build())
+    names = declared_symbols()
+    assert "mpgemmfi_gemm" in names and "mpgemmfi_campaign" in names
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in the header but not exported"
+    assert sorted(mpg.exported_symbols()) == [n for n in names if n in mpg.exported_symbols()]
+    for n in names:
+        assert n in mpg.exported_symbols(), f"{n} has no Python binding"
+
+
+def test_host_helpers():
+    assert mpg.mpgemmfi_version() >= 100
+    assert [mpg.mpgemmfi_kstep(d) for d in (0, 1, 2, 3)] == [64, 64, 32, 0]
+    assert mpg.mpgemmfi_flags_bitmap_offset(5) == 16 + 20
+    assert mpg.mpgemmfi_flags_bytes(10, 33, 5) == 4 * (36 + 10 * 2)
+    assert mpg.mpgemmfi_campaign_workspace_bytes(0, 8, 8, 8, 1000) % 256 == 0
+    assert mpg.mpgemmfi_campaign_workspace_bytes(0, 8, 8, 8, 1000) >= 12000
+    assert "align" in mpg.mpgemmfi_strerror(-3)
+    # struct sizes the ABI promises
+    assert mpg.SITE_DTYPE.itemsize == 32 and mpg.SITE_LOG_DTYPE.itemsize == 16 and mpg.RECORD_DTYPE.itemsize == 48
+
+
+def test_validate_sites_rules():
+    s = np.zeros(6, dtype=mpg.SITE_DTYPE)
+    s["kind"] = [mpg.SITE_A, mpg.SITE_B, mpg.SITE_ACC, mpg.SITE_OUT, mpg.SITE_TERM, mpg.SITE_ACC]
+    s["row"] = [3, 0, 3, 3, 3, 3]; s["col"] = [0, 4, 4, 4, 4, 4]; s["k"] = [99, 99, 64, 0, 99, 100]
+    assert mpg.mpgemmfi_validate_sites(s, mpg.BF16, 8, 8, 100) == (0, -1)       # k = K is a legal ACC boundary
+    s["k"][2] = 65
+    assert mpg.mpgemmfi_validate_sites(s, mpg.BF16, 8, 8, 100) == (-4, 2)        # not on a k-step boundary
+    s["k"][2] = 32
+    assert mpg.mpgemmfi_validate_sites(s, mpg.TF32, 8, 8, 100) == (0, -1)        # TF32 k-step is 32
+    s["row"][3] = 8
+    assert mpg.mpgemmfi_validate_sites(s, mpg.TF32, 8, 8, 100) == (-4, 3)
+    assert mpg.mpgemmfi_validate_sites(s, 5, 8, 8, 100)[0] == -2
