@@ -82,6 +82,7 @@ def check_gemm_against_oracle(dtype, A, Bt, sites, mode, max_fragile=0):
     assert hdr_g[3] == hdr_o[3] and hdr_g[4] == hdr_o[4]
     assert bool(hdr_g[0] & 1) == bool(hdr_o[0] & 1)
     fragile_elems = set()
+    seen = {}
     for t, s in enumerate(sites):
         if not valid[t]:
             continue
@@ -98,11 +99,16 @@ def check_gemm_against_oracle(dtype, A, Bt, sites, mode, max_fragile=0):
             # products of two low-precision operands are exact: bit-equal on both sides
             assert lg["before_bits"] == lo["before_bits"] and lg["final_bits"] == lo["final_bits"]
             assert lg["status"] == lo["status"]
-        else:
+        elif (i, j) not in seen:
+            # first site on this element: the value it meets is a (partial) clean sum
             assert close(bits_f32(lg["before_bits"]), bits_f32(lo["before_bits"]), tol[i, j])
             if (lg["before_bits"] ^ lo["before_bits"]) & 0xFF800000:
                 fragile += 1
                 fragile_elems.add((i, j))
+        elif kind == orc.KIND_OUT and seen[(i, j)][0] == orc.KIND_OUT:
+            # later output sites continue from the previous flip, bit for bit
+            assert lg["before_bits"] == log_g[seen[(i, j)][1]]["after_bits"]
+        seen[(i, j)] = (kind, t)
     # stored values
     ok = close(Cg, Co, tol) | touched
     assert ok.all(), f"{(~ok).sum()} elements out of tolerance, first at {np.argwhere(~ok)[:5].tolist()}"
@@ -155,6 +161,7 @@ def check_campaign_against_oracle(dtype, A, Bt, sites, mode, max_fragile=0):
     Cg, rg = run_gpu_campaign(dtype, A, Bt, sites, mode)
     Cclean, *_ = orc.gemm(dtype, A, Bt)
     ro = orc.campaign(dtype, A, Bt, Cclean, sites, mode)
+    ro_raw = orc.campaign(dtype, A, Bt, Cclean, sites, mode & ~orc.CORRECT) if mode & orc.CORRECT else ro
     ap = orc.absprod(dtype, A, Bt)
     assert close(Cg, Cclean, TOL * ap).all()
     fragile = 0
@@ -169,7 +176,12 @@ def check_campaign_against_oracle(dtype, A, Bt, sites, mode, max_fragile=0):
         assert g["after_bits"] == g["before_bits"] ^ (s["xor_mask"] if kind in ELEMENT_KINDS else 0) or kind in (orc.KIND_A, orc.KIND_B)
         if kind in (orc.KIND_ACC, orc.KIND_TERM):
             # recomputed in k order on both sides: everything is bit-exact
+            # ... except the payload of a NaN that the fault created and later additions carried along:
+            # IEEE 754 leaves it to the platform, so what a correction makes of it is not unique
+            nan_made = bool(np.isnan(bits_f32(ro_raw[t]["final_bits"])))
             for f in g.dtype.names:
+                if nan_made and f in ("final_bits", "max_abs_dev"):
+                    continue
                 assert g[f] == o[f] or (f == "max_abs_dev" and np.isnan(g[f]) and np.isnan(o[f])), (t, f, g, o)
         elif kind == orc.KIND_OUT:
             i, j = int(s["row"]), int(s["col"])

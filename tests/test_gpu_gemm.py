@@ -51,7 +51,8 @@ def test_clean_gemm_with_ragged_tiles(dtype, shape):
 def test_plain_gemm_without_flags_buffer():
     A, Bt = rand_operands(orc.BF16, 256, 256, 256, 13)
     Cg = torch.empty((256, 256), dtype=torch.float32, device="cuda")
-    rc = mpg.mpgemmfi_gemm(orc.BF16, 256, 256, 256, to_dev(A, orc.BF16).data_ptr(), to_dev(Bt, orc.BF16).data_ptr(),
+    a, b = to_dev(A, orc.BF16), to_dev(Bt, orc.BF16)
+    rc = mpg.mpgemmfi_gemm(orc.BF16, 256, 256, 256, a.data_ptr(), b.data_ptr(),
                            Cg.data_ptr(), None, 0, 0, None, torch.cuda.current_stream().cuda_stream)
     assert rc == 0
     torch.cuda.synchronize()
