@@ -202,6 +202,36 @@ int mpgemmfi_campaign(int dtype, int M, int N, int K, const void *A, const void 
                       mpgemmfi_trial_record *records, void *workspace, size_t workspace_bytes,
                       mpgemmfi_stream stream);
 
+/*
+ * The campaign for callers that must not allocate device memory. (The paper has no
+ * counterpart to this entry point; it exists for how the library gets embedded.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin or callback
+ * invoked from inside someone else's pipeline, a real-time or long-running service that
+ * froze its memory pools at start-up, or a host program whose device memory is handed
+ * out by another owner. Such a caller has nowhere to get the `workspace` that
+ * mpgemmfi_campaign asks for. Here the trial schedule lives instead in a fixed array
+ * that is part of the library image: 256 + 12 * MPGEMMFI_STATIC_MAX_TRIALS bytes
+ * (768.25 KiB) of device memory on every GPU that loads the library, held until the
+ * process unloads it. The call itself allocates and frees nothing.
+ *
+ * Arguments, results and errors are those of mpgemmfi_campaign without `workspace` and
+ * `workspace_bytes`; inputs, C_clean and records are still the caller's buffers.
+ * n_trials above MPGEMMFI_STATIC_MAX_TRIALS is refused with MPGEMMFI_ERR_WORKSPACE
+ * before anything is queued; split the table across several calls instead.
+ *
+ * The first call on each device looks up the array's device address (that device must be
+ * current) and sets kernel attributes; make that first call outside any stream capture.
+ * All calls on one device share the one array and it keeps whatever the previous call
+ * left: each call clears the counters it needs on `stream` before use, so calls queued
+ * one after another on a stream are safe, but two calls that can overlap on the GPU
+ * (different streams, different host threads) race on it and corrupt each other's records.
+ */
+#define MPGEMMFI_STATIC_MAX_TRIALS 65536
+int mpgemmfi_campaign_static(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C_clean,
+                             const mpgemmfi_site *sites, int n_trials, int detect_mode,
+                             mpgemmfi_trial_record *records, mpgemmfi_stream stream);
+
 /* k elements between two accumulator boundaries: 64 (FP16, BF16), 32 (TF32); 0 for a bad dtype. */
 int mpgemmfi_kstep(int dtype);
 

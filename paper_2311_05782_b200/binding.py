@@ -18,6 +18,7 @@ DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP = 0, 1, 2, 3
 CORRECT = 16
 STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT = 1, 2
 MAX_FAULTS = 4096
+STATIC_MAX_TRIALS = 65536
 HEADER_WORDS = 16
 
 SITE_DTYPE = np.dtype([("kind", "<u4"), ("row", "<u4"), ("col", "<u4"), ("k", "<u4"),
@@ -34,7 +35,7 @@ _lib = None
 _SYMBOLS = [
     "mpgemmfi_gemm", "mpgemmfi_campaign", "mpgemmfi_kstep", "mpgemmfi_flags_bytes",
     "mpgemmfi_flags_bitmap_offset", "mpgemmfi_campaign_workspace_bytes", "mpgemmfi_validate_sites",
-    "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version",
+    "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version", "mpgemmfi_campaign_static",
 ]
 
 
@@ -69,6 +70,8 @@ def load_library():
     L.mpgemmfi_gemm.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp]
     L.mpgemmfi_campaign.restype = i
     L.mpgemmfi_campaign.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp, sz, vp]
+    L.mpgemmfi_campaign_static.restype = i
+    L.mpgemmfi_campaign_static.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp]
     L.mpgemmfi_kstep.restype = i
     L.mpgemmfi_kstep.argtypes = [i]
     L.mpgemmfi_flags_bytes.restype = sz
@@ -99,6 +102,13 @@ def mpgemmfi_campaign(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mo
                       workspace_bytes, stream):
     return load_library().mpgemmfi_campaign(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mode, records,
                                             workspace, workspace_bytes, stream)
+
+
+def mpgemmfi_campaign_static(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mode, records, stream):
+    """Raw call of the campaign variant that keeps its schedule in the library's built-in device array,
+    for callers that are not allowed to allocate device memory. At most STATIC_MAX_TRIALS trials per call."""
+    return load_library().mpgemmfi_campaign_static(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mode,
+                                                   records, stream)
 
 
 def mpgemmfi_kstep(dtype):

@@ -9,6 +9,8 @@
 #include "checks.cuh"
 #include "gemm_sm100.cuh"
 
+static_assert(MPGEMMFI_STATIC_MAX_TRIALS == mpg::CAMPAIGN_STATIC_MAX_TRIALS, "header and kernel limits differ");
+
 namespace {
 
 int g_last_cuda_error = 0;
@@ -182,6 +184,36 @@ int mpgemmfi_campaign(int dtype, int M, int N, int K, const void *A, const void 
     p.A = A; p.Bt = Bt; p.C = C_clean; p.sites = sites; p.records = records;
     mpg::campaign_bind_schedule(p, workspace);
     const cudaError_t e = mpg::launch_campaign_trials(p, di.num_sms, st);
+    return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
+}
+
+int mpgemmfi_campaign_static(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C_clean,
+                             const mpgemmfi_site *sites, int n_trials, int detect_mode,
+                             mpgemmfi_trial_record *records, mpgemmfi_stream stream)
+{
+    int rc = check_common(dtype, M, N, K, A, Bt, C_clean);
+    if (rc) return rc;
+    if (n_trials < 0 || (n_trials > 0 && (!sites || !records))) return MPGEMMFI_ERR_ARG;
+    if (detect_mode & ~(MPGEMMFI_DETECT_TECHNIQUE_MASK | MPGEMMFI_CORRECT)) return MPGEMMFI_ERR_ARG;
+    if (((uintptr_t)sites & 15) || ((uintptr_t)records & 7)) return MPGEMMFI_ERR_ALIGN;
+    if (n_trials > MPGEMMFI_STATIC_MAX_TRIALS) return MPGEMMFI_ERR_WORKSPACE;   // built-in scratch too small
+    DeviceInfo di;
+    rc = device_info(di);
+    if (rc) return rc;
+    if (di.major != 10) return MPGEMMFI_ERR_ARCH;
+    void *scratch = nullptr;
+    size_t scratch_bytes = 0;
+    cudaError_t e = mpg::campaign_static_schedule(&scratch, &scratch_bytes);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (scratch_bytes < mpg::campaign_schedule_bytes(n_trials)) return MPGEMMFI_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = run_gemm(dtype, M, N, K, A, Bt, C_clean, nullptr, 0, MPGEMMFI_DETECT_NONE, nullptr, st, di);
+    if (rc) return rc;
+    mpg::CampaignParams p;
+    p.dtype = dtype; p.M = M; p.N = N; p.K = K; p.detect_mode = detect_mode; p.n_trials = n_trials;
+    p.A = A; p.Bt = Bt; p.C = C_clean; p.sites = sites; p.records = records;
+    mpg::campaign_bind_schedule(p, scratch);
+    e = mpg::launch_campaign_trials(p, di.num_sms, st);   // clears the schedule counters first
     return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
 }
 

@@ -247,6 +247,29 @@ void campaign_bind_schedule(CampaignParams &p, void *scratch)
     p.list_e = p.list_b + p.n_trials;
 }
 
+// Built-in schedule scratch for callers that cannot allocate device memory. It lives in every
+// context that loads the library, for as long as the library stays loaded.
+static __device__ __align__(256) unsigned char g_static_schedule[256 + 3 * sizeof(uint32_t) * CAMPAIGN_STATIC_MAX_TRIALS];
+
+cudaError_t campaign_static_schedule(void **ptr, size_t *bytes)
+{
+    // In host code `g_static_schedule` is only a handle for the runtime; the address a kernel can
+    // use has to be asked for, once per device, while that device is current.
+    static void *addr[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    void *a = (dev >= 0 && dev < 64) ? addr[dev] : nullptr;
+    if (!a) {
+        e = cudaGetSymbolAddress(&a, g_static_schedule);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) addr[dev] = a;
+    }
+    *ptr = a;
+    *bytes = sizeof(g_static_schedule);
+    return cudaSuccess;
+}
+
 cudaError_t launch_campaign_trials(const CampaignParams &p, int num_sms, cudaStream_t stream)
 {
     if (p.n_trials <= 0) return cudaSuccess;

@@ -30,6 +30,13 @@ size_t campaign_schedule_bytes(int n_trials);
 // point the schedule members of p into a scratch block of campaign_schedule_bytes(p.n_trials) bytes
 void campaign_bind_schedule(CampaignParams &p, void *scratch);
 
+// Most trials a call may carry when the schedule lives in the library's built-in scratch.
+constexpr int CAMPAIGN_STATIC_MAX_TRIALS = 65536;
+
+// Device address and size of the built-in schedule scratch of the current device. The first call
+// on a device resolves the address; nothing is allocated.
+cudaError_t campaign_static_schedule(void **ptr, size_t *bytes);
+
 // schedule + evaluate every trial; the clean product must already be queued on `stream`
 cudaError_t launch_campaign_trials(const CampaignParams &p, int num_sms, cudaStream_t stream);
 
