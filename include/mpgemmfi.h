@@ -232,6 +232,23 @@ int mpgemmfi_campaign_static(int dtype, int M, int N, int K, const void *A, cons
                              const mpgemmfi_site *sites, int n_trials, int detect_mode,
                              mpgemmfi_trial_record *records, mpgemmfi_stream stream);
 
+/*
+ * Tuning knob (no counterpart in the paper): how the GEMM kernel tiles the output.
+ *   AUTO   the library decides from M and N (default)
+ *   SINGLE every CTA computes whole 128 x {64,128,256} tiles
+ *   PAIR   two CTAs on neighbouring SMs share one 256 x 256 tile and the Bt tile (tcgen05
+ *          cta_group::2); falls back to SINGLE when the device cannot host such pairs
+ * Process-wide, not thread-safe against concurrent launches. Results are the same fault
+ * semantics either way; individual output values may differ in rounding between policies.
+ * Returns MPGEMMFI_OK or MPGEMMFI_ERR_ARG.
+ */
+enum {
+    MPGEMMFI_TILES_AUTO = 0,
+    MPGEMMFI_TILES_SINGLE = 1,
+    MPGEMMFI_TILES_PAIR = 2
+};
+int mpgemmfi_set_tile_policy(int policy);
+
 /* k elements between two accumulator boundaries: 64 (FP16, BF16), 32 (TF32); 0 for a bad dtype. */
 int mpgemmfi_kstep(int dtype);
 

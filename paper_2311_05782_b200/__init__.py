@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     SITE_A, SITE_B, SITE_ACC, SITE_OUT, SITE_TERM,
     DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP, CORRECT,
     STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT, MAX_FAULTS, HEADER_WORDS, STATIC_MAX_TRIALS,
+    TILES_AUTO, TILES_SINGLE, TILES_PAIR, mpgemmfi_set_tile_policy,
     SITE_DTYPE, SITE_LOG_DTYPE, RECORD_DTYPE,
     MpgemmfiError, library_path, load_library, exported_symbols,
     mpgemmfi_gemm, mpgemmfi_campaign, mpgemmfi_campaign_static, mpgemmfi_kstep, mpgemmfi_flags_bytes,

@@ -19,6 +19,7 @@ CORRECT = 16
 STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT = 1, 2
 MAX_FAULTS = 4096
 STATIC_MAX_TRIALS = 65536
+TILES_AUTO, TILES_SINGLE, TILES_PAIR = 0, 1, 2
 HEADER_WORDS = 16
 
 SITE_DTYPE = np.dtype([("kind", "<u4"), ("row", "<u4"), ("col", "<u4"), ("k", "<u4"),
@@ -36,6 +37,7 @@ _SYMBOLS = [
     "mpgemmfi_gemm", "mpgemmfi_campaign", "mpgemmfi_kstep", "mpgemmfi_flags_bytes",
     "mpgemmfi_flags_bitmap_offset", "mpgemmfi_campaign_workspace_bytes", "mpgemmfi_validate_sites",
     "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version", "mpgemmfi_campaign_static",
+    "mpgemmfi_set_tile_policy",
 ]
 
 
@@ -72,6 +74,8 @@ def load_library():
     L.mpgemmfi_campaign.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp, sz, vp]
     L.mpgemmfi_campaign_static.restype = i
     L.mpgemmfi_campaign_static.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp]
+    L.mpgemmfi_set_tile_policy.restype = i
+    L.mpgemmfi_set_tile_policy.argtypes = [i]
     L.mpgemmfi_kstep.restype = i
     L.mpgemmfi_kstep.argtypes = [i]
     L.mpgemmfi_flags_bytes.restype = sz
@@ -109,6 +113,11 @@ def mpgemmfi_campaign_static(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, de
     for callers that are not allowed to allocate device memory. At most STATIC_MAX_TRIALS trials per call."""
     return load_library().mpgemmfi_campaign_static(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mode,
                                                    records, stream)
+
+
+def mpgemmfi_set_tile_policy(policy):
+    """TILES_AUTO (0), TILES_SINGLE (1) or TILES_PAIR (2); process-wide."""
+    return load_library().mpgemmfi_set_tile_policy(policy)
 
 
 def mpgemmfi_kstep(dtype):

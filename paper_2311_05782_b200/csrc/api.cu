@@ -84,6 +84,8 @@ int encode_operand_map(CUtensorMap *map, int dtype, const void *base, int rows, 
     return MPGEMMFI_OK;
 }
 
+int g_tile_policy = MPGEMMFI_TILES_AUTO;
+
 // widest tile that still gives every SM a tile; narrow outputs get narrow tiles
 int choose_bn(int M, int N, int num_sms)
 {
@@ -95,6 +97,17 @@ int choose_bn(int M, int N, int num_sms)
         if (tiles_m * ((N + bn - 1) / bn) >= num_sms || i == 2) return bn;
     }
     return 64;
+}
+
+// 256 x 256 tiles on CTA pairs pay off once there are enough of them to occupy most pairs
+bool choose_pair(int dtype, int M, int N, int *max_pairs)
+{
+    if (g_tile_policy == MPGEMMFI_TILES_SINGLE) return false;
+    *max_pairs = mpg::gemm_max_resident_pairs(dtype);
+    if (*max_pairs <= 0) return false;
+    if (g_tile_policy == MPGEMMFI_TILES_PAIR) return true;
+    const long long tiles = (long long)((M + 255) / 256) * ((N + 255) / 256);
+    return M > 128 && N > 128 && tiles >= *max_pairs / 2;
 }
 
 int check_common(int dtype, int M, int N, int K, const void *A, const void *Bt, const void *C)
@@ -110,17 +123,20 @@ int check_common(int dtype, int M, int N, int K, const void *A, const void *Bt, 
 int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C, const mpgemmfi_site *sites,
              int n_faults, int detect_mode, uint32_t *flags, cudaStream_t stream, const DeviceInfo &di)
 {
-    const int bn = choose_bn(M, N, di.num_sms);
+    int max_pairs = 0;
+    const bool pair = choose_pair(dtype, M, N, &max_pairs);
+    const int bn = pair ? 256 : choose_bn(M, N, di.num_sms);
+    const int tm = pair ? 256 : 128;
     CUtensorMap tm_a, tm_b;
     int rc = encode_operand_map(&tm_a, dtype, A, M, K, 128);
     if (rc) return rc;
-    rc = encode_operand_map(&tm_b, dtype, Bt, N, K, bn);
+    rc = encode_operand_map(&tm_b, dtype, Bt, N, K, pair ? 128 : bn);
     if (rc) return rc;
 
     mpg::GemmParams p;
     p.dtype = dtype; p.M = M; p.N = N; p.K = K;
     p.detect_mode = detect_mode; p.n_faults = n_faults;
-    p.tiles_m = (M + 127) / 128; p.tiles_n = (N + bn - 1) / bn;
+    p.tiles_m = (M + tm - 1) / tm; p.tiles_n = (N + bn - 1) / bn;
     p.num_tiles = p.tiles_m * p.tiles_n;
     const int ks = mpg::kstep_of(dtype);
     p.num_kt = (K + ks - 1) / ks;
@@ -132,8 +148,9 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
         const cudaError_t e = cudaMemsetAsync(flags, 0, sizeof(uint32_t) * (MPGEMMFI_HEADER_WORDS + 4 * (size_t)n_faults), stream);
         if (e != cudaSuccess) return cuda_fail(e);
     }
-    const int grid = p.num_tiles < di.num_sms ? p.num_tiles : di.num_sms;
-    const cudaError_t e = mpg::launch_gemm(bn, tm_a, tm_b, p, grid, stream);
+    const int walkers = pair ? max_pairs : di.num_sms;
+    const int grid = (p.num_tiles < walkers ? p.num_tiles : walkers) * (pair ? 2 : 1);
+    const cudaError_t e = mpg::launch_gemm(bn, pair, tm_a, tm_b, p, grid, stream);
     return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
 }
 
@@ -215,6 +232,14 @@ int mpgemmfi_campaign_static(int dtype, int M, int N, int K, const void *A, cons
     mpg::campaign_bind_schedule(p, scratch);
     e = mpg::launch_campaign_trials(p, di.num_sms, st);   // clears the schedule counters first
     return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
+}
+
+int mpgemmfi_set_tile_policy(int policy)
+{
+    if (policy != MPGEMMFI_TILES_AUTO && policy != MPGEMMFI_TILES_SINGLE && policy != MPGEMMFI_TILES_PAIR)
+        return MPGEMMFI_ERR_ARG;
+    g_tile_policy = policy;
+    return MPGEMMFI_OK;
 }
 
 int mpgemmfi_kstep(int dtype)

@@ -12,6 +12,13 @@
 //
 // The fault-site table is decoded once per CTA into a list of the entries that touch any of
 // its tiles; a CTA whose list is empty never looks at a site again.
+//
+// Two launch shapes share this code. Single: every CTA owns whole 128 x BN tiles. Pair: two
+// CTAs (a cluster of two on neighbouring SMs) own one 256 x 256 tile; each stages its own 128
+// rows of A and its own 128-row half of Bt, the leader CTA issues cta_group::2 MMAs that read
+// both CTAs' shared memory and fill both CTAs' TMEM, and each CTA runs the epilogue of its own
+// 128 rows. Halving the Bt bytes each SM has to pull per MMA is what lifts the main loop off
+// the SM's shared-memory fill rate.
 #include <cstdint>
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -29,14 +36,16 @@ constexpr int BM = 128;
 constexpr int NUM_THREADS = 256;
 constexpr int MAX_STAGES = 8;
 
-template <int BN>
+template <int BN, bool kPair>
 struct Cfg {
+    static constexpr int B_ROWS = kPair ? BN / 2 : BN;     // Bt rows staged by one CTA
     static constexpr int A_BYTES = BM * 128;
-    static constexpr int B_BYTES = BN * 128;
+    static constexpr int B_BYTES = B_ROWS * 128;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGES = (200 * 1024 / STAGE_BYTES) < MAX_STAGES ? (200 * 1024 / STAGE_BYTES) : MAX_STAGES;
     static constexpr int TMEM_COLS = 2 * BN;   // two accumulators; 128, 256 or 512 columns
     static_assert(BN == 64 || BN == 128 || BN == 256, "BN must be 64, 128 or 256");
+    static_assert(!kPair || BN == 256, "pair tiles are 256 x 256");
 };
 
 // Control block that follows the stages in dynamic shared memory.
@@ -55,15 +64,21 @@ struct alignas(16) Control {
     uint16_t site_idx[MPGEMMFI_MAX_FAULTS];
 };
 
+// Ranges of one output tile as seen by one CTA. In single mode "own" and "tile" coincide; in pair
+// mode the tile is 256 rows tall, the CTA owns 128 of them and a 128-row half of the Bt tile.
 struct TileCtx {
     const GemmParams *p;
     const Control *ctl;
-    uint32_t m0, n0;
-    int bn;
+    uint32_t m0, n0;        // rows of C / A this CTA computes, first column of the tile
+    uint32_t tile_m0;       // first row of the whole tile
+    uint32_t b0;            // first Bt row (column of C) this CTA stages
+    uint32_t tile_rows, bn, b_rows;
 };
 
-__device__ __forceinline__ bool in_tile_rows(const TileCtx &c, uint32_t row) { return row - c.m0 < (uint32_t)BM; }
-__device__ __forceinline__ bool in_tile_cols(const TileCtx &c, uint32_t col) { return col - c.n0 < (uint32_t)c.bn; }
+__device__ __forceinline__ bool in_own_rows(const TileCtx &c, uint32_t row) { return row - c.m0 < (uint32_t)BM; }
+__device__ __forceinline__ bool in_tile_rows(const TileCtx &c, uint32_t row) { return row - c.tile_m0 < c.tile_rows; }
+__device__ __forceinline__ bool in_tile_cols(const TileCtx &c, uint32_t col) { return col - c.n0 < c.bn; }
+__device__ __forceinline__ bool in_own_b(const TileCtx &c, uint32_t col) { return col - c.b0 < c.b_rows; }
 
 // smallest k-tile >= kt_from in which this tile has an operand site (warp-wide)
 __device__ uint32_t scan_next_operand(const TileCtx &c, uint32_t kt_from, int lane)
@@ -72,8 +87,8 @@ __device__ uint32_t scan_next_operand(const TileCtx &c, uint32_t kt_from, int la
     uint32_t best = NONE;
     for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
         const mpgemmfi_site s = load_site(c.p->sites, c.ctl->site_idx[i]);
-        const bool hit = (s.kind == MPGEMMFI_SITE_A && in_tile_rows(c, s.row)) ||
-                         (s.kind == MPGEMMFI_SITE_B && in_tile_cols(c, s.col));
+        const bool hit = (s.kind == MPGEMMFI_SITE_A && in_own_rows(c, s.row)) ||
+                         (s.kind == MPGEMMFI_SITE_B && in_own_b(c, s.col));
         if (hit && s.k / ks >= kt_from) best = min(best, s.k / ks);
     }
     return __reduce_min_sync(0xFFFFFFFFu, best);
@@ -99,7 +114,7 @@ __device__ bool scan_has_out(const TileCtx &c, int lane)
     bool any = false;
     for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
         const mpgemmfi_site s = load_site(c.p->sites, c.ctl->site_idx[i]);
-        any |= s.kind == MPGEMMFI_SITE_OUT && in_tile_rows(c, s.row) && in_tile_cols(c, s.col);
+        any |= s.kind == MPGEMMFI_SITE_OUT && in_own_rows(c, s.row) && in_tile_cols(c, s.col);
     }
     return __any_sync(0xFFFFFFFFu, any);
 }
@@ -134,8 +149,8 @@ __device__ void apply_operand_sites(const TileCtx &c, uint32_t kt, uint8_t *smem
         uint8_t *tile;
         uint32_t r;
         bool log_here;
-        if (s.kind == MPGEMMFI_SITE_A && in_tile_rows(c, s.row)) { tile = smem_a; r = s.row - c.m0; log_here = c.n0 == 0; }
-        else if (s.kind == MPGEMMFI_SITE_B && in_tile_cols(c, s.col)) { tile = smem_b; r = s.col - c.n0; log_here = c.m0 == 0; }
+        if (s.kind == MPGEMMFI_SITE_A && in_own_rows(c, s.row)) { tile = smem_a; r = s.row - c.m0; log_here = c.n0 == 0; }
+        else if (s.kind == MPGEMMFI_SITE_B && in_own_b(c, s.col)) { tile = smem_b; r = s.col - c.b0; log_here = c.tile_m0 == 0; }
         else continue;
         if (s.k / ks != kt) continue;
         uint8_t *ptr = tile + swizzled_offset(r, (s.k % ks) * es);
@@ -178,7 +193,7 @@ __device__ void apply_boundary_sites(const TileCtx &c, uint32_t b, uint32_t tmem
         const uint32_t idx = c.ctl->site_idx[i];
         const mpgemmfi_site s = load_site(p.sites, idx);
         if (!(s.kind == MPGEMMFI_SITE_ACC || s.kind == MPGEMMFI_SITE_TERM)) continue;
-        if (!in_tile_rows(c, s.row) || !in_tile_cols(c, s.col)) continue;
+        if (!in_own_rows(c, s.row) || !in_tile_cols(c, s.col)) continue;
         if (site_boundary(s, p.dtype, p.K) != b) continue;
         const uint32_t r = s.row - c.m0;
         if ((int)(r >> 5) != q) continue;
@@ -236,29 +251,30 @@ __device__ void apply_out_sites(const TileCtx &c, uint32_t row, uint32_t c0, uin
     }
 }
 
-template <int BN>
-__device__ bool site_touches_cta(const mpgemmfi_site &s, const GemmParams &p)
+// Does a site touch a tile walked by tile-walker `gid` of `groups` (a CTA, or a CTA pair)?
+// Tiles are TM x BN and are dealt out round-robin: tile index = tn * tiles_m + tm.
+template <int TM, int BN>
+__device__ bool site_touches_group(const mpgemmfi_site &s, const GemmParams &p, uint32_t gid, uint32_t groups)
 {
-    const uint32_t g = gridDim.x, bid = blockIdx.x;
     if (s.kind == MPGEMMFI_SITE_A) {
-        const uint32_t tm = s.row / BM;
+        const uint32_t tm = s.row / TM;
         for (uint32_t tn = 0; tn < (uint32_t)p.tiles_n; ++tn)
-            if ((tn * p.tiles_m + tm) % g == bid) return true;
+            if ((tn * p.tiles_m + tm) % groups == gid) return true;
         return false;
     }
     if (s.kind == MPGEMMFI_SITE_B) {
         const uint32_t tn = s.col / BN;
         for (uint32_t tm = 0; tm < (uint32_t)p.tiles_m; ++tm)
-            if ((tn * p.tiles_m + tm) % g == bid) return true;
+            if ((tn * p.tiles_m + tm) % groups == gid) return true;
         return false;
     }
-    return ((s.col / BN) * p.tiles_m + s.row / BM) % g == bid;
+    return ((s.col / BN) * p.tiles_m + s.row / TM) % groups == gid;
 }
 
-// All threads: ordered list of the valid sites that touch a tile of this CTA. CTA 0 also
+// All threads: ordered list of the valid sites that touch a tile of this CTA (pair). CTA 0 also
 // reports invalid entries (skipped) and the applied count.
-template <int BN>
-__device__ void build_site_list(const GemmParams &p, Control *ctl)
+template <int TM, int BN>
+__device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid, uint32_t groups)
 {
     const int tid = threadIdx.x;
     const int n = p.n_faults;
@@ -272,7 +288,7 @@ __device__ void build_site_list(const GemmParams &p, Control *ctl)
     for (int i = beg; i < end; ++i) {
         const mpgemmfi_site s = load_site(p.sites, i);
         const bool ok = site_valid(s, p.dtype, p.M, p.N, p.K);
-        if (ok) { n_valid++; cnt += site_touches_cta<BN>(s, p) ? 1u : 0u; }
+        if (ok) { n_valid++; cnt += site_touches_group<TM, BN>(s, p, gid, groups) ? 1u : 0u; }
         else {
             n_bad++;
             if (blockIdx.x == 0) write_log(p, i, 0u, 0u, 0u, 2u);
@@ -293,17 +309,22 @@ __device__ void build_site_list(const GemmParams &p, Control *ctl)
     uint32_t off = ctl->scan[tid];
     for (int i = beg; i < end; ++i) {
         const mpgemmfi_site s = load_site(p.sites, i);
-        if (site_valid(s, p.dtype, p.M, p.N, p.K) && site_touches_cta<BN>(s, p)) ctl->site_idx[off++] = (uint16_t)i;
+        if (site_valid(s, p.dtype, p.M, p.N, p.K) && site_touches_group<TM, BN>(s, p, gid, groups))
+            ctl->site_idx[off++] = (uint16_t)i;
     }
 }
 
-template <int BN, bool kTF32>
+// kPair = false: grid of single CTAs, tiles 128 x BN.
+// kPair = true : grid of CTA pairs (cluster dimension 2), tiles 256 x BN, BN = 256.
+template <int BN, bool kTF32, bool kPair>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const GemmParams p)
 {
-    using C = Cfg<BN>;
+    using C = Cfg<BN, kPair>;
     constexpr int KT = kTF32 ? 32 : 64;      // elements per 128-byte row
     constexpr int STAGES = C::STAGES;
+    constexpr int TM = kPair ? 2 * BM : BM;  // rows of one tile
+    constexpr uint32_t EPI_ARRIVALS = kPair ? 8 : 4;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -312,64 +333,130 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t num_kt = (uint32_t)p.num_kt;
+    const uint32_t rank = kPair ? cluster_cta_rank() : 0u;          // 0 = leader of the pair
+    const uint32_t gid = kPair ? blockIdx.x >> 1 : blockIdx.x;      // tile walker id
+    const uint32_t groups = kPair ? gridDim.x >> 1 : gridDim.x;
+    const bool leader = rank == 0;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->acc_full[s]), 1); mbar_init(smem_u32(&ctl->acc_empty[s]), 4); }
+        for (int s = 0; s < STAGES; ++s) {
+            // pair mode, leader CTA: one arrival per CTA of the pair (each announces its own bytes)
+            mbar_init(smem_u32(&ctl->full[s]), (kPair && leader) ? 2 : 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->acc_full[s]), 1); mbar_init(smem_u32(&ctl->acc_empty[s]), EPI_ARRIVALS); }
         mbar_init(smem_u32(&ctl->pause_full), 1);
-        mbar_init(smem_u32(&ctl->pause_done), 4);
+        mbar_init(smem_u32(&ctl->pause_done), EPI_ARRIVALS);
         ctl->abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tm_a);
         tma_prefetch_desc(&tm_b);
     }
     if (warp == 2) {
-        tmem_alloc(smem_u32(&ctl->tmem_base), C::TMEM_COLS);
-        tmem_relinquish();
+        if constexpr (kPair) { tmem_alloc_pair(smem_u32(&ctl->tmem_base), C::TMEM_COLS); tmem_relinquish_pair(); }
+        else { tmem_alloc(smem_u32(&ctl->tmem_base), C::TMEM_COLS); tmem_relinquish(); }
     }
-    build_site_list<BN>(p, ctl);
+    build_site_list<TM, BN>(p, ctl, gid, groups);
     tc_fence_before_sync();
-    __syncthreads();
+    if constexpr (kPair) cluster_sync_all(); else __syncthreads();
     tc_fence_after_sync();
 
     const uint32_t tmem_base = ctl->tmem_base;
     const bool has_sites = ctl->site_count != 0;
     TileCtx tc;
-    tc.p = &p; tc.ctl = ctl; tc.bn = BN;
+    tc.p = &p; tc.ctl = ctl; tc.bn = BN; tc.tile_rows = TM; tc.b_rows = C::B_ROWS;
+    auto set_tile = [&](uint32_t t) {
+        tc.tile_m0 = (t % p.tiles_m) * TM;
+        tc.m0 = tc.tile_m0 + rank * BM;
+        tc.n0 = (t / p.tiles_m) * BN;
+        tc.b0 = tc.n0 + rank * C::B_ROWS;
+    };
+    // barriers of the leader CTA that this CTA's warps arrive on
+    const uint32_t lead_acc_empty0 = kPair ? map_to_cta(smem_u32(&ctl->acc_empty[0]), 0) : smem_u32(&ctl->acc_empty[0]);
+    const uint32_t lead_pause_done = kPair ? map_to_cta(smem_u32(&ctl->pause_done), 0) : smem_u32(&ctl->pause_done);
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            uint32_t stage = 0, phase = 0, armed = 0, armed_parity = 0;
-            bool ok = true;
-            for (uint32_t t = blockIdx.x; ok && t < (uint32_t)p.num_tiles; t += gridDim.x) {
-                const int m0 = (int)(t % p.tiles_m) * BM, n0 = (int)(t / p.tiles_m) * BN;
-                for (uint32_t kt = 0; kt < num_kt; ++kt) {
-                    if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t bar = smem_u32(&ctl->full[stage]);
-                    uint8_t *sa = smem + stage * C::STAGE_BYTES;
-                    mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
-                    tma_load_2d(smem_u32(sa), &tm_a, bar, (int)(kt * KT), m0);
-                    tma_load_2d(smem_u32(sa + C::A_BYTES), &tm_b, bar, (int)(kt * KT), n0);
-                    armed |= 1u << stage;
-                    armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        // Pair mode: both CTAs count their bytes on the LEADER's full barrier, so the leader's MMA
+        // warp waits on one barrier per stage. Exception: a stage in which the non-leader CTA has
+        // an operand site is loaded against that CTA's own barrier; its warp 1 flips the element
+        // and then delivers the CTA's arrival to the leader.
+        uint32_t stage = 0, phase = 0, armed = 0, armed_parity = 0;
+        const uint32_t lead_full0 = kPair ? map_to_cta(smem_u32(&ctl->full[0]), 0) : 0u;
+        bool ok = true;
+        for (uint32_t t = gid; ok && t < (uint32_t)p.num_tiles; t += groups) {
+            set_tile(t);
+            uint32_t next_op = NONE;
+            if (kPair && !leader && has_sites) next_op = scan_next_operand(tc, 0, lane);
+            for (uint32_t kt = 0; kt < num_kt; ++kt) {
+                const bool own_barrier = !kPair || leader || kt == next_op;
+                if (kPair && kt == next_op) next_op = scan_next_operand(tc, kt + 1, lane);
+                if (lane == 0) {
+                    ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag);
+                    if (ok) {
+                        uint8_t *sa = smem + stage * C::STAGE_BYTES;
+                        if (own_barrier) {
+                            const uint32_t bar = smem_u32(&ctl->full[stage]);
+                            mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
+                            tma_load_2d(smem_u32(sa), &tm_a, bar, (int)(kt * KT), (int)tc.m0);
+                            tma_load_2d(smem_u32(sa + C::A_BYTES), &tm_b, bar, (int)(kt * KT), (int)tc.b0);
+                            armed |= 1u << stage;
+                            armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+                        } else {
+                            const uint32_t bar = lead_full0 + stage * (uint32_t)sizeof(uint64_t);
+                            mbar_arrive_expect_tx_cluster(bar, C::STAGE_BYTES);
+                            tma_load_2d_pair(smem_u32(sa), &tm_a, bar, (int)(kt * KT), (int)tc.m0);
+                            tma_load_2d_pair(smem_u32(sa + C::A_BYTES), &tm_b, bar, (int)(kt * KT), (int)tc.b0);
+                        }
+                    }
                 }
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                if (!ok) break;
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
-            // wait (bounded) until every copy this thread started has landed
+        }
+        // wait (bounded) until every copy counted on this CTA's barriers has landed (the leader's
+        // barriers also count the other CTA's copies)
+        if (lane == 0 && (!kPair || leader)) {
             uint32_t never = 0;
             for (int s = 0; s < STAGES; ++s)
                 if (armed & (1u << s))
                     mbar_wait(smem_u32(&ctl->full[s]), (armed_parity >> s) & 1u, &never, 1000000000ull);
         }
+    } else if (warp == 1 && !leader) {
+        // ------------------------------------------------------------ pair mode, non-leader CTA: no MMAs to
+        // issue; only the stages that carry one of this CTA's operand sites need attention
+        if (has_sites) {
+            uint32_t lt = 0, own_phase = 0;     // own_phase: bit s = parity of this CTA's full[s]
+            bool ok = true;
+            const uint32_t lead_full0 = map_to_cta(smem_u32(&ctl->full[0]), 0);
+            for (uint32_t t = gid; ok && t < (uint32_t)p.num_tiles; t += groups, ++lt) {
+                set_tile(t);
+                uint32_t kt = scan_next_operand(tc, 0, lane);
+                while (kt != NONE) {
+                    const uint32_t g = lt * num_kt + kt, stage = g % STAGES;
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->full[stage]), (own_phase >> stage) & 1u, abort_flag));
+                    if (!ok) break;
+                    own_phase ^= 1u << stage;
+                    if (lane == 0) {
+                        uint8_t *sa = smem + stage * C::STAGE_BYTES;
+                        apply_operand_sites(tc, kt, sa, sa + C::A_BYTES);
+                        fence_proxy_async_smem();
+                        mbar_arrive_cluster(lead_full0 + stage * (uint32_t)sizeof(uint64_t));
+                    }
+                    __syncwarp();
+                    kt = scan_next_operand(tc, kt + 1, lane);
+                }
+            }
+        }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        const uint32_t idesc = umma_instr_desc((uint32_t)p.dtype, BM, BN);
+        const uint32_t idesc = umma_instr_desc((uint32_t)p.dtype, TM, BN);
         uint32_t stage = 0, phase = 0, lt = 0, pause_phase = 0;
         bool ok = true;
-        for (uint32_t t = blockIdx.x; ok && t < (uint32_t)p.num_tiles; t += gridDim.x, ++lt) {
+        for (uint32_t t = gid; ok && t < (uint32_t)p.num_tiles; t += groups, ++lt) {
             const uint32_t as = lt & 1u, ap = (lt >> 1) & 1u;
-            tc.m0 = (t % p.tiles_m) * BM; tc.n0 = (t / p.tiles_m) * BN;
+            set_tile(t);
             uint32_t next_op = NONE, next_b = NONE;
             if (has_sites) { next_op = scan_next_operand(tc, 0, lane); next_b = scan_next_boundary(tc, 1, lane); }
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_empty[as]), ap ^ 1u, abort_flag));
@@ -393,14 +480,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     const uint64_t a_desc = umma_smem_desc_sw128(smem_u32(sa));
                     const uint64_t b_desc = umma_smem_desc_sw128(smem_u32(sa + C::A_BYTES));
 #pragma unroll
-                    for (uint32_t k = 0; k < 4; ++k)     // 4 x 32 bytes along K inside the swizzle row
-                        umma_ss<kTF32>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kt | k) != 0 ? 1u : 0u);
-                    umma_commit(smem_u32(&ctl->empty[stage]));
+                    for (uint32_t k = 0; k < 4; ++k) {   // 4 x 32 bytes along K inside the swizzle row
+                        if constexpr (kPair) umma_ss_pair<kTF32>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kt | k) != 0 ? 1u : 0u);
+                        else umma_ss<kTF32>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kt | k) != 0 ? 1u : 0u);
+                    }
+                    if constexpr (kPair) umma_commit_pair(smem_u32(&ctl->empty[stage]), 3);
+                    else umma_commit(smem_u32(&ctl->empty[stage]));
                 }
                 __syncwarp();
                 if (kt + 1 == next_b) {
                     // an accumulator / term site takes effect here: let the epilogue warps edit TMEM
-                    if (lane == 0) umma_commit(smem_u32(&ctl->pause_full));
+                    if (lane == 0) {
+                        if constexpr (kPair) umma_commit_pair(smem_u32(&ctl->pause_full), 3);
+                        else umma_commit(smem_u32(&ctl->pause_full));
+                    }
                     __syncwarp();
                     ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->pause_done), pause_phase, abort_flag));
                     if (!ok) break;
@@ -411,20 +504,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
             if (!ok) break;
-            if (lane == 0) umma_commit(smem_u32(&ctl->acc_full[as]));
+            if (lane == 0) {
+                if constexpr (kPair) umma_commit_pair(smem_u32(&ctl->acc_full[as]), 3);
+                else umma_commit(smem_u32(&ctl->acc_full[as]));
+            }
             __syncwarp();
         }
     } else if (warp >= 4) {
-        // ------------------------------------------------------------ epilogue
+        // ------------------------------------------------------------ epilogue (own 128 rows)
         const int q = warp & 3;
         const bool do_bound = (p.detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK) == MPGEMMFI_DETECT_BOUNDCHECK;
         const bool do_corr = do_bound && (p.detect_mode & MPGEMMFI_CORRECT);
         uint32_t lt = 0, pause_phase = 0, n_det = 0;
         uint32_t *bitmap = p.flags ? p.flags + MPGEMMFI_HEADER_WORDS + 4 * (size_t)p.n_faults : nullptr;
         bool ok = true;
-        for (uint32_t t = blockIdx.x; ok && t < (uint32_t)p.num_tiles; t += gridDim.x, ++lt) {
+        for (uint32_t t = gid; ok && t < (uint32_t)p.num_tiles; t += groups, ++lt) {
             const uint32_t as = lt & 1u, ap = (lt >> 1) & 1u;
-            tc.m0 = (t % p.tiles_m) * BM; tc.n0 = (t / p.tiles_m) * BN;
+            set_tile(t);
             const uint32_t tmem_acc = tmem_base + as * BN;
             bool tile_has_out = false;
             if (has_sites) {
@@ -437,7 +533,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     apply_boundary_sites(tc, b, tmem_acc, q, lane);
                     tc_fence_before_sync();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&ctl->pause_done));
+                    if (lane == 0) {
+                        if constexpr (kPair) mbar_arrive_cluster(lead_pause_done);
+                        else mbar_arrive(lead_pause_done);
+                    }
                     b = scan_next_boundary(tc, b + 1, lane);
                 }
                 if (!ok) break;
@@ -460,7 +559,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     // accumulator fully read: hand the TMEM buffer back to the MMA warp
                     tc_fence_before_sync();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[as]));
+                    if (lane == 0) {
+                        if constexpr (kPair) mbar_arrive_cluster(lead_acc_empty0 + as * (uint32_t)sizeof(uint64_t));
+                        else mbar_arrive(lead_acc_empty0 + as * (uint32_t)sizeof(uint64_t));
+                    }
                 }
                 const uint32_t c0 = tc.n0 + (uint32_t)(c * 32);
                 if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 0);
@@ -507,45 +609,94 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     }
 
     tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 2) tmem_dealloc(tmem_base, C::TMEM_COLS);
+    // nobody leaves while the other CTA of a pair may still read this CTA's shared memory,
+    // arrive on its barriers or use the shared TMEM allocation
+    if constexpr (kPair) cluster_sync_all(); else __syncthreads();
+    if (warp == 2) {
+        if constexpr (kPair) tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+        else tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
     if (threadIdx.x == 0 && ctl->abort_flag && p.flags) atomicOr(&p.flags[0], MPGEMMFI_STATUS_WAIT_LIMIT);
 }
 
-template <int BN, bool kTF32>
+template <int BN, bool kTF32, bool kPair>
 cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p, int grid,
                        cudaStream_t stream)
 {
-    using C = Cfg<BN>;
+    using C = Cfg<BN, kPair>;
     const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + sizeof(Control) + 1024;
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(gemm_kernel<BN, kTF32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = cudaFuncSetAttribute(gemm_kernel<BN, kTF32, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    gemm_kernel<BN, kTF32><<<grid, NUM_THREADS, smem, stream>>>(tm_a, tm_b, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kPair ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, kTF32, kPair>, tm_a, tm_b, p);
 }
 
 }  // namespace
 
-int gemm_stage_count(int bn)
+int gemm_max_resident_pairs(int dtype)
 {
-    return bn == 256 ? Cfg<256>::STAGES : (bn == 128 ? Cfg<128>::STAGES : Cfg<64>::STAGES);
+    static int cache[64][2] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    const int tf = dtype == MPGEMMFI_TF32 ? 1 : 0;
+    if (cache[dev][tf] == 0) {
+        using C = Cfg<256, true>;
+        const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + sizeof(Control) + 1024;
+        auto kern = tf ? gemm_kernel<256, true, true> : gemm_kernel<256, false, true>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2, 1, 1);
+        cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+        cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+        cache[dev][tf] = n > 0 ? n : -1;
+    }
+    return cache[dev][tf] > 0 ? cache[dev][tf] : 0;
 }
 
-cudaError_t launch_gemm(int bn, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p, int grid,
-                        cudaStream_t stream)
+int gemm_stage_count(int bn, bool pair)
+{
+    if (pair) return Cfg<256, true>::STAGES;
+    return bn == 256 ? Cfg<256, false>::STAGES : (bn == 128 ? Cfg<128, false>::STAGES : Cfg<64, false>::STAGES);
+}
+
+cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p,
+                        int grid, cudaStream_t stream)
 {
     const bool tf32 = p.dtype == MPGEMMFI_TF32;
+    if (pair)
+        return tf32 ? launch_one<256, true, true>(tm_a, tm_b, p, grid, stream)
+                    : launch_one<256, false, true>(tm_a, tm_b, p, grid, stream);
     switch (bn) {
-    case 256: return tf32 ? launch_one<256, true>(tm_a, tm_b, p, grid, stream) : launch_one<256, false>(tm_a, tm_b, p, grid, stream);
-    case 128: return tf32 ? launch_one<128, true>(tm_a, tm_b, p, grid, stream) : launch_one<128, false>(tm_a, tm_b, p, grid, stream);
-    default:  return tf32 ? launch_one<64, true>(tm_a, tm_b, p, grid, stream) : launch_one<64, false>(tm_a, tm_b, p, grid, stream);
+    case 256: return tf32 ? launch_one<256, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<256, false, false>(tm_a, tm_b, p, grid, stream);
+    case 128: return tf32 ? launch_one<128, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<128, false, false>(tm_a, tm_b, p, grid, stream);
+    default:  return tf32 ? launch_one<64, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<64, false, false>(tm_a, tm_b, p, grid, stream);
     }
 }
 

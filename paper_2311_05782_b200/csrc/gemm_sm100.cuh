@@ -23,11 +23,18 @@ struct GemmParams {
 };
 
 // shared-memory pipeline depth used for an output tile that is bn columns wide
-int gemm_stage_count(int bn);
+int gemm_stage_count(int bn, bool pair);
 
-// bn in {64, 128, 256}: width of the output tile; tm_a / tm_b must have been encoded with
-// boxes of (128 bytes x 128 rows) and (128 bytes x bn rows), 128-byte swizzle.
-cudaError_t launch_gemm(int bn, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p, int grid,
-                        cudaStream_t stream);
+// Single mode (pair = false): bn in {64, 128, 256} is the width of the 128-row output tile; tm_b
+// must have been encoded with a box of (128 bytes x bn rows); `grid` CTAs; p.tiles_m counts
+// 128-row tiles.
+// Pair mode (pair = true): 256 x 256 tiles walked by CTA pairs; tm_b box is (128 bytes x 128 rows);
+// `grid` is even (two CTAs per pair); p.tiles_m counts 256-row tiles.
+// tm_a always has a box of (128 bytes x 128 rows). Both maps use the 128-byte swizzle.
+cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p,
+                        int grid, cudaStream_t stream);
+
+// how many CTA pairs of the pair-mode kernel can be resident at once on the current device (0 if none)
+int gemm_max_resident_pairs(int dtype);
 
 }  // namespace mpg

@@ -13,6 +13,14 @@ pytestmark = pytest.mark.gpu
 DTYPES = [orc.FP16, orc.BF16, orc.TF32]
 
 
+@pytest.fixture(params=["single", "pair"], autouse=True)
+def tile_policy(request):
+    """Every test of this file runs under both tilings of the kernel: whole tiles per CTA, and CTA pairs."""
+    assert mpg.mpgemmfi_set_tile_policy(mpg.TILES_PAIR if request.param == "pair" else mpg.TILES_SINGLE) == 0
+    yield request.param
+    mpg.mpgemmfi_set_tile_policy(mpg.TILES_AUTO)
+
+
 def site(kind, row=0, col=0, k=0, mask=0):
     s = np.zeros(1, dtype=orc.SITE)
     s["kind"], s["row"], s["col"], s["k"], s["xor_mask"] = kind, row, col, k, mask
