@@ -35,6 +35,7 @@ constexpr uint32_t NONE = 0xFFFFFFFFu;
 constexpr int BM = 128;
 constexpr int NUM_THREADS = 256;
 constexpr int MAX_STAGES = 8;
+constexpr int OUT_STAGING_BYTES = 4 * 32 * 128;   // output staging for the epilogue's TMA stores
 
 template <int BN, bool kPair>
 struct Cfg {
@@ -318,7 +319,8 @@ __device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid,
 // kPair = true : grid of CTA pairs (cluster dimension 2), tiles 256 x BN, BN = 256.
 template <int BN, bool kTF32, bool kPair>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const GemmParams p)
+gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+            const __grid_constant__ CUtensorMap tm_c, const GemmParams p)
 {
     using C = Cfg<BN, kPair>;
     constexpr int KT = kTF32 ? 32 : 64;      // elements per 128-byte row
@@ -328,7 +330,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    Control *ctl = reinterpret_cast<Control *>(smem + STAGES * C::STAGE_BYTES);
+    uint8_t *stage_out = smem + STAGES * C::STAGE_BYTES;     // 4 epilogue warps x (32 rows x 128 bytes)
+    Control *ctl = reinterpret_cast<Control *>(stage_out + OUT_STAGING_BYTES);
     volatile uint32_t *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -351,6 +354,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         mbar_fence_init();
         tma_prefetch_desc(&tm_a);
         tma_prefetch_desc(&tm_b);
+        if (p.c_vec_ok) tma_prefetch_desc(&tm_c);
     }
     if (warp == 2) {
         if constexpr (kPair) { tmem_alloc_pair(smem_u32(&ctl->tmem_base), C::TMEM_COLS); tmem_relinquish_pair(); }
@@ -517,6 +521,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         const bool do_corr = do_bound && (p.detect_mode & MPGEMMFI_CORRECT);
         uint32_t lt = 0, pause_phase = 0, n_det = 0;
         uint32_t *bitmap = p.flags ? p.flags + MPGEMMFI_HEADER_WORDS + 4 * (size_t)p.n_faults : nullptr;
+        uint8_t *my_out = stage_out + q * (32 * 128);
         bool ok = true;
         for (uint32_t t = gid; ok && t < (uint32_t)p.num_tiles; t += groups, ++lt) {
             const uint32_t as = lt & 1u, ap = (lt >> 1) & 1u;
@@ -578,18 +583,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 }
                 if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 1);
                 flagw[c] = fw;
-                if (row_ok) {
-                    if (c0 + 32 <= (uint32_t)p.N && p.c_vec_ok) {
-                        float4 *dst = reinterpret_cast<float4 *>(crow + c0);
+                if (p.c_vec_ok) {
+                    // stage the warp's 32 x 32 block (128-byte swizzle: 16-byte piece j of row r sits in
+                    // slot j ^ (r & 7)) and let TMA write it out in whole rows; TMA drops what lies
+                    // outside the matrix
+                    if (lane == 0) tma_store_wait_read();       // the previous block has left the staging area
+                    __syncwarp();
+                    uint8_t *srow = my_out + lane * 128;
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            dst[j] = make_float4(bits_f32(v[4 * j]), bits_f32(v[4 * j + 1]), bits_f32(v[4 * j + 2]),
-                                                 bits_f32(v[4 * j + 3]));
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (c0 + j < (uint32_t)p.N) crow[c0 + j] = bits_f32(v[j]);
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4 *>(srow + ((j ^ (lane & 7)) << 4)) =
+                            make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    const uint32_t row0 = tc.m0 + (uint32_t)(q * 32);
+                    if (lane == 0 && row0 < (uint32_t)p.M && c0 < (uint32_t)p.N) {
+                        tma_store_2d(&tm_c, smem_u32(my_out), (int)c0, (int)row0);
+                        tma_store_commit();
                     }
+                } else if (row_ok) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (c0 + j < (uint32_t)p.N) crow[c0 + j] = bits_f32(v[j]);
                 }
             }
             if (bitmap && row_ok) {
@@ -601,6 +616,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 }
             }
         }
+        if (lane == 0) tma_store_wait_all();     // every block this warp sent out has been written
         n_det = __reduce_add_sync(0xFFFFFFFFu, n_det);
         if (lane == 0 && n_det && p.flags) {
             atomicAdd(&p.flags[1], n_det);
@@ -620,11 +636,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
 }
 
 template <int BN, bool kTF32, bool kPair>
-cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p, int grid,
-                       cudaStream_t stream)
+cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c, const GemmParams &p,
+                       int grid, cudaStream_t stream)
 {
     using C = Cfg<BN, kPair>;
-    const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + sizeof(Control) + 1024;
+    const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024;
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -646,7 +662,7 @@ cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const G
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, kTF32, kPair>, tm_a, tm_b, p);
+    return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, kTF32, kPair>, tm_a, tm_b, tm_c, p);
 }
 
 }  // namespace
@@ -659,7 +675,7 @@ int gemm_max_resident_pairs(int dtype)
     const int tf = dtype == MPGEMMFI_TF32 ? 1 : 0;
     if (cache[dev][tf] == 0) {
         using C = Cfg<256, true>;
-        const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + sizeof(Control) + 1024;
+        const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024;
         auto kern = tf ? gemm_kernel<256, true, true> : gemm_kernel<256, false, true>;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
         cudaLaunchConfig_t cfg = {};
@@ -686,17 +702,17 @@ int gemm_stage_count(int bn, bool pair)
     return bn == 256 ? Cfg<256, false>::STAGES : (bn == 128 ? Cfg<128, false>::STAGES : Cfg<64, false>::STAGES);
 }
 
-cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p,
-                        int grid, cudaStream_t stream)
+cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c,
+                        const GemmParams &p, int grid, cudaStream_t stream)
 {
     const bool tf32 = p.dtype == MPGEMMFI_TF32;
     if (pair)
-        return tf32 ? launch_one<256, true, true>(tm_a, tm_b, p, grid, stream)
-                    : launch_one<256, false, true>(tm_a, tm_b, p, grid, stream);
+        return tf32 ? launch_one<256, true, true>(tm_a, tm_b, tm_c, p, grid, stream)
+                    : launch_one<256, false, true>(tm_a, tm_b, tm_c, p, grid, stream);
     switch (bn) {
-    case 256: return tf32 ? launch_one<256, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<256, false, false>(tm_a, tm_b, p, grid, stream);
-    case 128: return tf32 ? launch_one<128, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<128, false, false>(tm_a, tm_b, p, grid, stream);
-    default:  return tf32 ? launch_one<64, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<64, false, false>(tm_a, tm_b, p, grid, stream);
+    case 256: return tf32 ? launch_one<256, true, false>(tm_a, tm_b, tm_c, p, grid, stream) : launch_one<256, false, false>(tm_a, tm_b, tm_c, p, grid, stream);
+    case 128: return tf32 ? launch_one<128, true, false>(tm_a, tm_b, tm_c, p, grid, stream) : launch_one<128, false, false>(tm_a, tm_b, tm_c, p, grid, stream);
+    default:  return tf32 ? launch_one<64, true, false>(tm_a, tm_b, tm_c, p, grid, stream) : launch_one<64, false, false>(tm_a, tm_b, tm_c, p, grid, stream);
     }
 }
 
