@@ -1,0 +1,159 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times (default tile policy).
+
+c1 and c2 are compared in full against the oracle (the oracle's 4096^3 GEMM takes seconds on the host cores).
+The larger configs are compared on sampled outputs that the oracle computes one by one, plus properties
+that hold at any size (flag count = popcount of the bitmap, a flag exactly where the stored value calls for
+one, untouched rows/columns bit-identical to the fault-free run).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2311_05782_b200 as mpg
+import synth
+from parity import TOL, bits_f32, close, run_gpu_campaign, run_gpu_gemm, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def widen_np(dtype, bits):
+    """Library conversions only (numpy half, bit shifts): the test's own view of the operand values."""
+    if dtype == orc.FP16:
+        return bits.view(np.float16).astype(np.float64)
+    if dtype == orc.BF16:
+        return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    return (bits & np.uint32(0xFFFFE000)).view(np.float32).astype(np.float64)
+
+
+def absprod_np(dtype, A, Bt):
+    return np.abs(widen_np(dtype, A)) @ np.abs(widen_np(dtype, Bt)).T
+
+
+def test_c2_full_size_gemm_and_campaign():
+    w = synth.make_workload("c2")
+    M, N, K = w.M, w.N, w.K
+    sites = w.sites[:6]
+    Cg, hdr, log, bm = run_gpu_gemm(w.dtype, w.A, w.Bt, sites, w.detect_mode)
+    assert hdr[0] == 0 and hdr[3] == len(sites)
+    Co, hdr_o, log_o, bm_o = orc.gemm(w.dtype, w.A, w.Bt, sites, w.detect_mode)
+    A2, B2 = w.A.copy(), w.Bt.copy()
+    for s in sites:
+        if s["kind"] == orc.KIND_A:
+            A2[s["row"], s["k"]] = orc.flip_operand(w.dtype, int(A2[s["row"], s["k"]]), int(s["xor_mask"]))
+        else:
+            B2[s["col"], s["k"]] = orc.flip_operand(w.dtype, int(B2[s["col"], s["k"]]), int(s["xor_mask"]))
+    tol = TOL * absprod_np(w.dtype, A2, B2)
+    ok = close(Cg, Co, tol)
+    assert ok.all(), f"{(~ok).sum()} of {ok.size} elements out of tolerance"
+    assert np.array_equal(bm, bm_o) and hdr[1] == hdr_o[1] and hdr[2] == hdr_o[2]
+    assert np.array_equal(log.view(np.uint32), log_o.view(np.uint32))
+    # campaign: all 1024 trials; the oracle recomputes each affected row / column in full
+    Cc, rec = run_gpu_campaign(w.dtype, w.A, w.Bt, w.sites, w.detect_mode)
+    Cclean, *_ = orc.gemm(w.dtype, w.A, w.Bt)
+    assert close(Cc, Cclean, TOL * absprod_np(w.dtype, w.A, w.Bt)).all()
+    ro = orc.campaign(w.dtype, w.A, w.Bt, Cclean, w.sites, w.detect_mode)
+    for f in ("kind", "primary_index", "before_bits", "after_bits", "final_bits", "n_affected"):
+        assert np.array_equal(rec[f], ro[f]), f
+    fragile = (rec["n_detected"] != ro["n_detected"]) | (rec["idx_hash"] != ro["idx_hash"])
+    assert fragile.sum() <= 1, f"{fragile.sum()} trials disagree on their detected sets"
+    good = ~fragile
+    assert np.array_equal(rec["first_detected"][good], ro["first_detected"][good])
+    assert np.array_equal(rec["status"][good] & 6, ro["status"][good] & 6)
+    assert (rec["n_detected"] > 0).sum() > 20        # exponent-MSB flips of an operand light up a whole row/column
+    dev_ok = close(rec["max_abs_dev"], ro["max_abs_dev"], 1e-3 * np.abs(ro["max_abs_dev"]) + 1e-3)
+    assert dev_ok[good].all()
+
+
+def test_c1_full_size_all_trials_in_one_gemm_and_as_campaign():
+    from parity import check_campaign_against_oracle, check_gemm_against_oracle
+    w = synth.make_workload("c1")
+    check_gemm_against_oracle(w.dtype, w.A, w.Bt, w.sites, w.detect_mode, max_fragile=1)
+    check_campaign_against_oracle(w.dtype, w.A, w.Bt, w.sites, w.detect_mode, max_fragile=1)
+
+
+@pytest.mark.parametrize("name", ["c3a", "c3b", "c4", "c5"])
+def test_large_configs_on_sampled_outputs(name):
+    w = synth.make_workload(name, trials=256)
+    M, N, K = w.M, w.N, w.K
+    a, b = to_dev(w.A, w.dtype), to_dev(w.Bt, w.dtype)
+    # fault-free run, then a run with the first sites of the table
+    C0, f0 = mpg.gemm(w.dtype, a, b, None, w.detect_mode)
+    n_sites = 16
+    sites = w.sites[:n_sites]
+    C1, f1 = mpg.gemm(w.dtype, a, b, sites, w.detect_mode)
+    torch.cuda.synchronize()
+    hdr0, _, bm0 = mpg.split_flags(f0, M, N, 0)
+    hdr1, log1, bm1 = mpg.split_flags(f1, M, N, n_sites)
+    assert hdr0[0] == 0 and hdr0[1] == 0 and not bm0.any()          # clean workloads raise no flag
+    assert hdr1[0] == 0 and hdr1[3] == n_sites
+    assert sum(int(x) for x in np.bitwise_count(bm1).reshape(-1)) == hdr1[1]
+    # sampled clean outputs against the oracle, tile corners and tails included
+    rng = np.random.default_rng(5)
+    si = np.concatenate([rng.integers(0, M, 3000), [0, M - 1, 0, M - 1, 127, 128, 255, 256]]).astype(np.uint32)
+    sj = np.concatenate([rng.integers(0, N, 3000), [0, N - 1, N - 1, 0, N - 1, 0, 63, 32]]).astype(np.uint32)
+    ref, ap = orc.sample(w.dtype, w.A, w.Bt, si, sj)
+    got0 = C0[torch.from_numpy(si.astype(np.int64)).cuda(), torch.from_numpy(sj.astype(np.int64)).cuda()].cpu().numpy()
+    assert close(got0, ref, TOL * ap).all()
+    # the faulty run: rows / columns / elements no site reaches are bit-identical to the fault-free run
+    hit_rows = set(int(s["row"]) for s in sites if s["kind"] != orc.KIND_B)
+    hit_cols = set(int(s["col"]) for s in sites if s["kind"] == orc.KIND_B)
+    same = (C0 == C1) | (torch.isnan(C0) & torch.isnan(C1))
+    rows_ok = torch.ones(M, dtype=torch.bool, device="cuda"); rows_ok[list(hit_rows)] = False
+    cols_ok = torch.ones(N, dtype=torch.bool, device="cuda")
+    if hit_cols:
+        cols_ok[list(hit_cols)] = False
+    assert bool(same[rows_ok][:, cols_ok].all())
+    # each site against the oracle's element-level view
+    for t, s in enumerate(sites):
+        kind, i, j = int(s["kind"]), int(s["row"]), int(s["col"])
+        lg = log1[t]
+        assert lg["status"] & 1
+        if kind in (orc.KIND_A, orc.KIND_B):
+            src = w.A[i, s["k"]] if kind == orc.KIND_A else w.Bt[j, s["k"]]
+            assert lg["before_bits"] == int(src) and lg["after_bits"] == orc.flip_operand(w.dtype, int(src), int(s["xor_mask"]))
+            # a few elements of the affected row / column, recomputed by the oracle with the faulty operand
+            other = rng.integers(0, N if kind == orc.KIND_A else M, 64).astype(np.uint32)
+            fix = np.full(64, i if kind == orc.KIND_A else j, dtype=np.uint32)
+            ri, rj = (fix, other) if kind == orc.KIND_A else (other, fix)
+            ref1, ap1 = orc.sample(w.dtype, w.A, w.Bt, ri, rj, sites)
+            got1 = C1[torch.from_numpy(ri.astype(np.int64)).cuda(), torch.from_numpy(rj.astype(np.int64)).cuda()].cpu().numpy()
+            if w.detect_mode & orc.CORRECT:
+                ref1 = np.array([bits_f32(orc.boundcheck_correct(int(x))) for x in ref1.view(np.uint32)], dtype=np.float32)
+            assert close(got1, ref1, TOL * ap1).all()
+        else:
+            assert lg["after_bits"] == lg["before_bits"] ^ s["xor_mask"]
+            stored = int(C1[i, j].cpu().numpy().view(np.uint32))
+            flagged = bool((bm1[i, j // 32] >> (j % 32)) & 1)
+            if kind == orc.KIND_OUT:
+                r0, a0 = orc.sample(w.dtype, w.A, w.Bt, np.array([i], np.uint32), np.array([j], np.uint32))
+                assert close(bits_f32(lg["before_bits"]), r0[0], TOL * a0[0])
+                want = orc.boundcheck_correct(int(lg["after_bits"])) if w.detect_mode & orc.CORRECT else int(lg["after_bits"])
+                assert stored == want and flagged == bool(orc.boundcheck_detect(int(lg["after_bits"])))
+            elif not (w.detect_mode & orc.CORRECT):
+                assert flagged == bool(orc.boundcheck_detect(stored))
+    # campaign on the same table: single-element trials are exact against the oracle's element evaluation
+    Cc, rec = run_gpu_campaign(w.dtype, w.A, w.Bt, w.sites, w.detect_mode)
+    elem = np.isin(w.sites["kind"], [orc.KIND_ACC, orc.KIND_TERM])
+    if elem.any():
+        idx = np.nonzero(elem)[0][:64]
+        for t in idx:
+            s = w.sites[t]
+            i, j = int(s["row"]), int(s["col"])
+            # the oracle on the 1 x 1 problem made of row i of A and row j of Bt is the same dot product
+            sub = s.copy().reshape(1); sub["row"] = 0; sub["col"] = 0
+            Cs, *_ = orc.gemm(w.dtype, w.A[i:i + 1], w.Bt[j:j + 1])
+            ro = orc.campaign(w.dtype, w.A[i:i + 1], w.Bt[j:j + 1], Cs, sub, w.detect_mode)[0]
+            raw = orc.campaign(w.dtype, w.A[i:i + 1], w.Bt[j:j + 1], Cs, sub, w.detect_mode & ~orc.CORRECT)[0]
+            g = rec[t]
+            assert g["before_bits"] == ro["before_bits"] and g["after_bits"] == ro["after_bits"]
+            assert g["n_detected"] == ro["n_detected"] and (g["status"] & 7) == (ro["status"] & 7)
+            if not np.isnan(bits_f32(raw["final_bits"])):      # NaN payloads are not part of parity
+                assert g["final_bits"] == ro["final_bits"] and g["max_abs_dev"] == ro["max_abs_dev"]
+    out = w.sites["kind"] == orc.KIND_OUT
+    for t in np.nonzero(out)[0][:64]:
+        s = w.sites[t]
+        g = rec[t]
+        assert g["before_bits"] == int(Cc[int(s["row"]), int(s["col"])].view(np.uint32))
+        assert g["after_bits"] == g["before_bits"] ^ s["xor_mask"]
+        assert g["n_detected"] == orc.boundcheck_detect(int(g["after_bits"]))
