@@ -34,8 +34,27 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-WORKLOAD = "c2"
+WORKLOAD = "c2"      # the configuration the headline metric is quoted on; --config times another one
 METRIC = "fault-injected GEMM TFLOP/s"
+DTYPE_NAMES = {0: "fp16", 1: "bf16", 2: "tf32"}
+WORKLOAD_TEXT = {
+    "c1": "c1: FP16 GEMM M=N=K=256, A,B ~ N(0,1)/16; per step one single-bit output-element fault from the seeded "
+          "64-trial table; BoundCheck detection",
+    "c2": "c2: BF16 GEMM M=N=K=4096, A,B ~ N(0,1)/64, FP32 accumulate and output; per step one single-bit operand "
+          "fault (A or B, bit 0-15) from the seeded 1024-trial table; BoundCheck detection+correction",
+    "c3a": "c3a: FP16 GEMM M=16384 N=4096 K=1024, A ~ N(0,1), B ~ N(0,0.02); per step one single-bit output-element "
+           "fault from the seeded 4096-trial table; BoundCheck detection",
+    "c3b": "c3b: FP16 GEMM M=16384 N=1024 K=4096, A ~ GELU(N(0,1)), B ~ N(0,0.02); per step one single-bit "
+           "output-element fault from the seeded 4096-trial table; BoundCheck detection",
+    "c4": "c4: TF32 GEMM M=N=K=8192, A,B ~ U(-1,1); per step one accumulator fault (two adjacent bits after a "
+          "uniformly chosen k-step boundary) from the seeded 2048-trial table; BoundCheck detection",
+    "c5": "c5: FP16 GEMM M=802816 N=64 K=576 (im2col of a 3x3 conv), A ~ ReLU(N(0,1)), B ~ N(0,sqrt(2/576)); per step "
+          "one single-bit fault from the seeded 100000-trial table (operand / accumulator / output mix); BoundCheck "
+          "detection+correction",
+}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMM kernel, from the ncu capture summarised
+# under profiles/; None once the kernel has changed since the counters were taken
+KERNEL_TRAFFIC_BYTES = {"c2": None}
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 
 
@@ -121,14 +140,15 @@ def oracle_sample_run(w, rows, n_sites=1):
 def cpu_baseline(w, budget_s=12.0):
     import oracle as orc
     orc.build()
-    t_probe = oracle_sample_run(w, 32)
-    rows = int(min(w.M, max(32, 32 * budget_s / max(t_probe, 1e-3))))
+    t_small, t_probe = oracle_sample_run(w, 32), oracle_sample_run(w, 160)
+    per_row = max((t_probe - t_small) / 128.0, 1e-6)          # the fixed part (widening Bt) is not per-row work
+    rows = int(min(w.M, max(160, (budget_s - t_small) / per_row)))
     rows = max(32, (rows // 32) * 32)
     t = oracle_sample_run(w, rows)
     flops = 2.0 * rows * w.N * w.K
     return {"value": flops / t / 1e12, "unit": "TFLOP/s", "cores": orc.num_threads(), "kind": "oracle",
-            "sample": f"rows 0..{rows - 1} of A ({rows}x{w.N}x{w.K} of the {w.M}x{w.N}x{w.K} GEMM), one operand site, "
-                      f"BoundCheck+correction, {t:.2f} s"}
+            "sample": f"rows 0..{rows - 1} of A ({rows}x{w.N}x{w.K} of the {w.M}x{w.N}x{w.K} GEMM), one site of the "
+                      f"trial table, the config's check, {t:.2f} s"}
 
 
 def run_reference(args):
@@ -170,6 +190,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
+    ap.add_argument("--config", default=WORKLOAD, help="workload to time (c1, c2, c3a, c3b, c4, c5); default c2")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
@@ -194,13 +215,14 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     mpg.load_library()
 
-    w = synth.make_workload(WORKLOAD)
+    w = synth.make_workload(args.config)
     M, N, K, dtype, mode = w.M, w.N, w.K, w.dtype, w.detect_mode
+    view = np.int32 if dtype == synth.DTYPE_TF32 else np.int16
     lo, hi = shard_range(len(w.sites), rank, world)          # this rank's share of the trial table
     my_sites = w.sites[lo:hi]
     dev = torch.device("cuda", local_rank)
-    A = torch.from_numpy(w.A.view(np.int16)).to(dev)
-    Bt = torch.from_numpy(w.Bt.view(np.int16)).to(dev)
+    A = torch.from_numpy(w.A.view(view)).to(dev)
+    Bt = torch.from_numpy(w.Bt.view(view)).to(dev)
     sites_dev = torch.from_numpy(my_sites.view(np.int32).reshape(-1, 8)).to(dev)
     C = torch.empty((M, N), dtype=torch.float32, device=dev)
     flags = torch.empty(mpg.mpgemmfi_flags_bytes(M, N, 1) // 4, dtype=torch.int32, device=dev)
@@ -272,15 +294,16 @@ def main():
         if rc != 0:
             raise mpg.MpgemmfiError(rc, "mpgemmfi_campaign")
 
-    camp_steps = max(5, min(200, args.steps // 10))
-    ms_camp, _ = timed(campaign_step, camp_steps, 3)
+    ms_one, _ = timed(campaign_step, 1, 3)
+    camp_steps = max(3, min(200, args.steps // 10, int(3000.0 / max(ms_one, 1e-3))))     # about 3 s of launches
+    ms_camp, _ = timed(campaign_step, camp_steps, 0)
     ms_camp_max = reduce_max(ms_camp, world, dev)
     trials_total = reduce_sum(float(n_my * camp_steps), world, dev)
     trials_per_s = trials_total / (ms_camp_max * 1e-3)
 
     # ---- end to end: pinned host buffers, copies inside the timed region
-    hA = torch.from_numpy(w.A.view(np.int16)).pin_memory()
-    hB = torch.from_numpy(w.Bt.view(np.int16)).pin_memory()
+    hA = torch.from_numpy(w.A.view(view)).pin_memory()
+    hB = torch.from_numpy(w.Bt.view(view)).pin_memory()
     hS = torch.from_numpy(my_sites.view(np.int32).reshape(-1, 8)).pin_memory()
     hC = torch.empty((M, N), dtype=torch.float32).pin_memory()
     hF = torch.empty(flags.numel(), dtype=torch.int32).pin_memory()
@@ -301,11 +324,27 @@ def main():
     ms_e2e, _ = timed(e2e_step, e2e_steps, 3)
     ms_e2e_max = reduce_max(ms_e2e, world, dev)
     e2e_value = reduce_sum(flops * e2e_steps, world, dev) / (ms_e2e_max * 1e-3) / 1e12
-    h2d = hA.numel() * 2 + hB.numel() * 2 + 32
+    h2d = hA.numel() * hA.element_size() + hB.numel() * hB.element_size() + 32
     d2h = hC.numel() * 4 + hF.numel() * 4
 
     peaks, peak_src = load_peaks()
     achieved = flops / (ms_inj / args.steps * 1e-3) / 1e12
+
+    min_bytes = (M * K + N * K) * A.element_size() + M * N * 4 + M * ((N + 31) // 32) * 4
+    if args.config == "c5":
+        # narrow N: about 52 flop per byte, below the ridge; the GEMM is bound by HBM
+        gbs = min_bytes / (ms_inj / args.steps * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peak_src} (copy bandwidth)",
+                    "kernel": "gemm_kernel", "bytes_per_launch": min_bytes}
+    else:
+        tensor_peak = peaks["bf16_tflops"] * (0.5 if dtype == synth.DTYPE_TF32 else 1.0)
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": tensor_peak, "unit": "TFLOP/s",
+                    "frac": achieved / tensor_peak, "traffic": KERNEL_TRAFFIC_BYTES.get(args.config),
+                    "peak_source": f"{peak_src} (cuBLAS bf16 burst" + (", halved for tf32)" if dtype == synth.DTYPE_TF32 else ")"),
+                    "frac_of_sustained": achieved / (peaks["bf16_tflops_sustained"] * (0.5 if dtype == synth.DTYPE_TF32 else 1.0)),
+                    "frac_of_nominal": achieved / (1125.0 if dtype == synth.DTYPE_TF32 else 2250.0),
+                    "kernel": "gemm_kernel", "flops_per_launch": flops, "min_bytes_per_launch": min_bytes}
 
     if rank == 0:
         baseline = None
@@ -314,10 +353,8 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_inj_max / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "c2: BF16 GEMM M=N=K=4096, A,B ~ N(0,1)/64, FP32 accumulate and output; per step one "
-                                   "single-bit operand fault (A or B, bit 0-15) from the seeded 1024-trial table; "
-                                   "BoundCheck detection+correction",
+            "scaling": "weak", "vs_baseline": None, "dtype": DTYPE_NAMES[dtype], "data": "synthetic",
+            "config": {"workload": WORKLOAD_TEXT[args.config],
                        "l2": "flushed (256 MB memset) before every timed step",
                        "timing": "sum of per-step CUDA-event intervals on the launching stream",
                        "trials_per_rank": n_my},
@@ -325,12 +362,7 @@ def main():
             "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "ms_per_step": ms_e2e_max / e2e_steps},
             "gpu_launches": args.steps,
-            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                         "frac": achieved / peaks["bf16_tflops"], "traffic": None,
-                         "peak_source": f"{peak_src} (cuBLAS bf16 burst)",
-                         "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
-                         "frac_of_nominal_2250": achieved / 2250.0,
-                         "kernel": "gemm_kernel<256,bf16>", "flops_per_launch": flops},
+            "roofline": roofline,
             "injection_off": {"tflops": tflops_off, "steps": off_steps,
                               "injected_over_plain_time": tflops_off / tflops_on_local},
             "campaign": {"trials_per_s": trials_per_s, "trials_per_launch": n_my, "launches": camp_steps,

@@ -86,21 +86,6 @@ int encode_operand_map(CUtensorMap *map, int dtype, const void *base, int rows, 
 
 int g_tile_policy = MPGEMMFI_TILES_AUTO;
 
-// C as an M x N FP32 tensor, boxes of 32 columns x 32 rows (one 128-byte row segment each), 128-byte swizzle
-int encode_output_map(CUtensorMap *map, float *C, int M, int N)
-{
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return cuda_fail(cudaErrorUnknown);
-    const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-    const cuuint64_t strides[1] = {(cuuint64_t)N * sizeof(float)};
-    const cuuint32_t box[2] = {32, 32};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return MPGEMMFI_ERR_CUDA; }
-    return MPGEMMFI_OK;
-}
-
 // widest tile that still gives every SM a tile; narrow outputs get narrow tiles
 int choose_bn(int M, int N, int num_sms)
 {
@@ -158,21 +143,13 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
     p.wpr = (N + 31) / 32;
     p.c_vec_ok = (N % 4 == 0) && (((uintptr_t)C & 15) == 0);
     p.A = A; p.Bt = Bt; p.C = C; p.sites = sites; p.flags = flags;
-    CUtensorMap tm_c;
-    if (p.c_vec_ok) {
-        rc = encode_output_map(&tm_c, C, M, N);
-        if (rc) return rc;
-    } else {
-        memset(&tm_c, 0, sizeof(tm_c));
-    }
-
     if (flags) {
         const cudaError_t e = cudaMemsetAsync(flags, 0, sizeof(uint32_t) * (MPGEMMFI_HEADER_WORDS + 4 * (size_t)n_faults), stream);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     const int walkers = pair ? max_pairs : di.num_sms;
     const int grid = (p.num_tiles < walkers ? p.num_tiles : walkers) * (pair ? 2 : 1);
-    const cudaError_t e = mpg::launch_gemm(bn, pair, tm_a, tm_b, tm_c, p, grid, stream);
+    const cudaError_t e = mpg::launch_gemm(bn, pair, tm_a, tm_b, p, grid, stream);
     return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
 }
 

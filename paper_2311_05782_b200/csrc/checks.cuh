@@ -64,10 +64,11 @@ MPG_HD uint32_t site_boundary(const mpgemmfi_site &s, int dtype, int K)
     return s.k / ks + 1;   // TERM: the boundary that ends the k-step containing k
 }
 
-// ---- BoundCheck: exponent bit 7 set and any of exponent bits 6..4 set ("1eeexxxx")
+// ---- BoundCheck: exponent bit 7 set and any of exponent bits 6..4 set ("1eeexxxx"), i.e. an
+// exponent field of 0x90 or more: the magnitude bits are at least those of 131072.0f
 MPG_HD bool boundcheck_detect(uint32_t bits)
 {
-    return (bits & 0x40000000u) != 0 && (bits & 0x38000000u) != 0;
+    return (bits & 0x7FFFFFFFu) >= 0x48000000u;
 }
 MPG_HD uint32_t boundcheck_clear(uint32_t bits) { return bits & ~0x38000000u; }
 

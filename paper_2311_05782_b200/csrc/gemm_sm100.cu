@@ -7,8 +7,9 @@
 //             sites in the staged tiles before the tensor core reads them; pauses at the
 //             k-step boundaries where an accumulator or product-term site takes effect
 //   warp 2    TMEM allocation / release
-//   warps 4-7 epilogue: TMEM -> registers, accumulator / term write-back sites at the
-//             paused boundaries, output-site flips, BoundCheck flags (+ correction), stores
+//   warps 4-11 epilogue (warp w: TMEM lanes 32*(w%4).., left or right half of the tile's columns):
+//             TMEM -> registers, accumulator / term write-back sites at the paused boundaries,
+//             output-site flips, BoundCheck flags (+ correction), stores
 //
 // The fault-site table is decoded once per CTA into a list of the entries that touch any of
 // its tiles; a CTA whose list is empty never looks at a site again.
@@ -33,9 +34,11 @@ namespace {
 
 constexpr uint32_t NONE = 0xFFFFFFFFu;
 constexpr int BM = 128;
-constexpr int NUM_THREADS = 256;
+constexpr int NUM_THREADS = 384;     // 4 control warps + 8 epilogue warps
+constexpr int EPI_WARPS = 8;
+constexpr int SITE_CACHE = 64;
 constexpr int MAX_STAGES = 8;
-constexpr int OUT_STAGING_BYTES = 4 * 32 * 128;   // output staging for the epilogue's TMA stores
+constexpr int OUT_STAGING_BYTES = EPI_WARPS * 16 * 128;   // a 16-row x 32-column FP32 block per epilogue warp
 
 template <int BN, bool kPair>
 struct Cfg {
@@ -61,8 +64,9 @@ struct alignas(16) Control {
     uint32_t abort_flag;
     uint32_t site_count;
     uint32_t pad;
-    uint32_t scan[NUM_THREADS];
+    uint32_t scan[NUM_THREADS / 32];
     uint16_t site_idx[MPGEMMFI_MAX_FAULTS];
+    mpgemmfi_site site_cache[SITE_CACHE];     // the first entries of the CTA's list, so that scans stay on chip
 };
 
 // Ranges of one output tile as seen by one CTA. In single mode "own" and "tile" coincide; in pair
@@ -81,13 +85,20 @@ __device__ __forceinline__ bool in_tile_rows(const TileCtx &c, uint32_t row) { r
 __device__ __forceinline__ bool in_tile_cols(const TileCtx &c, uint32_t col) { return col - c.n0 < c.bn; }
 __device__ __forceinline__ bool in_own_b(const TileCtx &c, uint32_t col) { return col - c.b0 < c.b_rows; }
 
+// entry i of the CTA's site list: from shared memory for the first SITE_CACHE entries
+__device__ __forceinline__ mpgemmfi_site listed_site(const TileCtx &c, uint32_t i)
+{
+    if (i < (uint32_t)SITE_CACHE) return c.ctl->site_cache[i];
+    return load_site(c.p->sites, c.ctl->site_idx[i]);
+}
+
 // smallest k-tile >= kt_from in which this tile has an operand site (warp-wide)
 __device__ uint32_t scan_next_operand(const TileCtx &c, uint32_t kt_from, int lane)
 {
     const uint32_t ks = (uint32_t)kstep_of(c.p->dtype);
     uint32_t best = NONE;
     for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
-        const mpgemmfi_site s = load_site(c.p->sites, c.ctl->site_idx[i]);
+        const mpgemmfi_site s = listed_site(c, i);
         const bool hit = (s.kind == MPGEMMFI_SITE_A && in_own_rows(c, s.row)) ||
                          (s.kind == MPGEMMFI_SITE_B && in_own_b(c, s.col));
         if (hit && s.k / ks >= kt_from) best = min(best, s.k / ks);
@@ -100,7 +111,7 @@ __device__ uint32_t scan_next_boundary(const TileCtx &c, uint32_t b_from, int la
 {
     uint32_t best = NONE;
     for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
-        const mpgemmfi_site s = load_site(c.p->sites, c.ctl->site_idx[i]);
+        const mpgemmfi_site s = listed_site(c, i);
         if ((s.kind == MPGEMMFI_SITE_ACC || s.kind == MPGEMMFI_SITE_TERM) && in_tile_rows(c, s.row) &&
             in_tile_cols(c, s.col)) {
             const uint32_t b = site_boundary(s, c.p->dtype, c.p->K);
@@ -114,7 +125,7 @@ __device__ bool scan_has_out(const TileCtx &c, int lane)
 {
     bool any = false;
     for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
-        const mpgemmfi_site s = load_site(c.p->sites, c.ctl->site_idx[i]);
+        const mpgemmfi_site s = listed_site(c, i);
         any |= s.kind == MPGEMMFI_SITE_OUT && in_own_rows(c, s.row) && in_tile_cols(c, s.col);
     }
     return __any_sync(0xFFFFFFFFu, any);
@@ -146,7 +157,7 @@ __device__ void apply_operand_sites(const TileCtx &c, uint32_t kt, uint8_t *smem
     const uint32_t es = (uint32_t)esize_of(p.dtype);
     for (uint32_t i = 0; i < c.ctl->site_count; ++i) {
         const uint32_t idx = c.ctl->site_idx[i];
-        const mpgemmfi_site s = load_site(p.sites, idx);
+        const mpgemmfi_site s = listed_site(c, i);
         uint8_t *tile;
         uint32_t r;
         bool log_here;
@@ -177,7 +188,7 @@ __device__ uint32_t faulty_operand(const TileCtx &c, bool is_a, uint32_t rc, uin
     const GemmParams &p = *c.p;
     uint32_t w = load_operand(p.dtype, is_a ? p.A : p.Bt, (size_t)rc * p.K + k);
     for (uint32_t i = 0; i < c.ctl->site_count; ++i) {
-        const mpgemmfi_site s = load_site(p.sites, c.ctl->site_idx[i]);
+        const mpgemmfi_site s = listed_site(c, i);
         if (s.k != k) continue;
         if (is_a ? (s.kind == MPGEMMFI_SITE_A && s.row == rc) : (s.kind == MPGEMMFI_SITE_B && s.col == rc))
             w = flip_operand(p.dtype, w, s.xor_mask);
@@ -185,19 +196,19 @@ __device__ uint32_t faulty_operand(const TileCtx &c, bool is_a, uint32_t rc, uin
     return w;
 }
 
-// Epilogue warp of lane quarter q: apply, in table order, the accumulator and term sites of
-// boundary b that live in its 32 TMEM lanes.
-__device__ void apply_boundary_sites(const TileCtx &c, uint32_t b, uint32_t tmem_acc, int q, int lane)
+// Epilogue warp of lane quarter q and column half h: apply, in table order, the accumulator and
+// term sites of boundary b that live in its 32 TMEM lanes and its half of the columns.
+__device__ void apply_boundary_sites(const TileCtx &c, uint32_t b, uint32_t tmem_acc, int q, int h, int lane)
 {
     const GemmParams &p = *c.p;
     for (uint32_t i = 0; i < c.ctl->site_count; ++i) {
         const uint32_t idx = c.ctl->site_idx[i];
-        const mpgemmfi_site s = load_site(p.sites, idx);
+        const mpgemmfi_site s = listed_site(c, i);
         if (!(s.kind == MPGEMMFI_SITE_ACC || s.kind == MPGEMMFI_SITE_TERM)) continue;
         if (!in_own_rows(c, s.row) || !in_tile_cols(c, s.col)) continue;
         if (site_boundary(s, p.dtype, p.K) != b) continue;
         const uint32_t r = s.row - c.m0;
-        if ((int)(r >> 5) != q) continue;
+        if ((int)(r >> 5) != q || (int)((s.col - c.n0) / (c.bn / 2)) != h) continue;
         const uint32_t taddr = tmem_acc + ((uint32_t)(q * 32) << 16) + (s.col - c.n0);
         uint32_t v = tmem_ld_1(taddr);
         tmem_wait_ld();
@@ -226,18 +237,19 @@ __device__ void apply_boundary_sites(const TileCtx &c, uint32_t b, uint32_t tmem
     }
 }
 
-// Output sites of one thread's row inside the 32-column chunk starting at column c0.
+// Output sites of one thread's row inside the W-column piece starting at column c0.
 // pass 0: XOR and log before/after; pass 1 (after the check): log the final bits.
-__device__ void apply_out_sites(const TileCtx &c, uint32_t row, uint32_t c0, uint32_t (&v)[32], int pass)
+template <int W>
+__device__ void apply_out_sites(const TileCtx &c, uint32_t row, uint32_t c0, uint32_t (&v)[W], int pass)
 {
     const GemmParams &p = *c.p;
     for (uint32_t i = 0; i < c.ctl->site_count; ++i) {
         const uint32_t idx = c.ctl->site_idx[i];
-        const mpgemmfi_site s = load_site(p.sites, idx);
-        if (s.kind != MPGEMMFI_SITE_OUT || s.row != row || s.col - c0 >= 32u) continue;
+        const mpgemmfi_site s = listed_site(c, i);
+        if (s.kind != MPGEMMFI_SITE_OUT || s.row != row || s.col - c0 >= (uint32_t)W) continue;
         const uint32_t j = s.col - c0;
 #pragma unroll
-        for (uint32_t jj = 0; jj < 32; ++jj) {
+        for (uint32_t jj = 0; jj < (uint32_t)W; ++jj) {
             if (jj == j) {
                 if (pass == 0) {
                     const uint32_t before = v[jj];
@@ -272,46 +284,86 @@ __device__ bool site_touches_group(const mpgemmfi_site &s, const GemmParams &p, 
     return ((s.col / BN) * p.tiles_m + s.row / TM) % groups == gid;
 }
 
-// All threads: ordered list of the valid sites that touch a tile of this CTA (pair). CTA 0 also
-// reports invalid entries (skipped) and the applied count.
-template <int TM, int BN>
-__device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid, uint32_t groups)
+// Slice of the site table that one warp examines when the CTA builds its list.
+struct SiteSlice { int beg, end; };
+
+__device__ __forceinline__ SiteSlice site_slice(int n, int warp)
 {
-    const int tid = threadIdx.x;
+    constexpr int WARPS = NUM_THREADS / 32;
+    const int per = ((n + WARPS - 1) / WARPS + 31) / 32 * 32;       // whole 32-entry rounds
+    SiteSlice sl;
+    sl.beg = min(n, warp * per);
+    sl.end = min(n, sl.beg + per);
+    return sl;
+}
+
+// All threads: ordered list of the valid sites that touch a tile of this CTA (pair). CTA 0 also
+// reports invalid entries (skipped) and the applied count. Each warp compacts a contiguous slice
+// of the table with ballots, so the list keeps table order. `first` is the entry this thread
+// examines in its slice's first round, loaded by the caller ahead of time.
+template <int TM, int BN>
+__device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid, uint32_t groups,
+                                const mpgemmfi_site &first)
+{
+    constexpr int WARPS = NUM_THREADS / 32;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n = p.n_faults;
     if (n == 0) {
         if (tid == 0) ctl->site_count = 0;
         return;
     }
-    const int per = (n + NUM_THREADS - 1) / NUM_THREADS;
-    const int beg = min(n, tid * per), end = min(n, beg + per);
-    uint32_t cnt = 0, n_valid = 0, n_bad = 0;
-    for (int i = beg; i < end; ++i) {
-        const mpgemmfi_site s = load_site(p.sites, i);
-        const bool ok = site_valid(s, p.dtype, p.M, p.N, p.K);
-        if (ok) { n_valid++; cnt += site_touches_group<TM, BN>(s, p, gid, groups) ? 1u : 0u; }
-        else {
-            n_bad++;
-            if (blockIdx.x == 0) write_log(p, i, 0u, 0u, 0u, 2u);
+    const SiteSlice sl = site_slice(n, warp);
+    uint32_t cnt = 0, n_valid = 0, n_bad = 0, first_vote = 0;
+    for (int base = sl.beg; base < sl.end; base += 32) {
+        const int i = base + lane;
+        bool ok = false, mine = false;
+        if (i < sl.end) {
+            const mpgemmfi_site s = base == sl.beg ? first : load_site(p.sites, i);
+            ok = site_valid(s, p.dtype, p.M, p.N, p.K);
+            mine = ok && site_touches_group<TM, BN>(s, p, gid, groups);
+            if (!ok && blockIdx.x == 0) write_log(p, i, 0u, 0u, 0u, 2u);
+            n_valid += ok ? 1u : 0u;
+            n_bad += ok ? 0u : 1u;
         }
+        const uint32_t vote = __ballot_sync(0xFFFFFFFFu, mine);
+        if (base == sl.beg) first_vote = vote;
+        cnt += __popc(vote);
     }
     if (blockIdx.x == 0 && p.flags) {
-        if (n_valid) atomicAdd(&p.flags[3], n_valid);
-        if (n_bad) { atomicAdd(&p.flags[4], n_bad); atomicOr(&p.flags[0], MPGEMMFI_STATUS_SITE_SKIPPED); }
+        n_valid = __reduce_add_sync(0xFFFFFFFFu, n_valid);
+        n_bad = __reduce_add_sync(0xFFFFFFFFu, n_bad);
+        if (lane == 0 && n_valid) atomicAdd(&p.flags[3], n_valid);
+        if (lane == 0 && n_bad) { atomicAdd(&p.flags[4], n_bad); atomicOr(&p.flags[0], MPGEMMFI_STATUS_SITE_SKIPPED); }
     }
-    ctl->scan[tid] = cnt;
+    if (lane == 0) ctl->scan[warp] = cnt;
     __syncthreads();
-    if (tid == 0) {
-        uint32_t run = 0;
-        for (int t = 0; t < NUM_THREADS; ++t) { const uint32_t x = ctl->scan[t]; ctl->scan[t] = run; run += x; }
-        ctl->site_count = run;
+    uint32_t off = 0, total = 0;
+    for (int w = 0; w < WARPS; ++w) {
+        const uint32_t x = ctl->scan[w];
+        if (w < warp) off += x;
+        total += x;
     }
-    __syncthreads();
-    uint32_t off = ctl->scan[tid];
-    for (int i = beg; i < end; ++i) {
-        const mpgemmfi_site s = load_site(p.sites, i);
-        if (site_valid(s, p.dtype, p.M, p.N, p.K) && site_touches_group<TM, BN>(s, p, gid, groups))
-            ctl->site_idx[off++] = (uint16_t)i;
+    if (tid == 0) ctl->site_count = total;
+    for (int base = sl.beg; base < sl.end; base += 32) {
+        const int i = base + lane;
+        bool mine = false;
+        mpgemmfi_site s = first;
+        uint32_t vote = first_vote;
+        if (base != sl.beg) {
+            if (i < sl.end) {
+                s = load_site(p.sites, i);
+                mine = site_valid(s, p.dtype, p.M, p.N, p.K) && site_touches_group<TM, BN>(s, p, gid, groups);
+            }
+            vote = __ballot_sync(0xFFFFFFFFu, mine);
+        } else {
+            mine = (vote >> lane) & 1u;
+        }
+        if (mine) {
+            const uint32_t pos = off + __popc(vote & ((1u << lane) - 1u));
+            if (pos < (uint32_t)SITE_CACHE) ctl->site_cache[pos] = s;
+            ctl->site_idx[pos] = (uint16_t)i;
+        }
+        off += __popc(vote);
     }
 }
 
@@ -319,18 +371,17 @@ __device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid,
 // kPair = true : grid of CTA pairs (cluster dimension 2), tiles 256 x BN, BN = 256.
 template <int BN, bool kTF32, bool kPair>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-            const __grid_constant__ CUtensorMap tm_c, const GemmParams p)
+gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const GemmParams p)
 {
     using C = Cfg<BN, kPair>;
     constexpr int KT = kTF32 ? 32 : 64;      // elements per 128-byte row
     constexpr int STAGES = C::STAGES;
     constexpr int TM = kPair ? 2 * BM : BM;  // rows of one tile
-    constexpr uint32_t EPI_ARRIVALS = kPair ? 8 : 4;
+    constexpr uint32_t EPI_ARRIVALS = kPair ? 2 * EPI_WARPS : EPI_WARPS;   // one arrival per epilogue warp
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *stage_out = smem + STAGES * C::STAGE_BYTES;     // 4 epilogue warps x (32 rows x 128 bytes)
+    uint8_t *stage_out = smem + STAGES * C::STAGE_BYTES;     // output staging of the epilogue warps
     Control *ctl = reinterpret_cast<Control *>(stage_out + OUT_STAGING_BYTES);
     volatile uint32_t *abort_flag = &ctl->abort_flag;
 
@@ -340,6 +391,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     const uint32_t gid = kPair ? blockIdx.x >> 1 : blockIdx.x;      // tile walker id
     const uint32_t groups = kPair ? gridDim.x >> 1 : gridDim.x;
     const bool leader = rank == 0;
+
+    // this thread's first entry of the site table: requested now, needed only after the set-up below
+    mpgemmfi_site first_site = {};
+    if (p.n_faults > 0) {
+        const SiteSlice sl = site_slice(p.n_faults, warp);
+        if (sl.beg + lane < sl.end) first_site = load_site(p.sites, sl.beg + lane);
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -354,13 +412,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         mbar_fence_init();
         tma_prefetch_desc(&tm_a);
         tma_prefetch_desc(&tm_b);
-        if (p.c_vec_ok) tma_prefetch_desc(&tm_c);
     }
     if (warp == 2) {
         if constexpr (kPair) { tmem_alloc_pair(smem_u32(&ctl->tmem_base), C::TMEM_COLS); tmem_relinquish_pair(); }
         else { tmem_alloc(smem_u32(&ctl->tmem_base), C::TMEM_COLS); tmem_relinquish(); }
     }
-    build_site_list<TM, BN>(p, ctl, gid, groups);
+    build_site_list<TM, BN>(p, ctl, gid, groups, first_site);
     tc_fence_before_sync();
     if constexpr (kPair) cluster_sync_all(); else __syncthreads();
     tc_fence_after_sync();
@@ -516,12 +573,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         }
     } else if (warp >= 4) {
         // ------------------------------------------------------------ epilogue (own 128 rows)
-        const int q = warp & 3;
+        const int q = warp & 3;               // TMEM lane quarter this warp may access
+        const int h = (warp - 4) >> 2;        // column half of the tile this warp handles
         const bool do_bound = (p.detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK) == MPGEMMFI_DETECT_BOUNDCHECK;
         const bool do_corr = do_bound && (p.detect_mode & MPGEMMFI_CORRECT);
         uint32_t lt = 0, pause_phase = 0, n_det = 0;
         uint32_t *bitmap = p.flags ? p.flags + MPGEMMFI_HEADER_WORDS + 4 * (size_t)p.n_faults : nullptr;
-        uint8_t *my_out = stage_out + q * (32 * 128);
+        uint8_t *my_out = stage_out + (warp - 4) * (16 * 128);
         bool ok = true;
         for (uint32_t t = gid; ok && t < (uint32_t)p.num_tiles; t += groups, ++lt) {
             const uint32_t as = lt & 1u, ap = (lt >> 1) & 1u;
@@ -535,7 +593,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     if (!ok) break;
                     pause_phase ^= 1u;
                     tc_fence_after_sync();
-                    apply_boundary_sites(tc, b, tmem_acc, q, lane);
+                    apply_boundary_sites(tc, b, tmem_acc, q, h, lane);
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) {
@@ -552,71 +610,108 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             tc_fence_after_sync();
 
             const uint32_t row = tc.m0 + (uint32_t)(q * 32 + lane);
+            const uint32_t row0 = tc.m0 + (uint32_t)(q * 32);
             const bool row_ok = row < (uint32_t)p.M;
             float *crow = p.C + (size_t)row * p.N;
-            uint32_t flagw[BN / 32];
-#pragma unroll
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld_32x32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), v);
-                tmem_wait_ld();
-                if (c == BN / 32 - 1) {
-                    // accumulator fully read: hand the TMEM buffer back to the MMA warp
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if constexpr (kPair) mbar_arrive_cluster(lead_acc_empty0 + as * (uint32_t)sizeof(uint64_t));
-                        else mbar_arrive(lead_acc_empty0 + as * (uint32_t)sizeof(uint64_t));
-                    }
-                }
-                const uint32_t c0 = tc.n0 + (uint32_t)(c * 32);
+            const uint32_t t_lane = tmem_acc + ((uint32_t)(q * 32) << 16);
+            constexpr int MY_PIECES = BN / 64;          // 32-column pieces per warp (half the tile's columns)
+            const int first = h * MY_PIECES;
+            uint32_t flagw[MY_PIECES];
+
+            // One 32-column piece of this thread's row: output sites, check, flags, store.
+            auto finish_piece = [&](uint32_t (&v)[32], int i) {
+                const uint32_t c0 = tc.n0 + (uint32_t)((first + i) * 32);
                 if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 0);
                 uint32_t fw = 0;
                 if (do_bound) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        const bool det = boundcheck_detect(v[j]);
-                        fw |= (det ? 1u : 0u) << j;
+                        // exponent field >= 0x90 <=> not (|value| < 131072); NaN compares false, so it is caught
+                        const bool det = !(fabsf(bits_f32(v[j])) < 131072.0f);
+                        if (det) fw |= 1u << j;
                         if (do_corr && det) v[j] = boundcheck_clear(v[j]);
                     }
                     // columns past N hold zeros (zero-filled operand rows) and never flag
                 }
                 if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 1);
-                flagw[c] = fw;
+                flagw[i] = fw;
                 if (p.c_vec_ok) {
-                    // stage the warp's 32 x 32 block (128-byte swizzle: 16-byte piece j of row r sits in
-                    // slot j ^ (r & 7)) and let TMA write it out in whole rows; TMA drops what lies
-                    // outside the matrix
-                    if (lane == 0) tma_store_wait_read();       // the previous block has left the staging area
-                    __syncwarp();
-                    uint8_t *srow = my_out + lane * 128;
+                    // Transpose through shared memory so that every store instruction writes whole
+                    // 128-byte rows, 16 rows at a time: threads of one half-warp park their rows
+                    // (16-byte piece j of row r in slot j ^ (r & 7), conflict-free), then lane l stores
+                    // piece l % 8 of rows l / 8 + 4 i.
+                    const uint32_t j = (uint32_t)lane & 7u;
+                    const uint32_t col = c0 + 4 * j;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        *reinterpret_cast<uint4 *>(srow + ((j ^ (lane & 7)) << 4)) =
-                            make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    const uint32_t row0 = tc.m0 + (uint32_t)(q * 32);
-                    if (lane == 0 && row0 < (uint32_t)p.M && c0 < (uint32_t)p.N) {
-                        tma_store_2d(&tm_c, smem_u32(my_out), (int)c0, (int)row0);
-                        tma_store_commit();
+                    for (int half = 0; half < 2; ++half) {
+                        __syncwarp();                           // the previous rows have been read back
+                        if ((lane >> 4) == half) {
+                            uint8_t *srow = my_out + (lane & 15) * 128;
+#pragma unroll
+                            for (int jj = 0; jj < 8; ++jj)
+                                *reinterpret_cast<uint4 *>(srow + ((jj ^ (lane & 7)) << 4)) =
+                                    make_uint4(v[4 * jj], v[4 * jj + 1], v[4 * jj + 2], v[4 * jj + 3]);
+                        }
+                        __syncwarp();
+#pragma unroll
+                        for (int it = 0; it < 4; ++it) {
+                            const uint32_t r = (uint32_t)(4 * it) + ((uint32_t)lane >> 3);      // row within the 16
+                            const uint4 val = *reinterpret_cast<const uint4 *>(my_out + r * 128 + ((j ^ (r & 7u)) << 4));
+                            const uint32_t grow = row0 + (uint32_t)(16 * half) + r;
+                            if (grow < (uint32_t)p.M && col < (uint32_t)p.N)
+                                *reinterpret_cast<uint4 *>(p.C + (size_t)grow * p.N + col) = val;
+                        }
                     }
                 } else if (row_ok) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (c0 + j < (uint32_t)p.N) crow[c0 + j] = bits_f32(v[j]);
+                    for (int jj = 0; jj < 32; ++jj)
+                        if (c0 + jj < (uint32_t)p.N) crow[c0 + jj] = bits_f32(v[jj]);
+                }
+            };
+            // accumulator columns of this warp fully read: one arrival towards handing the TMEM
+            // buffer back to the MMA warp
+            auto release_acc = [&]() {
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) {
+                    if constexpr (kPair) mbar_arrive_cluster(lead_acc_empty0 + as * (uint32_t)sizeof(uint64_t));
+                    else mbar_arrive(lead_acc_empty0 + as * (uint32_t)sizeof(uint64_t));
+                }
+            };
+
+            // software pipeline: the TMEM read of the next piece is in flight while this one is finished
+            uint32_t va[32], vb[32];
+            const uint32_t t_first = t_lane + (uint32_t)(first * 32);
+            tmem_ld_32x32(t_first, va);
+#pragma unroll
+            for (int i = 0; i < MY_PIECES; i += 2) {
+                tmem_wait_ld();
+                if (i + 1 < MY_PIECES) tmem_ld_32x32(t_first + (uint32_t)((i + 1) * 32), vb);
+                else release_acc();
+                finish_piece(va, i);
+                if (i + 1 < MY_PIECES) {
+                    tmem_wait_ld();
+                    if (i + 2 < MY_PIECES) tmem_ld_32x32(t_first + (uint32_t)((i + 2) * 32), va);
+                    else release_acc();
+                    finish_piece(vb, i + 1);
                 }
             }
             if (bitmap && row_ok) {
-                uint32_t *frow = bitmap + (size_t)row * p.wpr + tc.n0 / 32;
+                const uint32_t w0 = tc.n0 / 32 + (uint32_t)first;
+                uint32_t *frow = bitmap + (size_t)row * p.wpr + w0;
+                if (MY_PIECES == 4 && (p.wpr & 3) == 0) {       // this thread's 4 words are 16-byte aligned
+                    if (w0 < (uint32_t)p.wpr)
+                    *reinterpret_cast<uint4 *>(frow) = make_uint4(flagw[0], flagw[MY_PIECES > 1 ? 1 : 0],
+                                                                   flagw[MY_PIECES > 2 ? 2 : 0], flagw[MY_PIECES > 3 ? 3 : 0]);
+                } else {
 #pragma unroll
-                for (int c = 0; c < BN / 32; ++c) {
-                    if (tc.n0 / 32 + c < (uint32_t)p.wpr) frow[c] = flagw[c];
-                    n_det += __popc(flagw[c]);
+                    for (int i = 0; i < MY_PIECES; ++i)
+                        if (w0 + i < (uint32_t)p.wpr) frow[i] = flagw[i];
                 }
+#pragma unroll
+                for (int i = 0; i < MY_PIECES; ++i) n_det += __popc(flagw[i]);
             }
         }
-        if (lane == 0) tma_store_wait_all();     // every block this warp sent out has been written
         n_det = __reduce_add_sync(0xFFFFFFFFu, n_det);
         if (lane == 0 && n_det && p.flags) {
             atomicAdd(&p.flags[1], n_det);
@@ -636,8 +731,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
 }
 
 template <int BN, bool kTF32, bool kPair>
-cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c, const GemmParams &p,
-                       int grid, cudaStream_t stream)
+cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p, int grid,
+                       cudaStream_t stream)
 {
     using C = Cfg<BN, kPair>;
     const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024;
@@ -662,7 +757,7 @@ cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const C
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, kTF32, kPair>, tm_a, tm_b, tm_c, p);
+    return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, kTF32, kPair>, tm_a, tm_b, p);
 }
 
 }  // namespace
@@ -702,17 +797,17 @@ int gemm_stage_count(int bn, bool pair)
     return bn == 256 ? Cfg<256, false>::STAGES : (bn == 128 ? Cfg<128, false>::STAGES : Cfg<64, false>::STAGES);
 }
 
-cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c,
-                        const GemmParams &p, int grid, cudaStream_t stream)
+cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p,
+                        int grid, cudaStream_t stream)
 {
     const bool tf32 = p.dtype == MPGEMMFI_TF32;
     if (pair)
-        return tf32 ? launch_one<256, true, true>(tm_a, tm_b, tm_c, p, grid, stream)
-                    : launch_one<256, false, true>(tm_a, tm_b, tm_c, p, grid, stream);
+        return tf32 ? launch_one<256, true, true>(tm_a, tm_b, p, grid, stream)
+                    : launch_one<256, false, true>(tm_a, tm_b, p, grid, stream);
     switch (bn) {
-    case 256: return tf32 ? launch_one<256, true, false>(tm_a, tm_b, tm_c, p, grid, stream) : launch_one<256, false, false>(tm_a, tm_b, tm_c, p, grid, stream);
-    case 128: return tf32 ? launch_one<128, true, false>(tm_a, tm_b, tm_c, p, grid, stream) : launch_one<128, false, false>(tm_a, tm_b, tm_c, p, grid, stream);
-    default:  return tf32 ? launch_one<64, true, false>(tm_a, tm_b, tm_c, p, grid, stream) : launch_one<64, false, false>(tm_a, tm_b, tm_c, p, grid, stream);
+    case 256: return tf32 ? launch_one<256, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<256, false, false>(tm_a, tm_b, p, grid, stream);
+    case 128: return tf32 ? launch_one<128, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<128, false, false>(tm_a, tm_b, p, grid, stream);
+    default:  return tf32 ? launch_one<64, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<64, false, false>(tm_a, tm_b, p, grid, stream);
     }
 }
 

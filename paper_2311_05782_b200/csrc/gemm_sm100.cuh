@@ -14,7 +14,7 @@ struct GemmParams {
     int detect_mode, n_faults;
     int tiles_m, tiles_n, num_tiles, num_kt;
     int wpr;        // bitmap words per row = ceil(N / 32)
-    int c_vec_ok;   // C is 16-byte aligned with a 16-byte row pitch: the epilogue stores through TMA (tm_c)
+    int c_vec_ok;   // C is 16-byte aligned with a 16-byte row pitch: the epilogue may use 16-byte stores
     const void *A;
     const void *Bt;
     float *C;
@@ -31,10 +31,8 @@ int gemm_stage_count(int bn, bool pair);
 // Pair mode (pair = true): 256 x 256 tiles walked by CTA pairs; tm_b box is (128 bytes x 128 rows);
 // `grid` is even (two CTAs per pair); p.tiles_m counts 256-row tiles.
 // tm_a always has a box of (128 bytes x 128 rows). Both maps use the 128-byte swizzle.
-// tm_c describes C (FP32, N contiguous) with a box of 32 columns x 32 rows and the 128-byte swizzle; it is
-// only used when p.c_vec_ok is set.
-cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c,
-                        const GemmParams &p, int grid, cudaStream_t stream);
+cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p,
+                        int grid, cudaStream_t stream);
 
 // how many CTA pairs of the pair-mode kernel can be resident at once on the current device (0 if none)
 int gemm_max_resident_pairs(int dtype);

@@ -189,32 +189,6 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const CUtens
         : "memory");
 }
 
-// 2-D tiled store shared -> global (bulk async group); elements outside the tensor are dropped.
-// c0 must address a 16-byte boundary; coordinates must not be negative.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *m, uint32_t src_smem, int c0, int c1)
-{
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src_smem), "r"(c0), "r"(c1)
-                 : "memory");
-}
-
-__device__ __forceinline__ void tma_store_commit()
-{
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-
-// all of this thread's bulk stores have finished READING their shared-memory source
-__device__ __forceinline__ void tma_store_wait_read()
-{
-    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-}
-
-// all of this thread's bulk stores are complete
-__device__ __forceinline__ void tma_store_wait_all()
-{
-    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-}
-
 // ---------------------------------------------------------------- tensor memory
 
 // whole warp; writes the TMEM base address of the allocation to *dst_smem
