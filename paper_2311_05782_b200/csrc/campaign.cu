@@ -9,6 +9,8 @@
 //              (the write-back of Eq. 1-2 applied to a finished sum)
 // and every evaluated element goes through the output check.
 //
+//   B (long columns, short rows): batched by row panel, see panel_kernel
+//
 // Scratch (the "schedule"): three compacted lists of trial indices (A sites, B sites,
 // single-element sites) plus their counters, so that each evaluation kernel walks only its
 // own kind of trial.
@@ -230,6 +232,175 @@ __global__ void __launch_bounds__(VEC_THREADS) vector_kernel(CampaignParams p, i
     }
 }
 
+// ---------------------------------------------------------------- B-site trials, batched by row panel
+
+// When a row panel of A (R rows x K) and of C (R rows x N) fits in shared memory, B-site trials
+// are evaluated panel by panel: a CTA loads a panel once and applies a whole group of trials to
+// it, so A and C are streamed once per GROUP of trials instead of once per trial (each trial
+// alone would pull one 32-byte sector per row out of both matrices).
+// Work item = (group of up to PANEL_GROUP trials) x (contiguous chunk of panels); partial
+// statistics are kept in shared memory per trial and merged into the records with atomics.
+constexpr int PANEL_GROUP = 1024;
+constexpr int PANEL_THREADS = 1024;
+
+struct PanelShape {
+    int rows;        // R, multiple of 32
+    int a_words;     // 32-bit words per staged A row (odd: conflict-free column reads)
+    int c_words;     // 32-bit words per staged C row (odd)
+    size_t smem;
+};
+
+__host__ __device__ inline PanelShape panel_shape(int dtype, int N, int K, size_t smem_limit)
+{
+    PanelShape s;
+    s.a_words = (K * esize_of(dtype) + 3) / 4;
+    s.a_words |= 1;
+    s.c_words = N | 1;
+    const size_t fixed = (size_t)PANEL_GROUP * (5 * 4 + 4 * 4 + 8) + 1024;    // trial parameters + statistics
+    const size_t row_bytes = 4 * (size_t)(s.a_words + s.c_words);
+    long long r = smem_limit > fixed ? (long long)((smem_limit - fixed) / row_bytes) : 0;
+    r = r / 32 * 32;
+    if (r > 256) r = 256;
+    s.rows = (int)r;
+    s.smem = fixed + row_bytes * (size_t)(r > 0 ? r : 0);
+    return s;
+}
+
+__global__ void __launch_bounds__(PANEL_THREADS) panel_kernel(CampaignParams p, PanelShape ps)
+{
+    extern __shared__ __align__(16) unsigned char panel_smem[];
+    uint32_t *As = reinterpret_cast<uint32_t *>(panel_smem);
+    uint32_t *Cs = As + (size_t)ps.rows * ps.a_words;
+    uint32_t *t_id = Cs + (size_t)ps.rows * ps.c_words;
+    uint32_t *t_j = t_id + PANEL_GROUP;
+    uint32_t *t_k = t_j + PANEL_GROUP;
+    float *t_b = reinterpret_cast<float *>(t_k + PANEL_GROUP);
+    float *t_bf = t_b + PANEL_GROUP;
+    uint32_t *s_ndet = reinterpret_cast<uint32_t *>(t_bf + PANEL_GROUP);
+    uint32_t *s_first = s_ndet + PANEL_GROUP;
+    uint32_t *s_maxdev = s_first + PANEL_GROUP;
+    uint32_t *s_changed = s_maxdev + PANEL_GROUP;
+    unsigned long long *s_hash = reinterpret_cast<unsigned long long *>(
+        (reinterpret_cast<uintptr_t>(s_changed + PANEL_GROUP) + 7) & ~uintptr_t(7));
+
+    const uint32_t count = p.counters[1];
+    if (count == 0) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int es = esize_of(p.dtype);
+    const uint32_t n_groups = (count + PANEL_GROUP - 1) / PANEL_GROUP;
+    const uint32_t n_panels = ((uint32_t)p.M + ps.rows - 1) / ps.rows;
+    // enough items to occupy the grid about twice over, but never fewer than 4 panels per item
+    uint32_t n_chunks = (2 * gridDim.x + n_groups - 1) / n_groups;
+    n_chunks = max(1u, min(n_chunks, (n_panels + 3) / 4));
+    const uint32_t panels_per_chunk = (n_panels + n_chunks - 1) / n_chunks;
+
+    for (uint32_t item = blockIdx.x; item < n_groups * n_chunks; item += gridDim.x) {
+        const uint32_t g = item / n_chunks, ch = item % n_chunks;
+        const uint32_t g_beg = g * PANEL_GROUP, g_n = min((uint32_t)PANEL_GROUP, count - g_beg);
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < g_n; i += PANEL_THREADS) {
+            const uint32_t t = p.list_b[g_beg + i];
+            const mpgemmfi_site s = load_site(p.sites, t);
+            const uint32_t w_clean = load_operand(p.dtype, p.Bt, (size_t)s.col * p.K + s.k);
+            t_id[i] = t; t_j[i] = s.col; t_k[i] = s.k;
+            t_b[i] = widen_operand(p.dtype, w_clean);
+            t_bf[i] = widen_operand(p.dtype, flip_operand(p.dtype, w_clean, s.xor_mask));
+            s_ndet[i] = 0; s_first[i] = 0xFFFFFFFFu; s_maxdev[i] = 0; s_changed[i] = 0; s_hash[i] = 0ull;
+        }
+        const uint32_t p_beg = ch * panels_per_chunk, p_end = min(n_panels, p_beg + panels_per_chunk);
+        for (uint32_t pn = p_beg; pn < p_end; ++pn) {
+            const uint32_t row0 = pn * (uint32_t)ps.rows;
+            const uint32_t rows = min((uint32_t)ps.rows, (uint32_t)p.M - row0);
+            __syncthreads();       // the previous panel is no longer read; the trial tables are written
+            // stage the A and C rows of this panel (global reads in 16-byte pieces, rows padded in smem)
+            const uint32_t a_vec = (uint32_t)(p.K * es) / 16;     // K * es is a multiple of 16
+            const uint4 *Ag = reinterpret_cast<const uint4 *>(reinterpret_cast<const unsigned char *>(p.A) + (size_t)row0 * p.K * es);
+            for (uint32_t i = threadIdx.x; i < rows * a_vec; i += PANEL_THREADS) {
+                const uint32_t r = i / a_vec, v = i % a_vec;
+                const uint4 x = __ldg(Ag + (size_t)r * a_vec + v);
+                uint32_t *dst = As + (size_t)r * ps.a_words + 4 * v;
+                dst[0] = x.x; dst[1] = x.y; dst[2] = x.z; dst[3] = x.w;
+            }
+            const float *Cg = p.C + (size_t)row0 * p.N;
+            for (uint32_t i = threadIdx.x; i < rows * (uint32_t)p.N; i += PANEL_THREADS) {
+                const uint32_t r = i / (uint32_t)p.N, c = i % (uint32_t)p.N;
+                Cs[(size_t)r * ps.c_words + c] = f32_bits(Cg[i]);
+            }
+            __syncthreads();
+            // trials of the group: warp w takes trials w, w + 8, ...; lanes walk the rows
+            for (uint32_t i = warp; i < g_n; i += PANEL_THREADS / 32) {
+                const uint32_t j = t_j[i], k = t_k[i];
+                const float b = t_b[i], bf = t_bf[i];
+                uint32_t maxdev = 0, changed = 0;
+                // 128 rows per pass: every lane evaluates 4 independent rows
+                for (uint32_t rb = 0; rb < (uint32_t)ps.rows; rb += 128) {
+                    bool det[4];
+                    uint32_t lin[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t r = rb + (uint32_t)(32 * u) + (uint32_t)lane;
+                        det[u] = false;
+                        lin[u] = 0;
+                        if (r < rows) {
+                            uint32_t aw;
+                            if (es == 2) aw = reinterpret_cast<const unsigned short *>(As + (size_t)r * ps.a_words)[k];
+                            else aw = As[(size_t)r * ps.a_words + k];
+                            const float a = widen_operand(p.dtype, aw);
+                            const uint32_t c_bits = Cs[(size_t)r * ps.c_words + j];
+                            const float rep = __fsub_rn(bits_f32(c_bits), __fmul_rn(a, b));      // Eq. 1 on the finished sum
+                            const float cf = __fadd_rn(rep, __fmul_rn(a, bf));                    // Eq. 2
+                            const uint32_t fin = output_check(p.detect_mode, f32_bits(cf), det[u]);
+                            changed |= fin != c_bits ? 1u : 0u;
+                            float dev = fabsf(__fsub_rn(bits_f32(fin), bits_f32(c_bits)));
+                            if (dev != dev) dev = __uint_as_float(0x7F800000u);
+                            maxdev = max(maxdev, f32_bits(dev));
+                            lin[u] = (row0 + r) * (uint32_t)p.N + j;
+                        }
+                    }
+                    if (__any_sync(0xFFFFFFFFu, det[0] | det[1] | det[2] | det[3])) {
+                        // rare: fold the flagged elements of these rows
+                        unsigned long long h = 0ull;
+                        uint32_t first = 0xFFFFFFFFu, n = 0;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (det[u]) { h += ((unsigned long long)lin[u] + 1ull) * HASH_MUL; first = min(first, lin[u]); ++n; }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) h += __shfl_xor_sync(0xFFFFFFFFu, h, o);
+                        first = __reduce_min_sync(0xFFFFFFFFu, first);
+                        n = __reduce_add_sync(0xFFFFFFFFu, n);
+                        if (lane == 0) {
+                            s_ndet[i] += n;
+                            s_hash[i] += h;
+                            s_first[i] = min(s_first[i], first);
+                        }
+                    }
+                }
+                maxdev = __reduce_max_sync(0xFFFFFFFFu, maxdev);
+                changed = __reduce_or_sync(0xFFFFFFFFu, changed);
+                if (lane == 0) {
+                    s_maxdev[i] = max(s_maxdev[i], maxdev);
+                    s_changed[i] |= changed;
+                }
+            }
+        }
+        __syncthreads();
+        // merge this item's partial statistics into the records
+        const bool corr = (p.detect_mode & MPGEMMFI_CORRECT) &&
+                          (p.detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK) == MPGEMMFI_DETECT_BOUNDCHECK;
+        for (uint32_t i = threadIdx.x; i < g_n; i += PANEL_THREADS) {
+            mpgemmfi_trial_record *r = &p.records[t_id[i]];
+            if (s_ndet[i]) {
+                atomicAdd(&r->n_detected, s_ndet[i]);
+                atomicAdd(reinterpret_cast<unsigned long long *>(&r->idx_hash), s_hash[i]);
+                atomicMin(&r->first_detected, s_first[i]);
+            }
+            if (s_maxdev[i]) atomicMax(reinterpret_cast<uint32_t *>(&r->max_abs_dev), s_maxdev[i]);
+            const uint32_t st = (s_changed[i] ? 1u : 0u) | (s_ndet[i] ? 2u : 0u) | ((s_ndet[i] && corr) ? 4u : 0u);
+            if (st) atomicOr(&r->status, st);
+        }
+    }
+}
+
 }  // namespace
 
 size_t campaign_schedule_bytes(int n_trials)
@@ -281,7 +452,22 @@ cudaError_t launch_campaign_trials(const CampaignParams &p, int num_sms, cudaStr
     element_kernel<<<grid_e, 256, 0, stream>>>(p);
     const int grid_v = min(p.n_trials, max_ctas);
     vector_kernel<<<grid_v, VEC_THREADS, 0, stream>>>(p, 0);
-    vector_kernel<<<grid_v, VEC_THREADS, 0, stream>>>(p, 1);
+    // B-site trials: by row panel when a useful panel fits in shared memory and the columns are long
+    const PanelShape ps = panel_shape(p.dtype, p.N, p.K, 227 * 1024);
+    if (ps.rows >= 64 && p.M >= 16 * ps.rows) {
+        static bool configured[64] = {};
+        int dev = 0;
+        e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= 64 || !configured[dev]) {
+            e = cudaFuncSetAttribute(panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < 64) configured[dev] = true;
+        }
+        panel_kernel<<<num_sms, PANEL_THREADS, ps.smem, stream>>>(p, ps);
+    } else {
+        vector_kernel<<<grid_v, VEC_THREADS, 0, stream>>>(p, 1);
+    }
     return cudaGetLastError();
 }
 
