@@ -327,59 +327,70 @@ __global__ void __launch_bounds__(PANEL_THREADS) panel_kernel(CampaignParams p, 
                 Cs[(size_t)r * ps.c_words + c] = f32_bits(Cg[i]);
             }
             __syncthreads();
-            // trials of the group: warp w takes trials w, w + 8, ...; lanes walk the rows
-            for (uint32_t i = warp; i < g_n; i += PANEL_THREADS / 32) {
-                const uint32_t j = t_j[i], k = t_k[i];
-                const float b = t_b[i], bf = t_bf[i];
-                uint32_t maxdev = 0, changed = 0;
-                // 128 rows per pass: every lane evaluates 4 independent rows
-                for (uint32_t rb = 0; rb < (uint32_t)ps.rows; rb += 128) {
-                    bool det[4];
-                    uint32_t lin[4];
+            // trials of the group: warp w takes trials w, w + 32, ...; every lane evaluates 4 rows per
+            // 128-row pass. Row addresses do not depend on the trial: hoist them.
+            const bool do_bound = (p.detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK) == MPGEMMFI_DETECT_BOUNDCHECK;
+            const bool do_corr = do_bound && (p.detect_mode & MPGEMMFI_CORRECT);
+            for (uint32_t rb = 0; rb < rows; rb += 128) {
+                const uint32_t *a_row[4];
+                const uint32_t *c_row[4];
+                bool live[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t r = rb + (uint32_t)(32 * u) + (uint32_t)lane;
+                    live[u] = r < rows;
+                    const uint32_t rr = live[u] ? r : 0u;           // dead lanes read row 0 and discard
+                    a_row[u] = As + rr * (uint32_t)ps.a_words;
+                    c_row[u] = Cs + rr * (uint32_t)ps.c_words;
+                }
+                const uint32_t lin0 = (row0 + rb + (uint32_t)lane) * (uint32_t)p.N;
+                for (uint32_t i = warp; i < g_n; i += PANEL_THREADS / 32) {
+                    const uint32_t j = t_j[i], k = t_k[i];
+                    const float b = t_b[i], bf = t_bf[i];
+                    uint32_t maxdev = 0, changed = 0, det_mask = 0;
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        const uint32_t r = rb + (uint32_t)(32 * u) + (uint32_t)lane;
-                        det[u] = false;
-                        lin[u] = 0;
-                        if (r < rows) {
-                            uint32_t aw;
-                            if (es == 2) aw = reinterpret_cast<const unsigned short *>(As + (size_t)r * ps.a_words)[k];
-                            else aw = As[(size_t)r * ps.a_words + k];
-                            const float a = widen_operand(p.dtype, aw);
-                            const uint32_t c_bits = Cs[(size_t)r * ps.c_words + j];
-                            const float rep = __fsub_rn(bits_f32(c_bits), __fmul_rn(a, b));      // Eq. 1 on the finished sum
-                            const float cf = __fadd_rn(rep, __fmul_rn(a, bf));                    // Eq. 2
-                            const uint32_t fin = output_check(p.detect_mode, f32_bits(cf), det[u]);
-                            changed |= fin != c_bits ? 1u : 0u;
-                            float dev = fabsf(__fsub_rn(bits_f32(fin), bits_f32(c_bits)));
-                            if (dev != dev) dev = __uint_as_float(0x7F800000u);
-                            maxdev = max(maxdev, f32_bits(dev));
-                            lin[u] = (row0 + r) * (uint32_t)p.N + j;
+                        const uint32_t aw = es == 2 ? (uint32_t)reinterpret_cast<const unsigned short *>(a_row[u])[k] : a_row[u][k];
+                        const float a = widen_operand(p.dtype, aw);
+                        const uint32_t c_bits = c_row[u][j];
+                        const float rep = __fsub_rn(bits_f32(c_bits), __fmul_rn(a, b));      // Eq. 1 on the finished sum
+                        const float cf = __fadd_rn(rep, __fmul_rn(a, bf));                    // Eq. 2
+                        uint32_t fin = f32_bits(cf);
+                        const bool det = do_bound && live[u] && !(fabsf(cf) < 131072.0f);      // exponent field >= 0x90
+                        if (det) { det_mask |= 1u << u; if (do_corr) fin = boundcheck_clear(fin); }
+                        if (live[u]) {
+                            changed |= fin ^ c_bits;
+                            // |deviation| as raw bits: NaN patterns sort above +inf and are clamped to it below
+                            maxdev = max(maxdev, f32_bits(fabsf(__fsub_rn(bits_f32(fin), bits_f32(c_bits)))));
                         }
                     }
-                    if (__any_sync(0xFFFFFFFFu, det[0] | det[1] | det[2] | det[3])) {
+                    if (__any_sync(0xFFFFFFFFu, det_mask != 0)) {
                         // rare: fold the flagged elements of these rows
                         unsigned long long h = 0ull;
-                        uint32_t first = 0xFFFFFFFFu, n = 0;
+                        uint32_t first = 0xFFFFFFFFu;
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
-                            if (det[u]) { h += ((unsigned long long)lin[u] + 1ull) * HASH_MUL; first = min(first, lin[u]); ++n; }
+                            if (det_mask & (1u << u)) {
+                                const uint32_t lin = lin0 + (uint32_t)(32 * u) * (uint32_t)p.N + j;
+                                h += ((unsigned long long)lin + 1ull) * HASH_MUL;
+                                first = min(first, lin);
+                            }
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1) h += __shfl_xor_sync(0xFFFFFFFFu, h, o);
                         first = __reduce_min_sync(0xFFFFFFFFu, first);
-                        n = __reduce_add_sync(0xFFFFFFFFu, n);
+                        const uint32_t n = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)__popc(det_mask));
                         if (lane == 0) {
                             s_ndet[i] += n;
                             s_hash[i] += h;
                             s_first[i] = min(s_first[i], first);
                         }
                     }
-                }
-                maxdev = __reduce_max_sync(0xFFFFFFFFu, maxdev);
-                changed = __reduce_or_sync(0xFFFFFFFFu, changed);
-                if (lane == 0) {
-                    s_maxdev[i] = max(s_maxdev[i], maxdev);
-                    s_changed[i] |= changed;
+                    maxdev = min(__reduce_max_sync(0xFFFFFFFFu, maxdev), 0x7F800000u);
+                    changed = __reduce_or_sync(0xFFFFFFFFu, changed);
+                    if (lane == 0) {
+                        if (maxdev > s_maxdev[i]) s_maxdev[i] = maxdev;
+                        if (changed) s_changed[i] = 1;
+                    }
                 }
             }
         }
