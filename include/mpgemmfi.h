@@ -16,7 +16,8 @@
  *
  * Layouts: A is M x K row-major (K contiguous). B is passed K-major as Bt[N][K]
  * (row j of Bt is column j of B). C is M x N row-major FP32. FP16/BF16 elements
- * are 2 bytes, TF32 elements are 4-byte FP32 words whose low 13 bits are zero.
+ * are 2 bytes, TF32 elements are 4-byte FP32 words of which only the top 19 bits count
+ * (the low 13 bits are ignored: truncated, not rounded).
  * A and Bt must be 16-byte aligned and K * element_size a multiple of 16 bytes.
  */
 #ifndef MPGEMMFI_H
@@ -231,6 +232,34 @@ int mpgemmfi_campaign(int dtype, int M, int N, int K, const void *A, const void 
 int mpgemmfi_campaign_static(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C_clean,
                              const mpgemmfi_site *sites, int n_trials, int detect_mode,
                              mpgemmfi_trial_record *records, mpgemmfi_stream stream);
+
+/*
+ * Numeric-deviation summary of a campaign (Section V-B: the share of trials whose sum did
+ * not change, "zero difference" as in Table II, and the distribution of the non-zero
+ * differences, which the paper plots as an ECDF on a log scale).
+ *   dev_exponent_hist[e]  number of valid trials whose max_abs_dev is non-zero and has FP32
+ *                         exponent field e: bin e covers [2^(e-127), 2^(e-126)); e = 0 holds
+ *                         subnormal deviations, e = 255 infinite ones (NaN counts as infinite)
+ *   kind_*[k]             the same counts split by site kind (index = MPGEMMFI_SITE_*)
+ */
+typedef struct {
+    uint32_t n_trials;          /* records examined */
+    uint32_t n_invalid;         /* records whose site was invalid (status bit 8); not counted below */
+    uint32_t n_zero_diff;       /* status bit0 clear: every affected element kept its clean bits */
+    uint32_t n_detected;        /* status bit1 */
+    uint32_t n_corrected;       /* status bit2 */
+    uint32_t n_nonfinite;       /* max_abs_dev infinite */
+    uint32_t kind_trials[5];
+    uint32_t kind_zero_diff[5];
+    uint32_t dev_exponent_hist[256];
+} mpgemmfi_summary;
+
+/*
+ * Reduce n_trials records (device) into *summary (device, 4-byte aligned, written in full).
+ * Errors: ERR_ARG, ERR_ALIGN, ERR_CUDA.
+ */
+int mpgemmfi_campaign_summary(const mpgemmfi_trial_record *records, int n_trials, mpgemmfi_summary *summary,
+                              mpgemmfi_stream stream);
 
 /*
  * Tuning knob (no counterpart in the paper): how the GEMM kernel tiles the output.

@@ -74,6 +74,8 @@ def lib():
         L.orc_campaign.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, vp]
         L.orc_sample.restype = C.c_int
         L.orc_sample.argtypes = [C.c_int] * 4 + [vp, vp, vp, C.c_int, vp, vp, C.c_int, vp, vp]
+        L.orc_summary.restype = None
+        L.orc_summary.argtypes = [vp, C.c_int, vp]
         L.orc_absprod.restype = C.c_int
         L.orc_absprod.argtypes = [C.c_int] * 4 + [vp, vp, vp]
     return _lib
@@ -191,6 +193,15 @@ def sample(dtype, A, Bt, si, sj, sites=None):
     rc = lib().orc_sample(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(s), len(s), _ptr(si), _ptr(sj), len(si), _ptr(out), _ptr(ap))
     assert rc == 0
     return out, ap
+
+
+def summary(records):
+    """Deviation summary of trial records: 272 uint32 words (6 counts, 5 + 5 per-kind counts, 256 histogram bins)."""
+    rec = np.ascontiguousarray(records)
+    assert rec.dtype.itemsize == 48
+    out = np.zeros(272, dtype=np.uint32)
+    lib().orc_summary(_ptr(rec), len(rec), _ptr(out))
+    return out
 
 
 def absprod(dtype, A, Bt):

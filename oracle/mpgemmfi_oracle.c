@@ -546,6 +546,34 @@ int orc_absprod(int dtype, int M, int N, int K, const void *A, const void *Bt, d
     return 0;
 }
 
+/* ------------------------------------------------------------------ deviation summary */
+
+/*
+ * Section V-B: share of trials with zero difference (Table II) and the spread of the
+ * non-zero differences, binned by the FP32 exponent field of the trial's largest
+ * |final - clean|. out[0..5]: trials, invalid, zero-diff, detected, corrected, non-finite;
+ * out[6..10]: trials per site kind; out[11..15]: zero-diff trials per kind;
+ * out[16..271]: histogram over the exponent field (NaN counted with the infinities).
+ */
+void orc_summary(const orc_trial_record *rec, int n, uint32_t *out)
+{
+    memset(out, 0, sizeof(uint32_t) * 272);
+    out[0] = (uint32_t)n;
+    for (int t = 0; t < n; ++t) {
+        const orc_trial_record *r = &rec[t];
+        if (r->status & (1u << 8)) { out[1]++; continue; }
+        int zero = (r->status & 1u) == 0;
+        if (zero) out[2]++;
+        if (r->status & 2u) out[3]++;
+        if (r->status & 4u) out[4]++;
+        if (r->kind < 5) { out[6 + r->kind]++; if (zero) out[11 + r->kind]++; }
+        float d = r->max_abs_dev;
+        if (d != d || isinf(d)) { out[5]++; out[16 + 255]++; continue; }
+        if (d == 0.0f) continue;
+        out[16 + ((f2u(d) >> 23) & 0xFFu)]++;
+    }
+}
+
 int orc_num_threads(void)
 {
 #ifdef _OPENMP

@@ -11,10 +11,10 @@ from .binding import (  # noqa: F401
     DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP, CORRECT,
     STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT, MAX_FAULTS, HEADER_WORDS, STATIC_MAX_TRIALS,
     TILES_AUTO, TILES_SINGLE, TILES_PAIR, mpgemmfi_set_tile_policy,
-    SITE_DTYPE, SITE_LOG_DTYPE, RECORD_DTYPE,
+    SITE_DTYPE, SITE_LOG_DTYPE, RECORD_DTYPE, SUMMARY_DTYPE,
     MpgemmfiError, library_path, load_library, exported_symbols,
     mpgemmfi_gemm, mpgemmfi_campaign, mpgemmfi_campaign_static, mpgemmfi_kstep, mpgemmfi_flags_bytes,
     mpgemmfi_flags_bitmap_offset, mpgemmfi_campaign_workspace_bytes,
     mpgemmfi_validate_sites, mpgemmfi_strerror, mpgemmfi_last_cuda_error, mpgemmfi_version,
-    gemm, campaign, split_flags,
+    gemm, campaign, split_flags, mpgemmfi_campaign_summary, campaign_summary,
 )

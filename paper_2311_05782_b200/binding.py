@@ -29,6 +29,10 @@ RECORD_DTYPE = np.dtype([("status", "<u4"), ("kind", "<u4"), ("primary_index", "
                          ("after_bits", "<u4"), ("final_bits", "<u4"), ("n_affected", "<u4"), ("n_detected", "<u4"),
                          ("idx_hash", "<u8"), ("first_detected", "<u4"), ("max_abs_dev", "<f4")])
 
+SUMMARY_DTYPE = np.dtype([("n_trials", "<u4"), ("n_invalid", "<u4"), ("n_zero_diff", "<u4"), ("n_detected", "<u4"),
+                          ("n_corrected", "<u4"), ("n_nonfinite", "<u4"), ("kind_trials", "<u4", (5,)),
+                          ("kind_zero_diff", "<u4", (5,)), ("dev_exponent_hist", "<u4", (256,))])
+
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libmpgemmfi.so")
 _lib = None
@@ -37,7 +41,7 @@ _SYMBOLS = [
     "mpgemmfi_gemm", "mpgemmfi_campaign", "mpgemmfi_kstep", "mpgemmfi_flags_bytes",
     "mpgemmfi_flags_bitmap_offset", "mpgemmfi_campaign_workspace_bytes", "mpgemmfi_validate_sites",
     "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version", "mpgemmfi_campaign_static",
-    "mpgemmfi_set_tile_policy",
+    "mpgemmfi_set_tile_policy", "mpgemmfi_campaign_summary",
 ]
 
 
@@ -74,6 +78,8 @@ def load_library():
     L.mpgemmfi_campaign.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp, sz, vp]
     L.mpgemmfi_campaign_static.restype = i
     L.mpgemmfi_campaign_static.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp]
+    L.mpgemmfi_campaign_summary.restype = i
+    L.mpgemmfi_campaign_summary.argtypes = [vp, i, vp, vp]
     L.mpgemmfi_set_tile_policy.restype = i
     L.mpgemmfi_set_tile_policy.argtypes = [i]
     L.mpgemmfi_kstep.restype = i
@@ -113,6 +119,22 @@ def mpgemmfi_campaign_static(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, de
     for callers that are not allowed to allocate device memory. At most STATIC_MAX_TRIALS trials per call."""
     return load_library().mpgemmfi_campaign_static(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mode,
                                                    records, stream)
+
+
+def mpgemmfi_campaign_summary(records, n_trials, summary, stream):
+    """Raw call: reduce n_trials device records into a device mpgemmfi_summary (SUMMARY_DTYPE.itemsize bytes)."""
+    return load_library().mpgemmfi_campaign_summary(records, n_trials, summary, stream)
+
+
+def campaign_summary(records, stream=None):
+    """Deviation summary of a records tensor ([n, 12] int32 on CUDA); returns a host numpy record of SUMMARY_DTYPE."""
+    torch = _torch()
+    out = torch.empty(SUMMARY_DTYPE.itemsize // 4, dtype=torch.int32, device=records.device)
+    stream_h = (torch.cuda.current_stream(records.device) if stream is None else stream).cuda_stream
+    rc = mpgemmfi_campaign_summary(records.data_ptr() if records.shape[0] else None, records.shape[0], out.data_ptr(), stream_h)
+    if rc != 0:
+        raise MpgemmfiError(rc, "mpgemmfi_campaign_summary")
+    return out.cpu().numpy().view(np.uint32).view(SUMMARY_DTYPE)[0]
 
 
 def mpgemmfi_set_tile_policy(policy):

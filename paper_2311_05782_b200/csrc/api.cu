@@ -233,6 +233,18 @@ int mpgemmfi_campaign_static(int dtype, int M, int N, int K, const void *A, cons
     return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
 }
 
+int mpgemmfi_campaign_summary(const mpgemmfi_trial_record *records, int n_trials, mpgemmfi_summary *summary,
+                              mpgemmfi_stream stream)
+{
+    if (n_trials < 0 || (n_trials > 0 && !records) || !summary) return MPGEMMFI_ERR_ARG;
+    if (((uintptr_t)records & 7) || ((uintptr_t)summary & 3)) return MPGEMMFI_ERR_ALIGN;
+    DeviceInfo di;
+    const int rc = device_info(di);
+    if (rc) return rc;
+    const cudaError_t e = mpg::launch_campaign_summary(records, n_trials, summary, di.num_sms, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
+}
+
 int mpgemmfi_set_tile_policy(int policy)
 {
     if (policy != MPGEMMFI_TILES_AUTO && policy != MPGEMMFI_TILES_SINGLE && policy != MPGEMMFI_TILES_PAIR)

@@ -412,7 +412,58 @@ __global__ void __launch_bounds__(PANEL_THREADS) panel_kernel(CampaignParams p, 
     }
 }
 
+// ---------------------------------------------------------------- deviation summary
+
+__global__ void __launch_bounds__(256) summary_kernel(const mpgemmfi_trial_record *records, int n, mpgemmfi_summary *out)
+{
+    __shared__ uint32_t hist[256];
+    __shared__ uint32_t cnt[16];      // 0 invalid, 1 zero-diff, 2 detected, 3 corrected, 4 non-finite, 5.. unused
+    __shared__ uint32_t kind_trials[5], kind_zero[5];
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+    if (threadIdx.x < 16) cnt[threadIdx.x] = 0;
+    if (threadIdx.x < 5) { kind_trials[threadIdx.x] = 0; kind_zero[threadIdx.x] = 0; }
+    __syncthreads();
+    for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < n; t += gridDim.x * blockDim.x) {
+        const mpgemmfi_trial_record r = records[t];
+        if (r.status & (1u << 8)) { atomicAdd(&cnt[0], 1u); continue; }
+        const bool zero = (r.status & 1u) == 0;
+        if (zero) atomicAdd(&cnt[1], 1u);
+        if (r.status & 2u) atomicAdd(&cnt[2], 1u);
+        if (r.status & 4u) atomicAdd(&cnt[3], 1u);
+        if (r.kind < 5) { atomicAdd(&kind_trials[r.kind], 1u); if (zero) atomicAdd(&kind_zero[r.kind], 1u); }
+        uint32_t d = f32_bits(r.max_abs_dev) & 0x7FFFFFFFu;
+        if (d > 0x7F800000u) d = 0x7F800000u;                      // NaN counts as infinite
+        if (d == 0x7F800000u) atomicAdd(&cnt[4], 1u);
+        if (d != 0) atomicAdd(&hist[d >> 23], 1u);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 256; i += blockDim.x)
+        if (hist[i]) atomicAdd(&out->dev_exponent_hist[i], hist[i]);
+    if (threadIdx.x == 0) {
+        if (blockIdx.x == 0) out->n_trials = (uint32_t)n;
+        if (cnt[0]) atomicAdd(&out->n_invalid, cnt[0]);
+        if (cnt[1]) atomicAdd(&out->n_zero_diff, cnt[1]);
+        if (cnt[2]) atomicAdd(&out->n_detected, cnt[2]);
+        if (cnt[3]) atomicAdd(&out->n_corrected, cnt[3]);
+        if (cnt[4]) atomicAdd(&out->n_nonfinite, cnt[4]);
+        for (int k = 0; k < 5; ++k) {
+            if (kind_trials[k]) atomicAdd(&out->kind_trials[k], kind_trials[k]);
+            if (kind_zero[k]) atomicAdd(&out->kind_zero_diff[k], kind_zero[k]);
+        }
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_campaign_summary(const mpgemmfi_trial_record *records, int n_trials, mpgemmfi_summary *out,
+                                    int num_sms, cudaStream_t stream)
+{
+    cudaError_t e = cudaMemsetAsync(out, 0, sizeof(mpgemmfi_summary), stream);
+    if (e != cudaSuccess) return e;
+    const int grid = max(1, min((n_trials + 255) / 256, 4 * num_sms));
+    summary_kernel<<<grid, 256, 0, stream>>>(records, n_trials, out);
+    return cudaGetLastError();
+}
 
 size_t campaign_schedule_bytes(int n_trials)
 {

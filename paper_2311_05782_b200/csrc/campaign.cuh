@@ -40,4 +40,8 @@ cudaError_t campaign_static_schedule(void **ptr, size_t *bytes);
 // schedule + evaluate every trial; the clean product must already be queued on `stream`
 cudaError_t launch_campaign_trials(const CampaignParams &p, int num_sms, cudaStream_t stream);
 
+// zero *out and reduce the records into it
+cudaError_t launch_campaign_summary(const mpgemmfi_trial_record *records, int n_trials, mpgemmfi_summary *out,
+                                    int num_sms, cudaStream_t stream);
+
 }  // namespace mpg

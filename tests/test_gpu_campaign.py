@@ -80,3 +80,32 @@ def test_campaign_edge_cases():
     assert mpg.mpgemmfi_campaign(0, 128, 128, 64, a.data_ptr(), b.data_ptr(), c.data_ptr(), st.data_ptr(), 3, 1,
                                  r.data_ptr(), ws.data_ptr() + 8, 2048, cs) == -5
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("name,shape,trials", [("c5", (2048, 64, 576), 400), ("c2", (256, 384, 256), 200), ("c4", (256, 256, 256), 150)])
+def test_campaign_summary_matches_oracle_reduction(name, shape, trials):
+    """The device reduction of the records (zero-difference share, deviation histogram) against the oracle's."""
+    M, N, K = shape
+    w = synth.make_workload(name, M, N, K, trials=trials)
+    sites = w.sites.copy()
+    sites["kind"][3] = 9                                        # an invalid site must be left out of the counts
+    view = np.int32 if w.dtype == orc.TF32 else np.int16
+    a = torch.from_numpy(w.A.view(view)).cuda(); b = torch.from_numpy(w.Bt.view(view)).cuda()
+    Cc, rec = mpg.campaign(w.dtype, a, b, sites, w.detect_mode)
+    got = mpg.campaign_summary(rec)
+    host = rec.cpu().numpy().view(np.uint32).reshape(-1).view(mpg.RECORD_DTYPE)
+    want = orc.summary(host)                                    # same records: the reduction itself is bit-exact
+    flat = np.concatenate([[got["n_trials"], got["n_invalid"], got["n_zero_diff"], got["n_detected"], got["n_corrected"],
+                            got["n_nonfinite"]], got["kind_trials"], got["kind_zero_diff"], got["dev_exponent_hist"]])
+    assert np.array_equal(flat.astype(np.uint32), want)
+    assert got["n_invalid"] == 1 and got["n_trials"] == trials
+    # and end to end against the oracle's own campaign: same zero-difference share for the exactly reproducible kinds
+    Cclean, *_ = orc.gemm(w.dtype, w.A, w.Bt)
+    ro = orc.campaign(w.dtype, w.A, w.Bt, Cclean, sites, w.detect_mode)
+    so = orc.summary(ro)
+    for kind in (orc.KIND_ACC, orc.KIND_TERM):
+        assert got["kind_trials"][kind] == so[6 + kind] and got["kind_zero_diff"][kind] == so[11 + kind]
+    assert np.array_equal(got["kind_trials"], so[6:11])
+    # empty input
+    empty = mpg.campaign_summary(rec[:0])
+    assert empty["n_trials"] == 0 and empty["dev_exponent_hist"].sum() == 0

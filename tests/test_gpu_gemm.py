@@ -220,3 +220,19 @@ def test_maximum_site_count():
     a, b = to_dev(w.A, w.dtype), to_dev(w.Bt, w.dtype)
     with pytest.raises(mpg.MpgemmfiError):
         mpg.gemm(w.dtype, a, b, np.zeros(mpg.MAX_FAULTS + 1, dtype=orc.SITE), 0)
+
+
+def test_tf32_low_mantissa_bits_are_ignored(tile_policy):
+    """FP32 words whose low 13 bits are not zero: the tensor core must see only the top 19 bits (the oracle masks them)."""
+    rng = np.random.default_rng(23)
+    M, N, K = 256, 256, 96
+    a = rng.standard_normal((M, K)).astype(np.float32).view(np.uint32)
+    b = rng.standard_normal((N, K)).astype(np.float32).view(np.uint32)
+    assert (a & 0x1FFF).any()
+    Cg, *_ = run_gpu_gemm(orc.TF32, a, b, None, orc.T_NONE)
+    Co, *_ = orc.gemm(orc.TF32, a, b)                       # widens with the low 13 bits dropped
+    ok = close(Cg, Co, TOL * orc.absprod(orc.TF32, a, b))
+    # a tensor core that rounded instead of truncating would be off by up to 2^-11 relative per operand: still inside
+    # the 1e-3 tolerance, so also demand the tight bound that only truncation meets
+    tight = np.abs(Cg - Co) <= 2e-6 * orc.absprod(orc.TF32, a, b)
+    assert ok.all() and tight.mean() > 0.999

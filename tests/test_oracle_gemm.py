@@ -292,3 +292,37 @@ def test_site_generators_follow_the_recipes():
     assert (a.view(np.float16) >= 0).all() and (a == 0).mean() > 0.3          # ReLU: about half zeros
     a, _ = synth.make_operands("c4", 64, 8, 32)
     assert a.dtype == np.uint32 and not (a & 0x1FFF).any()
+
+
+def test_summary_bruteforce_and_bin_edges():
+    """Deviation summary: counts and exponent bins against a Python loop; bin e covers [2^(e-127), 2^(e-126))."""
+    import math
+    w = synth.make_workload("c5", 48, 40, 128, trials=300)
+    Cc, *_ = orc.gemm(w.dtype, w.A, w.Bt)
+    sites = w.sites.copy()
+    sites["row"][7] = 10 ** 6                                   # one invalid site
+    rec = orc.campaign(w.dtype, w.A, w.Bt, Cc, sites, w.detect_mode)
+    out = orc.summary(rec)
+    want = np.zeros(272, dtype=np.uint32)
+    want[0] = len(rec)
+    for r in rec:
+        if r["status"] & 0x100:
+            want[1] += 1; continue
+        zero = not (r["status"] & 1)
+        want[2] += zero; want[3] += bool(r["status"] & 2); want[4] += bool(r["status"] & 4)
+        want[6 + r["kind"]] += 1; want[11 + r["kind"]] += zero
+        d = float(r["max_abs_dev"])
+        if math.isinf(d) or math.isnan(d):
+            want[5] += 1; want[16 + 255] += 1
+        elif d > 0:
+            e = math.floor(math.log2(d)) + 127 if d >= 2.0 ** -126 else 0
+            want[16 + e] += 1
+    assert np.array_equal(out, want)
+    assert want[1] == 1 and want[2] > 0 and want[16:].sum() > 100
+    assert out[6:11].sum() == out[0] - out[1] and out[2] == out[11:16].sum()
+    # hand-made records pin the bin edges
+    r = np.zeros(6, dtype=orc.RECORD)
+    r["status"] = 1
+    r["max_abs_dev"] = [1.0, 1.9999999, 2.0, 2.0 ** -126, 2.0 ** -127, np.inf]
+    h = orc.summary(r)[16:]
+    assert h[127] == 2 and h[128] == 1 and h[1] == 1 and h[0] == 1 and h[255] == 1 and h.sum() == 6
