@@ -93,7 +93,15 @@ enum {
     MPGEMMFI_DETECT_RANGE_MAX = 2,
     MPGEMMFI_DETECT_RANGE_FLIP = 3,
     MPGEMMFI_DETECT_TECHNIQUE_MASK = 3,
-    MPGEMMFI_CORRECT = 16
+    MPGEMMFI_CORRECT = 16,
+    /*
+     * Campaigns only (mpgemmfi_gemm rejects it): a TERM trial's write-back takes place at the end
+     * of the group of 16 (FP16, BF16) or 8 (TF32) terms that contains the term, i.e. on the
+     * running sum as one HMMA instruction of the paper's platform leaves it (Section III-C:
+     * shapes 16x8x16 and 16x8x8; Section IV-A: 16 or 8 terms per destination register), instead
+     * of at the next mpgemmfi_kstep boundary.
+     */
+    MPGEMMFI_TERM_HMMA_STEP = 32
 };
 
 enum {

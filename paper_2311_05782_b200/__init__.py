@@ -8,7 +8,7 @@ fails loudly when the CUDA library is missing.
 from .binding import (  # noqa: F401
     FP16, BF16, TF32,
     SITE_A, SITE_B, SITE_ACC, SITE_OUT, SITE_TERM,
-    DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP, CORRECT,
+    DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP, CORRECT, TERM_HMMA_STEP,
     STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT, MAX_FAULTS, HEADER_WORDS, STATIC_MAX_TRIALS,
     TILES_AUTO, TILES_SINGLE, TILES_PAIR, mpgemmfi_set_tile_policy,
     SITE_DTYPE, SITE_LOG_DTYPE, RECORD_DTYPE, SUMMARY_DTYPE,

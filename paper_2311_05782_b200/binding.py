@@ -16,6 +16,7 @@ FP16, BF16, TF32 = 0, 1, 2
 SITE_A, SITE_B, SITE_ACC, SITE_OUT, SITE_TERM = 0, 1, 2, 3, 4
 DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP = 0, 1, 2, 3
 CORRECT = 16
+TERM_HMMA_STEP = 32
 STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT = 1, 2
 MAX_FAULTS = 4096
 STATIC_MAX_TRIALS = 65536

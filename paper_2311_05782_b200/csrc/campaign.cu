@@ -113,7 +113,9 @@ __global__ void __launch_bounds__(256) element_kernel(CampaignParams p)
     const uint32_t warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t n_warps = (gridDim.x * blockDim.x) >> 5;
     const uint32_t count = p.counters[2];
-    const uint32_t ks = (uint32_t)kstep_of(p.dtype);
+    // granularity of a TERM write-back: the GEMM kernel's k-step, or one HMMA's worth of terms
+    const uint32_t ks = (p.detect_mode & MPGEMMFI_TERM_HMMA_STEP) ? (p.dtype == MPGEMMFI_TF32 ? 8u : 16u)
+                                                                  : (uint32_t)kstep_of(p.dtype);
     for (uint32_t w = warp_global; w < count; w += n_warps) {
         const uint32_t t = p.list_e[w];
         const mpgemmfi_site s = load_site(p.sites, t);

@@ -109,3 +109,32 @@ def test_campaign_summary_matches_oracle_reduction(name, shape, trials):
     # empty input
     empty = mpg.campaign_summary(rec[:0])
     assert empty["n_trials"] == 0 and empty["dev_exponent_hist"].sum() == 0
+
+
+@pytest.mark.parametrize("dtype,name", [(orc.FP16, "c1"), (orc.BF16, "c2"), (orc.TF32, "c4")])
+@pytest.mark.parametrize("nbits", [1, 2, 4])
+def test_campaign_term_trials_at_hmma_granularity(dtype, name, nbits):
+    """The paper's own trial (Section IV-A): uniform element, uniform term, 1/2/4 flipped bits of the product,
+    written back into the sum that one HMMA leaves (16 terms for FP16/BF16, 8 for TF32)."""
+    M, N, K = 192, 160, 208
+    A, Bt = synth.make_operands(name, M, N, K)
+    sites = synth.make_sites("term", dtype, M, N, K, 300, 99 + nbits, nbits=nbits)
+    step = 8 if dtype == orc.TF32 else 16
+    for tech in (orc.T_NONE, orc.T_BOUND | orc.CORRECT, orc.T_RMAX | orc.CORRECT, orc.T_RFLIP | orc.CORRECT):
+        _, rg = run_gpu_campaign(dtype, A, Bt, sites, tech | mpg.TERM_HMMA_STEP)
+        Cclean, *_ = orc.gemm(dtype, A, Bt)
+        ro = orc.campaign(dtype, A, Bt, Cclean, sites, tech, kstep=step)
+        raw = orc.campaign(dtype, A, Bt, Cclean, sites, tech & ~orc.CORRECT, kstep=step)
+        nan_made = np.isnan(raw["final_bits"].view(np.float32))
+        for f in rg.dtype.names:
+            same = rg[f] == ro[f]
+            if f in ("final_bits", "max_abs_dev"):
+                same |= nan_made                                 # NaN payloads are not part of parity
+            assert same.all(), (f, np.nonzero(~same)[0][:5])
+        # the granularity matters: with the GEMM's k-step some of these trials end differently
+        _, rk = run_gpu_campaign(dtype, A, Bt, sites, tech)
+        assert np.array_equal(rk["before_bits"], rg["before_bits"])
+    # the flag is a campaign-only option
+    a, b = to_dev(A, dtype), to_dev(Bt, dtype)
+    with pytest.raises(mpg.MpgemmfiError):
+        mpg.gemm(dtype, a, b, sites[:1], mpg.TERM_HMMA_STEP)
