@@ -138,6 +138,9 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
     p.detect_mode = detect_mode; p.n_faults = n_faults;
     p.tiles_m = (M + tm - 1) / tm; p.tiles_n = (N + bn - 1) / bn;
     p.num_tiles = p.tiles_m * p.tiles_n;
+    // the walkers' tiles of one round should cover about as many bytes of A as of Bt
+    p.group_m = pair ? 8 : (bn == 256 ? 16 : (bn == 128 ? 12 : 8));
+    if (p.group_m > p.tiles_m) p.group_m = p.tiles_m;
     const int ks = mpg::kstep_of(dtype);
     p.num_kt = (K + ks - 1) / ks;
     p.wpr = (N + 31) / 32;

@@ -264,24 +264,45 @@ __device__ void apply_out_sites(const TileCtx &c, uint32_t row, uint32_t c0, uin
     }
 }
 
+// Tile order. Tiles are numbered so that the tiles in flight at one time (consecutive numbers, dealt
+// out round-robin to the walkers) form a block of group_m tile rows by several tile columns rather
+// than one long column strip: each round then touches few row panels of A and few column panels of
+// Bt, which keeps them in L2 when A or Bt alone is larger than L2.
+// Within a band of group_m tile rows the number runs down the rows first, then across the columns.
+__device__ __forceinline__ void tile_coords(const GemmParams &p, uint32_t t, uint32_t &tm, uint32_t &tn)
+{
+    const uint32_t band_tiles = (uint32_t)p.group_m * (uint32_t)p.tiles_n;
+    const uint32_t band = t / band_tiles, within = t % band_tiles;
+    const uint32_t rows = min((uint32_t)p.group_m, (uint32_t)p.tiles_m - band * (uint32_t)p.group_m);
+    tm = band * (uint32_t)p.group_m + within % rows;
+    tn = within / rows;
+}
+
+__device__ __forceinline__ uint32_t tile_number(const GemmParams &p, uint32_t tm, uint32_t tn)
+{
+    const uint32_t band = tm / (uint32_t)p.group_m;
+    const uint32_t rows = min((uint32_t)p.group_m, (uint32_t)p.tiles_m - band * (uint32_t)p.group_m);
+    return band * (uint32_t)p.group_m * (uint32_t)p.tiles_n + tn * rows + (tm - band * (uint32_t)p.group_m);
+}
+
 // Does a site touch a tile walked by tile-walker `gid` of `groups` (a CTA, or a CTA pair)?
-// Tiles are TM x BN and are dealt out round-robin: tile index = tn * tiles_m + tm.
+// Tiles are TM x BN and are dealt out round-robin by tile number.
 template <int TM, int BN>
 __device__ bool site_touches_group(const mpgemmfi_site &s, const GemmParams &p, uint32_t gid, uint32_t groups)
 {
     if (s.kind == MPGEMMFI_SITE_A) {
         const uint32_t tm = s.row / TM;
         for (uint32_t tn = 0; tn < (uint32_t)p.tiles_n; ++tn)
-            if ((tn * p.tiles_m + tm) % groups == gid) return true;
+            if (tile_number(p, tm, tn) % groups == gid) return true;
         return false;
     }
     if (s.kind == MPGEMMFI_SITE_B) {
         const uint32_t tn = s.col / BN;
         for (uint32_t tm = 0; tm < (uint32_t)p.tiles_m; ++tm)
-            if ((tn * p.tiles_m + tm) % groups == gid) return true;
+            if (tile_number(p, tm, tn) % groups == gid) return true;
         return false;
     }
-    return ((s.col / BN) * p.tiles_m + s.row / TM) % groups == gid;
+    return tile_number(p, s.row / TM, s.col / BN) % groups == gid;
 }
 
 // Slice of the site table that one warp examines when the CTA builds its list.
@@ -427,9 +448,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     TileCtx tc;
     tc.p = &p; tc.ctl = ctl; tc.bn = BN; tc.tile_rows = TM; tc.b_rows = C::B_ROWS;
     auto set_tile = [&](uint32_t t) {
-        tc.tile_m0 = (t % p.tiles_m) * TM;
+        uint32_t tm, tn;
+        tile_coords(p, t, tm, tn);
+        tc.tile_m0 = tm * TM;
         tc.m0 = tc.tile_m0 + rank * BM;
-        tc.n0 = (t / p.tiles_m) * BN;
+        tc.n0 = tn * BN;
         tc.b0 = tc.n0 + rank * C::B_ROWS;
     };
     // barriers of the leader CTA that this CTA's warps arrive on

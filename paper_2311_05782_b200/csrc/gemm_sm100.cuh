@@ -13,6 +13,7 @@ struct GemmParams {
     int dtype, M, N, K;
     int detect_mode, n_faults;
     int tiles_m, tiles_n, num_tiles, num_kt;
+    int group_m;    // tile rows per band of the tile order (>= 1)
     int wpr;        // bitmap words per row = ceil(N / 32)
     int c_vec_ok;   // C is 16-byte aligned with a 16-byte row pitch: the epilogue may use 16-byte stores
     const void *A;
