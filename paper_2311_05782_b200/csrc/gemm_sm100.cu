@@ -654,7 +654,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                         if (det) fw |= 1u << j;
                         if (do_corr && det) v[j] = boundcheck_clear(v[j]);
                     }
-                    // columns past N hold zeros (zero-filled operand rows) and never flag
+                    // columns past N are not part of C (their zero-filled Bt rows still give NaN against an
+                    // Inf or NaN in A): their flag bits stay 0
+                    if (c0 + 32 > (uint32_t)p.N) fw &= c0 < (uint32_t)p.N ? (1u << ((uint32_t)p.N - c0)) - 1u : 0u;
                 }
                 if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 1);
                 flagw[i] = fw;

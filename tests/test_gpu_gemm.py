@@ -236,3 +236,36 @@ def test_tf32_low_mantissa_bits_are_ignored(tile_policy):
     # the 1e-3 tolerance, so also demand the tight bound that only truncation meets
     tight = np.abs(Cg - Co) <= 2e-6 * orc.absprod(orc.TF32, a, b)
     assert ok.all() and tight.mean() > 0.999
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_degenerate_shapes_and_special_values(dtype, tile_policy):
+    """One row, one column, the shortest legal K; zeros, subnormals, huge values, Inf and NaN among the operands."""
+    kmin = 4 if dtype == orc.TF32 else 8                      # K * element size must be a multiple of 16 bytes
+    for (M, N, K) in [(1, 1, kmin), (1, 37, kmin), (129, 1, 3 * kmin), (5, 7, 72)]:
+        A, Bt = rand_operands(dtype, M, N, K, 40 + M + N)
+        check_gemm_against_oracle(dtype, A, Bt, site(orc.KIND_OUT, M - 1, N - 1, 0, 1 << 30), orc.T_BOUND | orc.CORRECT)
+    M, N, K = 130, 70, 80
+    rng = np.random.default_rng(41)
+    a = rng.standard_normal((M, K)).astype(np.float32)
+    b = rng.standard_normal((N, K)).astype(np.float32)
+    a[rng.random((M, K)) < 0.3] = 0.0                         # sparse rows, as after a ReLU
+    a[3, 5] = np.inf; a[7, 9] = -np.inf; a[11, 2] = np.nan
+    a[20, :] = 0.0                                            # a whole zero row: exact zeros out
+    a[30, 1] = 3e4 if dtype == orc.FP16 else 1e30             # products far above the BoundCheck threshold
+    b[4, 5] = 1e-7 if dtype == orc.FP16 else 1e-39            # FP16 / FP32 subnormal after rounding
+    b[6, :] = 0.0
+    b[8, 9] = np.inf                                          # meets -inf * ... and 0 * inf -> NaN
+    A, Bt = synth.round_to_storage(a, dtype), synth.round_to_storage(b, dtype)
+    for mode in (orc.T_BOUND, orc.T_BOUND | orc.CORRECT, orc.T_NONE):
+        Cg, hdr, log, bm = run_gpu_gemm(dtype, A, Bt, None, mode)
+        Co, hdr_o, _, bm_o = orc.gemm(dtype, A, Bt, None, mode)
+        tol = TOL * orc.absprod(dtype, A, Bt)                 # infinite or NaN where a special value takes part
+        assert close(Cg, Co, tol).all()
+        special = ~np.isfinite(tol)
+        assert np.array_equal(np.isnan(Cg[special]) | np.isinf(Cg[special]) | (mode == (orc.T_BOUND | orc.CORRECT)),
+                              np.isnan(Co[special]) | np.isinf(Co[special]) | (mode == (orc.T_BOUND | orc.CORRECT)))
+        d = np.argwhere(bm != bm_o)
+        info = [(int(i), int(w), hex(int(bm[i, w])), hex(int(bm_o[i, w])), Cg[i, 32 * w:32 * w + 32][:12].tolist(), Co[i, 32 * w:32 * w + 32][:12].tolist()) for i, w in d[:3]]
+        assert np.array_equal(bm, bm_o) and hdr[1] == hdr_o[1], info      # NaN, Inf and huge values are flagged alike
+        assert (Cg[20][np.isfinite(tol[20])] == 0).all() and (Cg[:, 6][np.isfinite(tol[:, 6])] == 0).all()
