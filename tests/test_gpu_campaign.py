@@ -138,3 +138,43 @@ def test_campaign_term_trials_at_hmma_granularity(dtype, name, nbits):
     a, b = to_dev(A, dtype), to_dev(Bt, dtype)
     with pytest.raises(mpg.MpgemmfiError):
         mpg.gemm(dtype, a, b, sites[:1], mpg.TERM_HMMA_STEP)
+
+
+def test_campaign_single_element_trials_with_special_values():
+    """ACC / TERM / OUT trials on operands that hold zeros, Inf, NaN and huge values: both sides walk the same
+    sums in the same order, so the records agree bit for bit (NaN payloads aside)."""
+    M, N, K = 96, 80, 200
+    rng = np.random.default_rng(51)
+    a = rng.standard_normal((M, K)).astype(np.float32); b = rng.standard_normal((N, K)).astype(np.float32)
+    a[rng.random((M, K)) < 0.4] = 0.0
+    a[5, 17] = np.inf; a[9, 3] = np.nan; a[20, 100] = 1e30; b[7, 17] = -np.inf; b[30, 100] = 1e30; b[11, :] = 0.0
+    A, Bt = synth.round_to_storage(a, orc.BF16), synth.round_to_storage(b, orc.BF16)
+    parts = []
+    for mix, seed in (("acc", 1), ("term", 2), ("out", 3)):
+        s = synth.make_sites(mix, orc.BF16, M, N, K, 200, seed, nbits=2)
+        parts.append(s)
+    sites = np.concatenate(parts)
+    sites["row"][:12] = [5, 5, 9, 9, 20, 20, 5, 9, 20, 5, 9, 20]          # make sure the special rows / columns are hit
+    sites["col"][:12] = [7, 30, 7, 11, 30, 11, 0, 1, 2, 11, 30, 7]
+    for mode in (orc.T_BOUND | orc.CORRECT, orc.T_RMAX | orc.CORRECT, orc.T_NONE):
+        Cg, rg = run_gpu_campaign(orc.BF16, A, Bt, sites, mode)
+        Cclean, *_ = orc.gemm(orc.BF16, A, Bt)
+        elem = sites["kind"] != orc.KIND_OUT
+        ro = orc.campaign(orc.BF16, A, Bt, Cclean, sites, mode)
+        raw = orc.campaign(orc.BF16, A, Bt, Cclean, sites, mode & ~orc.CORRECT)
+        nan_made = np.isnan(raw["final_bits"].view(np.float32)) | np.isnan(raw["before_bits"].view(np.float32))
+        for f in rg.dtype.names:
+            same = (rg[f] == ro[f])
+            if f in ("final_bits", "max_abs_dev", "before_bits", "after_bits"):
+                same |= nan_made
+            if f == "max_abs_dev":
+                same |= np.isnan(rg[f]) & np.isnan(ro[f])
+            if f == "status":
+                # "changed" compares bit patterns: between two NaNs it depends on payloads, which are not part of parity
+                clean_nan = np.isnan(Cclean.reshape(-1)[np.minimum(ro["primary_index"], M * N - 1)])
+                same |= ((rg[f] ^ ro[f]) == 1) & (nan_made | clean_nan)
+            assert same[elem].all(), (mode, f, np.nonzero(~same & elem)[0][:5])
+        out = ~elem
+        assert np.array_equal(rg["after_bits"][out], rg["before_bits"][out] ^ sites["xor_mask"][out])
+        assert np.array_equal(rg["n_detected"][out], np.array([orc.boundcheck_detect(int(x)) if (mode & 3) == 1 else 0
+                                                               for x in rg["after_bits"][out]]))
