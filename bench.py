@@ -90,7 +90,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -252,6 +252,7 @@ def main():
         torch.cuda.synchronize(dev)
         if sampler:
             sampler.start()
+        t_region0 = time.perf_counter()
         starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
         stops = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
         for i in range(steps):
@@ -263,8 +264,22 @@ def main():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize(dev)
-        clocks = sampler.stop() if sampler else None
         ms = sum(s.elapsed_time(e) for s, e in zip(starts, stops))
+        clocks = None
+        if sampler:
+            # nvidia-smi needs a few hundred ms to deliver samples: when the timed region was shorter, keep the
+            # same load running (untimed, identical steps) until the sampler has seen about 0.4 s of it
+            t_end = time.perf_counter() + max(0.0, 0.4 - (time.perf_counter() - t_region0))
+            i = 0
+            while time.perf_counter() < t_end:
+                flush.zero_()
+                fn(warmup + steps + i)
+                i += 1
+                if i % 32 == 0:
+                    torch.cuda.synchronize(dev)
+            torch.cuda.synchronize(dev)
+            clocks = sampler.stop()
+            clocks["untimed_tail_steps"] = i
         return ms, clocks
 
     # ---- main arm: injection + detection + correction, inputs resident in HBM
@@ -356,6 +371,8 @@ def main():
             "config": {"workload": WORKLOAD_TEXT[args.config],
                        "l2": "flushed (256 MB memset) before every timed step",
                        "timing": "sum of per-step CUDA-event intervals on the launching stream",
+                       "clocks_sampling": "nvidia-smi every 20 ms over the timed steps, continued over identical untimed "
+                                          "steps until 0.4 s of load have been seen",
                        "trials_per_rank": n_my},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
