@@ -139,31 +139,46 @@ __global__ void __launch_bounds__(256) element_kernel(CampaignParams p)
             }
             float acc_c = 0.0f, acc_f = 0.0f;
             before = 0; after = 0;
-            for (uint32_t k0 = 0; k0 < (uint32_t)p.K; k0 += 32) {
+            // product of term k0 + lane, fetched one 32-term chunk ahead of its use
+            auto fetch = [&](uint32_t k0) -> float {
                 const uint32_t k = k0 + lane;
-                float prod = 0.0f;
-                if (k < (uint32_t)p.K) {
-                    const float a = widen_operand(p.dtype, load_operand(p.dtype, p.A, (size_t)s.row * p.K + k));
-                    const float b = widen_operand(p.dtype, load_operand(p.dtype, p.Bt, (size_t)s.col * p.K + k));
-                    prod = __fmul_rn(a, b);
+                if (k >= (uint32_t)p.K) return 0.0f;
+                const float a = widen_operand(p.dtype, load_operand(p.dtype, p.A, (size_t)s.row * p.K + k));
+                const float b = widen_operand(p.dtype, load_operand(p.dtype, p.Bt, (size_t)s.col * p.K + k));
+                return __fmul_rn(a, b);
+            };
+            auto site_hook = [&]() {
+                if (s.kind == MPGEMMFI_SITE_ACC) {
+                    before = f32_bits(acc_f);
+                    after = before ^ s.xor_mask;
+                    acc_f = bits_f32(after);
+                } else {
+                    before = f32_bits(re2);
+                    after = before ^ s.xor_mask;
+                    bool det;
+                    const uint32_t fin = product_check(p.detect_mode, after, f32_bits(a_site), f32_bits(b_site), det);
+                    acc_f = __fadd_rn(__fsub_rn(acc_f, re2), bits_f32(fin));
                 }
+            };
+            float prod_next = fetch(0);
+            for (uint32_t k0 = 0; k0 < (uint32_t)p.K; k0 += 32) {
+                const float prod = prod_next;
+                prod_next = fetch(k0 + 32);
                 const uint32_t n_here = min(32u, (uint32_t)p.K - k0);
-                for (uint32_t j = 0; j < n_here; ++j) {
-                    const float pj = __shfl_sync(0xFFFFFFFFu, prod, j);
-                    acc_c = __fadd_rn(acc_c, pj);
-                    acc_f = __fadd_rn(acc_f, pj);
-                    if (k0 + j + 1 == kb) {
-                        if (s.kind == MPGEMMFI_SITE_ACC) {
-                            before = f32_bits(acc_f);
-                            after = before ^ s.xor_mask;
-                            acc_f = bits_f32(after);
-                        } else {
-                            before = f32_bits(re2);
-                            after = before ^ s.xor_mask;
-                            bool det;
-                            const uint32_t fin = product_check(p.detect_mode, after, f32_bits(a_site), f32_bits(b_site), det);
-                            acc_f = __fadd_rn(__fsub_rn(acc_f, re2), bits_f32(fin));
-                        }
+                if (n_here == 32 && (kb <= k0 || kb > k0 + 32)) {
+                    // whole chunk, the site does not fall inside it: straight-line additions in k order
+#pragma unroll
+                    for (uint32_t j = 0; j < 32; ++j) {
+                        const float pj = __shfl_sync(0xFFFFFFFFu, prod, j);
+                        acc_c = __fadd_rn(acc_c, pj);
+                        acc_f = __fadd_rn(acc_f, pj);
+                    }
+                } else {
+                    for (uint32_t j = 0; j < n_here; ++j) {
+                        const float pj = __shfl_sync(0xFFFFFFFFu, prod, j);
+                        acc_c = __fadd_rn(acc_c, pj);
+                        acc_f = __fadd_rn(acc_f, pj);
+                        if (k0 + j + 1 == kb) site_hook();
                     }
                 }
             }
