@@ -21,6 +21,7 @@ FP16, BF16, TF32 = 0, 1, 2
 KIND_A, KIND_B, KIND_ACC, KIND_OUT, KIND_TERM = 0, 1, 2, 3, 4
 T_NONE, T_BOUND, T_RMAX, T_RFLIP = 0, 1, 2, 3
 CORRECT = 16
+OUTPUT_RANGE = 64
 
 SITE = np.dtype([("kind", "<u4"), ("row", "<u4"), ("col", "<u4"), ("k", "<u4"),
                  ("xor_mask", "<u4"), ("trial", "<u4"), ("pad0", "<u4"), ("pad1", "<u4")])
@@ -74,6 +75,10 @@ def lib():
         L.orc_campaign.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, vp]
         L.orc_sample.restype = C.c_int
         L.orc_sample.argtypes = [C.c_int] * 4 + [vp, vp, vp, C.c_int, vp, vp, C.c_int, vp, vp]
+        L.orc_operand_exponents.restype = None
+        L.orc_operand_exponents.argtypes = [C.c_int, C.c_int, C.c_int, vp, vp]
+        L.orc_output_range_bound.restype = C.c_int
+        L.orc_output_range_bound.argtypes = [C.c_uint32, C.c_uint32, C.c_int]
         L.orc_summary.restype = None
         L.orc_summary.argtypes = [vp, C.c_int, vp]
         L.orc_absprod.restype = C.c_int
@@ -193,6 +198,18 @@ def sample(dtype, A, Bt, si, sj, sites=None):
     rc = lib().orc_sample(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(s), len(s), _ptr(si), _ptr(sj), len(si), _ptr(out), _ptr(ap))
     assert rc == 0
     return out, ap
+
+
+def operand_exponents(dtype, X):
+    """Largest FP32 exponent field per row of an operand matrix (uint32[rows])."""
+    X = _storage(X, dtype)
+    out = np.zeros(X.shape[0], dtype=np.uint32)
+    lib().orc_operand_exponents(dtype, X.shape[0], X.shape[1], _ptr(X), _ptr(out))
+    return out
+
+
+def output_range_bound(EA, EB, K):
+    return int(lib().orc_output_range_bound(int(EA), int(EB), int(K)))
 
 
 def summary(records):

@@ -263,13 +263,56 @@ static float *widen_matrix(int dtype, const void *src, size_t rows, size_t cols)
 
 static const uint64_t HASH_MUL = 0x9E3779B97F4A7C15ull;
 
-/* output-element check (technique 1 only): returns final bits, sets *det */
-static uint32_t output_check(int detect_mode, uint32_t bits, int *det)
+#define ORC_OUTPUT_RANGE 64
+
+/*
+ * Largest FP32 exponent field in each row of a rows x K operand matrix (for the output-level
+ * range check below). Zero rows give 0, Inf/NaN give 255.
+ */
+void orc_operand_exponents(int dtype, int rows, int K, const void *X, uint32_t *out)
 {
+    for (int r = 0; r < rows; ++r) {
+        uint32_t e = 0;
+        for (int k = 0; k < K; ++k) {
+            uint32_t f = (orc_widen_bits(dtype, load_storage(dtype, X, (size_t)r * K + k)) >> 23) & 0xFFu;
+            if (f > e) e = f;
+        }
+        out[r] = e;
+    }
+}
+
+/*
+ * Output-level range bound (an extension of the product bound of Section VI-A to a dot product):
+ * every |a_ik| < 2^(eA+1) and |b_kj| < 2^(eB+1) with eA, eB the largest exponents of row i of A and of
+ * column j of B, so |C_ij| < K * 2^(eA+eB+2) <= 2^(eA+eB+2+ceil(log2 K)), i.e. the exponent of C_ij is at
+ * most eA + eB + 1 + ceil(log2 K). With biased fields: E <= EA + EB - 126 + ceil(log2 K), clamped to 0..255.
+ */
+int orc_output_range_bound(uint32_t EA, uint32_t EB, int K)
+{
+    int L = 0;
+    while ((1 << L) < K) ++L;
+    int b = (int)EA + (int)EB - 126 + L;
+    if (b < 0) b = 0;
+    if (b > 255) b = 255;
+    return b;
+}
+
+/* output-element check: returns final bits, sets *det. BoundCheck for technique 1; for the RangeCheck
+ * techniques only when an output bound is given (bound >= 0: ORC_OUTPUT_RANGE was requested). */
+static uint32_t output_check(int detect_mode, uint32_t bits, int bound, int *det)
+{
+    int tech = detect_mode & 3;
     *det = 0;
-    if ((detect_mode & 3) != ORC_T_BOUND) return bits;
-    *det = orc_boundcheck_detect(bits);
-    if (*det && (detect_mode & ORC_CORRECT)) return orc_boundcheck_correct(bits);
+    if (tech == ORC_T_BOUND) {
+        *det = orc_boundcheck_detect(bits);
+        if (*det && (detect_mode & ORC_CORRECT)) return orc_boundcheck_correct(bits);
+        return bits;
+    }
+    if ((tech == ORC_T_RMAX || tech == ORC_T_RFLIP) && bound >= 0) {
+        *det = orc_rangecheck_detect(bits, bound);
+        if (*det && (detect_mode & ORC_CORRECT))
+            return tech == ORC_T_RMAX ? orc_rangecheck_max(bits, bound) : orc_rangecheck_flip(bits, bound);
+    }
     return bits;
 }
 
@@ -296,6 +339,17 @@ int orc_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
     float *Bf = widen_matrix(dtype, Bt, (size_t)N, (size_t)K);
     float *BfT = (float *)malloc(sizeof(float) * (size_t)K * (size_t)N);
     if (!Af || !Bf || !BfT) { free(Af); free(Bf); free(BfT); return -1; }
+
+    /* output-level range check: exponent maxima of the CLEAN operands (a faulty operand must not widen its own bound) */
+    uint32_t *EA = NULL, *EB = NULL;
+    int range_out = (detect_mode & ORC_OUTPUT_RANGE) && ((detect_mode & 3) == ORC_T_RMAX || (detect_mode & 3) == ORC_T_RFLIP);
+    if (range_out) {
+        EA = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)M);
+        EB = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)N);
+        orc_operand_exponents(dtype, M, K, A, EA);
+        orc_operand_exponents(dtype, N, K, Bt, EB);
+    }
+#define OUT_BOUND(i, j) (range_out ? orc_output_range_bound(EA[i], EB[j], K) : -1)
 
     uint32_t applied = 0, skipped = 0;
     /* step 3, operand sites: flip the storage word, the faulty value serves the whole row/column */
@@ -367,7 +421,7 @@ int orc_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
         int det;
         *c = u2f(after);
         if (log) { log[t].before_bits = before; log[t].after_bits = after;
-                   log[t].final_bits = output_check(detect_mode, after, &det); log[t].status = 1; }
+                   log[t].final_bits = output_check(detect_mode, after, OUT_BOUND(s->row, s->col), &det); log[t].status = 1; }
     }
     /* a later OUT site on the same element changes what the earlier one finally became */
     if (log)
@@ -375,16 +429,16 @@ int orc_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
             const orc_site *s = &sites[t];
             if (s->kind != ORC_OUT || log[t].status != 1) continue;
             int det;
-            log[t].final_bits = output_check(detect_mode, f2u(C[(size_t)s->row * N + s->col]), &det);
+            log[t].final_bits = output_check(detect_mode, f2u(C[(size_t)s->row * N + s->col]), OUT_BOUND(s->row, s->col), &det);
         }
 
     /* step 4 on every output element */
     uint32_t n_det = 0;
-    if ((detect_mode & 3) == ORC_T_BOUND) {
+    if ((detect_mode & 3) == ORC_T_BOUND || range_out) {
         for (int i = 0; i < M; ++i)
             for (int j = 0; j < N; ++j) {
                 int det;
-                uint32_t fin = output_check(detect_mode, f2u(C[(size_t)i * N + j]), &det);
+                uint32_t fin = output_check(detect_mode, f2u(C[(size_t)i * N + j]), OUT_BOUND(i, j), &det);
                 if (det) {
                     n_det++;
                     if (bitmap) bitmap[(size_t)i * wpr + (size_t)j / 32] |= 1u << (j % 32);
@@ -399,7 +453,8 @@ int orc_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
         hdr[4] = skipped;
         if (skipped) hdr[0] |= 1u;
     }
-    free(Af); free(Bf); free(BfT);
+    free(Af); free(Bf); free(BfT); free(EA); free(EB);
+#undef OUT_BOUND
     return 0;
 }
 
@@ -415,7 +470,7 @@ typedef struct {
 static void trial_account(trial_acc *t, int detect_mode, float value, float clean, uint32_t lin, uint32_t *final_bits)
 {
     int det;
-    uint32_t fin = output_check(detect_mode, f2u(value), &det);
+    uint32_t fin = output_check(detect_mode, f2u(value), -1, &det);   /* campaigns have no output-level range check */
     t->n_aff++;
     if (det) {
         t->n_det++;

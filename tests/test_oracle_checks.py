@@ -125,3 +125,69 @@ def test_term_site_uses_the_selected_technique():
         assert log["final_bits"][0] == want, mode
         # (0 - p) + p' with exact arithmetic here: C equals the checked product (0 + p - p = 0, + p')
         assert f32_bits(float(Cm[0, 0])) == (orc.boundcheck_correct(want) if mode == (orc.T_BOUND | orc.CORRECT) else want)
+
+
+def test_output_range_bound_has_no_false_positive_and_is_tight():
+    """Extension of the product bound to a dot product: E(C_ij) <= EA_i + EB_j - 126 + ceil(log2 K).
+    Never exceeded by a clean GEMM (adversarial: every operand at the top of its binade), reached exactly for
+    K a power of two, and it flags what raises an exponent beyond it."""
+    import synth
+    rng = np.random.default_rng(61)
+    mode = orc.T_RMAX | orc.OUTPUT_RANGE
+    for K in (1, 2, 3, 4, 5, 8, 33, 64, 100, 128):
+        # adversarial: all |a| = |b| = largest BF16 below 2.0, same signs: the sum is as large as it can get
+        a = np.full((3, K), 1.9921875, dtype=np.float32); b = np.full((4, K), 1.9921875, dtype=np.float32)
+        A, Bt = synth.round_to_storage(a, orc.BF16), synth.round_to_storage(b, orc.BF16)
+        Cm, hdr, _, bm = orc.gemm(orc.BF16, A, Bt, None, mode)
+        assert hdr[1] == 0 and not bm.any(), K
+        EA, EB = orc.operand_exponents(orc.BF16, A), orc.operand_exponents(orc.BF16, Bt)
+        assert (EA == 127).all() and (EB == 127).all()
+        bound = orc.output_range_bound(127, 127, K)
+        L = int(np.ceil(np.log2(K))) if K > 1 else 0
+        assert bound == 128 + L
+        E = (Cm.view(np.uint32) >> 23) & 0xFF
+        assert (E <= bound).all()
+        if K & (K - 1) == 0:
+            assert (E == bound).all()                       # tight: K * 1.99^2 sits in the top binade allowed
+        # random data, mixed magnitudes per row: still no flag
+        a = (rng.standard_normal((6, K)) * np.exp2(rng.integers(-20, 20, (6, 1)))).astype(np.float32)
+        b = (rng.standard_normal((5, K)) * np.exp2(rng.integers(-20, 20, (5, 1)))).astype(np.float32)
+        for dt in (orc.FP16, orc.BF16, orc.TF32):
+            aa = np.clip(a, -6e4, 6e4) if dt == orc.FP16 else a
+            bb = np.clip(b, -6e4, 6e4) if dt == orc.FP16 else b
+            A, Bt = synth.round_to_storage(aa, dt), synth.round_to_storage(bb, dt)
+            _, hdr, _, bm = orc.gemm(dt, A, Bt, None, mode)
+            assert hdr[1] == 0, (K, dt)
+    # exponent maxima: zero rows give 0, Inf gives 255, the largest |value| decides otherwise
+    X = synth.round_to_storage(np.array([[0, 0, 0], [0.5, -3.0, 1.0], [np.inf, 1, 1], [1e-3, 0, 0]], dtype=np.float32), orc.BF16)
+    assert list(orc.operand_exponents(orc.BF16, X)) == [0, 128, 255, 117]
+    # detection and the two corrections on an output site, and on an operand fault that the clean maxima expose
+    a = rng.standard_normal((4, 16)).astype(np.float32); b = rng.standard_normal((5, 16)).astype(np.float32)
+    A, Bt = synth.round_to_storage(a, orc.BF16), synth.round_to_storage(b, orc.BF16)
+    s = np.zeros(2, dtype=orc.SITE)
+    s["kind"] = [orc.KIND_OUT, orc.KIND_A]; s["row"] = [1, 3]; s["col"] = [2, 0]; s["k"] = [0, 5]
+    C0, *_ = orc.gemm(orc.BF16, A, Bt)
+    c_bits = int(C0[1, 2].view(np.uint32))
+    up = 1 << 30 if not c_bits & (1 << 30) else 1 << 29          # a flip that raises the exponent by 64 or more
+    assert not c_bits & up
+    s["xor_mask"] = [up, 1 << 14]
+    Cd, hdr, log, bm = orc.gemm(orc.BF16, A, Bt, s, orc.T_RMAX | orc.OUTPUT_RANGE)
+    assert bm[1, 0] & (1 << 2) and hdr[1] >= 2 and hdr[2] == 0
+    assert bin(int(bm[3, 0])).count("1") >= 4                       # the faulty operand lights up most of its row
+    EA, EB = orc.operand_exponents(orc.BF16, A), orc.operand_exponents(orc.BF16, Bt)
+    for tech in (orc.T_RMAX, orc.T_RFLIP):
+        Cc, hdrc, _, bmc = orc.gemm(orc.BF16, A, Bt, s, tech | orc.CORRECT | orc.OUTPUT_RANGE)
+        assert np.array_equal(bmc, bm) and hdrc[2] == hdrc[1]
+        for i in range(4):
+            for j in range(5):
+                bound = orc.output_range_bound(EA[i], EB[j], 16)
+                Ec = (int(Cc[i, j].view(np.uint32)) >> 23) & 0xFF
+                assert Ec <= bound
+                if not (bm[i, 0] >> j) & 1:
+                    assert Cc[i, j].view(np.uint32) == Cd[i, j].view(np.uint32)
+                else:
+                    want = (orc.rangecheck_max if tech == orc.T_RMAX else orc.rangecheck_flip)(int(Cd[i, j].view(np.uint32)), bound)
+                    assert int(Cc[i, j].view(np.uint32)) == want
+    # without the flag the RangeCheck techniques leave outputs alone (they act on TERM products only)
+    _, hdrn, _, bmn = orc.gemm(orc.BF16, A, Bt, s, orc.T_RMAX | orc.CORRECT)
+    assert hdrn[1] == 0 and not bmn.any()
