@@ -101,7 +101,17 @@ enum {
      * shapes 16x8x16 and 16x8x8; Section IV-A: 16 or 8 terms per destination register), instead
      * of at the next mpgemmfi_kstep boundary.
      */
-    MPGEMMFI_TERM_HMMA_STEP = 32
+    MPGEMMFI_TERM_HMMA_STEP = 32,
+    /*
+     * mpgemmfi_gemm_ranged only, together with RANGE_MAX or RANGE_FLIP: also range-check every
+     * OUTPUT element. This extends the product bound of Section VI-A to a dot product and is not in
+     * the paper: with EA_i / EB_j the largest FP32 exponent fields in row i of A / row j of Bt,
+     * |C_ij| < K * 2^(eA+1) * 2^(eB+1), so the exponent field of C_ij is at most
+     * EA_i + EB_j - 126 + ceil(log2 K) (clamped to 0..255). Detection: exponent above that bound;
+     * correction as the technique says (replace by the bound / clear low exponent bits). The
+     * maxima are taken over the CLEAN operands, so a faulty operand shows up in its row or column.
+     */
+    MPGEMMFI_OUTPUT_RANGE = 64
 };
 
 enum {
@@ -188,6 +198,25 @@ typedef struct {
 int mpgemmfi_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C,
                   const mpgemmfi_site *fault_sites, int n_faults, int detect_mode,
                   uint32_t *flags_out, mpgemmfi_stream stream);
+
+/*
+ * Largest FP32 exponent field of each row of a rows x K operand matrix (A, or Bt): out[r] in
+ * 0..255; 0 for an all-zero row, 255 if the row holds Inf or NaN. X and out are device pointers
+ * (X 16-byte aligned, K * element size a multiple of 16 bytes). Input of mpgemmfi_gemm_ranged.
+ * No counterpart in the paper. Errors: ERR_ARG, ERR_DTYPE, ERR_ALIGN, ERR_CUDA.
+ */
+int mpgemmfi_operand_exponents(int dtype, int rows, int K, const void *X, uint32_t *out, mpgemmfi_stream stream);
+
+/*
+ * mpgemmfi_gemm with the output-level range check available: exp_a[M] and exp_bt[N] (device) are the
+ * row maxima of the operands as mpgemmfi_operand_exponents gives them; they are only read when
+ * detect_mode carries MPGEMMFI_OUTPUT_RANGE (and may be NULL otherwise). Everything else as
+ * mpgemmfi_gemm, which itself rejects that flag.
+ */
+int mpgemmfi_gemm_ranged(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C,
+                         const mpgemmfi_site *fault_sites, int n_faults, int detect_mode,
+                         uint32_t *flags_out, const uint32_t *exp_a, const uint32_t *exp_bt,
+                         mpgemmfi_stream stream);
 
 /*
  * Injection campaign: ONE clean GEMM, then every trial is evaluated on the output

@@ -8,7 +8,7 @@ fails loudly when the CUDA library is missing.
 from .binding import (  # noqa: F401
     FP16, BF16, TF32,
     SITE_A, SITE_B, SITE_ACC, SITE_OUT, SITE_TERM,
-    DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP, CORRECT, TERM_HMMA_STEP,
+    DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP, CORRECT, TERM_HMMA_STEP, OUTPUT_RANGE,
     STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT, MAX_FAULTS, HEADER_WORDS, STATIC_MAX_TRIALS,
     TILES_AUTO, TILES_SINGLE, TILES_PAIR, mpgemmfi_set_tile_policy,
     SITE_DTYPE, SITE_LOG_DTYPE, RECORD_DTYPE, SUMMARY_DTYPE,
@@ -17,4 +17,5 @@ from .binding import (  # noqa: F401
     mpgemmfi_flags_bitmap_offset, mpgemmfi_campaign_workspace_bytes,
     mpgemmfi_validate_sites, mpgemmfi_strerror, mpgemmfi_last_cuda_error, mpgemmfi_version,
     gemm, campaign, split_flags, mpgemmfi_campaign_summary, campaign_summary,
+    mpgemmfi_operand_exponents, mpgemmfi_gemm_ranged,
 )

@@ -17,6 +17,7 @@ SITE_A, SITE_B, SITE_ACC, SITE_OUT, SITE_TERM = 0, 1, 2, 3, 4
 DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP = 0, 1, 2, 3
 CORRECT = 16
 TERM_HMMA_STEP = 32
+OUTPUT_RANGE = 64
 STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT = 1, 2
 MAX_FAULTS = 4096
 STATIC_MAX_TRIALS = 65536
@@ -42,7 +43,7 @@ _SYMBOLS = [
     "mpgemmfi_gemm", "mpgemmfi_campaign", "mpgemmfi_kstep", "mpgemmfi_flags_bytes",
     "mpgemmfi_flags_bitmap_offset", "mpgemmfi_campaign_workspace_bytes", "mpgemmfi_validate_sites",
     "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version", "mpgemmfi_campaign_static",
-    "mpgemmfi_set_tile_policy", "mpgemmfi_campaign_summary",
+    "mpgemmfi_set_tile_policy", "mpgemmfi_campaign_summary", "mpgemmfi_operand_exponents", "mpgemmfi_gemm_ranged",
 ]
 
 
@@ -79,6 +80,10 @@ def load_library():
     L.mpgemmfi_campaign.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp, sz, vp]
     L.mpgemmfi_campaign_static.restype = i
     L.mpgemmfi_campaign_static.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp]
+    L.mpgemmfi_operand_exponents.restype = i
+    L.mpgemmfi_operand_exponents.argtypes = [i, i, i, vp, vp, vp]
+    L.mpgemmfi_gemm_ranged.restype = i
+    L.mpgemmfi_gemm_ranged.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp, vp, vp]
     L.mpgemmfi_campaign_summary.restype = i
     L.mpgemmfi_campaign_summary.argtypes = [vp, i, vp, vp]
     L.mpgemmfi_set_tile_policy.restype = i
@@ -120,6 +125,17 @@ def mpgemmfi_campaign_static(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, de
     for callers that are not allowed to allocate device memory. At most STATIC_MAX_TRIALS trials per call."""
     return load_library().mpgemmfi_campaign_static(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mode,
                                                    records, stream)
+
+
+def mpgemmfi_operand_exponents(dtype, rows, K, X, out, stream):
+    """Raw call: out[r] = largest FP32 exponent field of row r of the rows x K operand matrix X (device pointers)."""
+    return load_library().mpgemmfi_operand_exponents(dtype, rows, K, X, out, stream)
+
+
+def mpgemmfi_gemm_ranged(dtype, M, N, K, A, Bt, C_out, fault_sites, n_faults, detect_mode, flags_out, exp_a, exp_bt, stream):
+    """Raw call: mpgemmfi_gemm with the operands' exponent maxima for the output-level range check (OUTPUT_RANGE)."""
+    return load_library().mpgemmfi_gemm_ranged(dtype, M, N, K, A, Bt, C_out, fault_sites, n_faults, detect_mode,
+                                               flags_out, exp_a, exp_bt, stream)
 
 
 def mpgemmfi_campaign_summary(records, n_trials, summary, stream):
@@ -228,6 +244,20 @@ def gemm(dtype, A, Bt, sites=None, detect_mode=DETECT_NONE, C_out=None, flags_ou
     if flags_out is None:
         flags_out = torch.empty(mpgemmfi_flags_bytes(M, N, n_faults) // 4, dtype=torch.int32, device=A.device)
     stream_h = (torch.cuda.current_stream(A.device) if stream is None else stream).cuda_stream
+    if detect_mode & OUTPUT_RANGE:
+        # output-level range check: the exponent maxima of the (clean) operands come first
+        ea = torch.empty(M, dtype=torch.int32, device=A.device)
+        eb = torch.empty(N, dtype=torch.int32, device=A.device)
+        for X, rows, e in ((A, M, ea), (Bt, N, eb)):
+            rc = mpgemmfi_operand_exponents(dtype, rows, K, X.data_ptr(), e.data_ptr(), stream_h)
+            if rc != 0:
+                raise MpgemmfiError(rc, "mpgemmfi_operand_exponents")
+        rc = mpgemmfi_gemm_ranged(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), C_out.data_ptr(),
+                                  st.data_ptr() if st is not None else None, n_faults, detect_mode,
+                                  flags_out.data_ptr(), ea.data_ptr(), eb.data_ptr(), stream_h)
+        if rc != 0:
+            raise MpgemmfiError(rc, "mpgemmfi_gemm_ranged")
+        return C_out, flags_out
     rc = mpgemmfi_gemm(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), C_out.data_ptr(),
                        st.data_ptr() if st is not None else None, n_faults, detect_mode,
                        flags_out.data_ptr(), stream_h)

@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmpgemmfi.so")
-SOURCES = ["api.cu", "gemm_sm100.cu", "campaign.cu"]
+SOURCES = ["api.cu", "gemm_sm100.cu", "campaign.cu", "operands.cu"]
 
 
 def _newest_source_mtime() -> float:

@@ -8,6 +8,7 @@
 #include "campaign.cuh"
 #include "checks.cuh"
 #include "gemm_sm100.cuh"
+#include "operands.cuh"
 
 static_assert(MPGEMMFI_STATIC_MAX_TRIALS == mpg::CAMPAIGN_STATIC_MAX_TRIALS, "header and kernel limits differ");
 
@@ -121,7 +122,8 @@ int check_common(int dtype, int M, int N, int K, const void *A, const void *Bt, 
 }
 
 int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C, const mpgemmfi_site *sites,
-             int n_faults, int detect_mode, uint32_t *flags, cudaStream_t stream, const DeviceInfo &di)
+             int n_faults, int detect_mode, uint32_t *flags, cudaStream_t stream, const DeviceInfo &di,
+             const uint32_t *exp_a = nullptr, const uint32_t *exp_bt = nullptr)
 {
     int max_pairs = 0;
     const bool pair = choose_pair(dtype, M, N, &max_pairs);
@@ -146,6 +148,9 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
     p.wpr = (N + 31) / 32;
     p.c_vec_ok = (N % 4 == 0) && (((uintptr_t)C & 15) == 0);
     p.A = A; p.Bt = Bt; p.C = C; p.sites = sites; p.flags = flags;
+    p.exp_a = exp_a; p.exp_b = exp_bt;
+    p.log2_k = 0;
+    while ((1 << p.log2_k) < K) ++p.log2_k;
     if (flags) {
         const cudaError_t e = cudaMemsetAsync(flags, 0, sizeof(uint32_t) * (MPGEMMFI_HEADER_WORDS + 4 * (size_t)n_faults), stream);
         if (e != cudaSuccess) return cuda_fail(e);
@@ -176,6 +181,43 @@ int mpgemmfi_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt,
     if (di.major != 10) return MPGEMMFI_ERR_ARCH;
     return run_gemm(dtype, M, N, K, A, Bt, C, fault_sites, n_faults, detect_mode, flags_out,
                     static_cast<cudaStream_t>(stream), di);
+}
+
+int mpgemmfi_gemm_ranged(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C,
+                         const mpgemmfi_site *fault_sites, int n_faults, int detect_mode, uint32_t *flags_out,
+                         const uint32_t *exp_a, const uint32_t *exp_bt, mpgemmfi_stream stream)
+{
+    int rc = check_common(dtype, M, N, K, A, Bt, C);
+    if (rc) return rc;
+    if (n_faults < 0 || n_faults > MPGEMMFI_MAX_FAULTS || (n_faults > 0 && !fault_sites)) return MPGEMMFI_ERR_ARG;
+    if (detect_mode & ~(MPGEMMFI_DETECT_TECHNIQUE_MASK | MPGEMMFI_CORRECT | MPGEMMFI_OUTPUT_RANGE)) return MPGEMMFI_ERR_ARG;
+    const int tech = detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK;
+    if (detect_mode & MPGEMMFI_OUTPUT_RANGE) {
+        if (tech != MPGEMMFI_DETECT_RANGE_MAX && tech != MPGEMMFI_DETECT_RANGE_FLIP) return MPGEMMFI_ERR_ARG;
+        if (!exp_a || !exp_bt) return MPGEMMFI_ERR_ARG;
+        if (((uintptr_t)exp_a & 3) || ((uintptr_t)exp_bt & 3)) return MPGEMMFI_ERR_ALIGN;
+    }
+    if (!flags_out && (n_faults > 0 || tech)) return MPGEMMFI_ERR_ARG;
+    if (((uintptr_t)fault_sites & 15) || ((uintptr_t)flags_out & 15)) return MPGEMMFI_ERR_ALIGN;
+    DeviceInfo di;
+    rc = device_info(di);
+    if (rc) return rc;
+    if (di.major != 10) return MPGEMMFI_ERR_ARCH;
+    const bool ranged = (detect_mode & MPGEMMFI_OUTPUT_RANGE) != 0;
+    return run_gemm(dtype, M, N, K, A, Bt, C, fault_sites, n_faults, detect_mode, flags_out,
+                    static_cast<cudaStream_t>(stream), di, ranged ? exp_a : nullptr, ranged ? exp_bt : nullptr);
+}
+
+int mpgemmfi_operand_exponents(int dtype, int rows, int K, const void *X, uint32_t *out, mpgemmfi_stream stream)
+{
+    if (dtype != MPGEMMFI_FP16 && dtype != MPGEMMFI_BF16 && dtype != MPGEMMFI_TF32) return MPGEMMFI_ERR_DTYPE;
+    if (rows <= 0 || K <= 0 || !X || !out) return MPGEMMFI_ERR_ARG;
+    if (((uintptr_t)X & 15) || ((uintptr_t)out & 3) || ((size_t)K * mpg::esize_of(dtype)) % 16) return MPGEMMFI_ERR_ALIGN;
+    DeviceInfo di;
+    const int rc = device_info(di);
+    if (rc) return rc;
+    const cudaError_t e = mpg::launch_operand_exponents(dtype, rows, K, X, out, di.num_sms, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
 }
 
 int mpgemmfi_campaign(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C_clean,

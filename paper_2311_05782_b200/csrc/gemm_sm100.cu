@@ -598,8 +598,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         // ------------------------------------------------------------ epilogue (own 128 rows)
         const int q = warp & 3;               // TMEM lane quarter this warp may access
         const int h = (warp - 4) >> 2;        // column half of the tile this warp handles
-        const bool do_bound = (p.detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK) == MPGEMMFI_DETECT_BOUNDCHECK;
-        const bool do_corr = do_bound && (p.detect_mode & MPGEMMFI_CORRECT);
+        const int tech = p.detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK;
+        const bool do_bound = tech == MPGEMMFI_DETECT_BOUNDCHECK;
+        const bool do_range = (p.detect_mode & MPGEMMFI_OUTPUT_RANGE) && p.exp_a != nullptr &&
+                              (tech == MPGEMMFI_DETECT_RANGE_MAX || tech == MPGEMMFI_DETECT_RANGE_FLIP);
+        const bool range_flip = tech == MPGEMMFI_DETECT_RANGE_FLIP;
+        const bool do_corr = (do_bound || do_range) && (p.detect_mode & MPGEMMFI_CORRECT);
         uint32_t lt = 0, pause_phase = 0, n_det = 0;
         uint32_t *bitmap = p.flags ? p.flags + MPGEMMFI_HEADER_WORDS + 4 * (size_t)p.n_faults : nullptr;
         uint8_t *my_out = stage_out + (warp - 4) * (16 * 128);
@@ -635,6 +639,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             const uint32_t row = tc.m0 + (uint32_t)(q * 32 + lane);
             const uint32_t row0 = tc.m0 + (uint32_t)(q * 32);
             const bool row_ok = row < (uint32_t)p.M;
+            const uint32_t row_e = (do_range && row_ok) ? __ldg(p.exp_a + row) : 0u;
             float *crow = p.C + (size_t)row * p.N;
             const uint32_t t_lane = tmem_acc + ((uint32_t)(q * 32) << 16);
             constexpr int MY_PIECES = BN / 64;          // 32-column pieces per warp (half the tile's columns)
@@ -644,8 +649,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             // One 32-column piece of this thread's row: output sites, check, flags, store.
             auto finish_piece = [&](uint32_t (&v)[32], int i) {
                 const uint32_t c0 = tc.n0 + (uint32_t)((first + i) * 32);
+                // output-level range check: this lane fetches the exponent maximum of column c0 + lane early
+                uint32_t col_e = 0;
+                if (do_range && c0 + (uint32_t)lane < (uint32_t)p.N) col_e = __ldg(p.exp_b + c0 + lane);
                 if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 0);
                 uint32_t fw = 0;
+                if (do_range) {
+                    const int row_part = (int)row_e - 126 + p.log2_k;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int bound = min(255, max(0, row_part + (int)__shfl_sync(0xFFFFFFFFu, col_e, j)));
+                        const bool det = (int)((v[j] >> 23) & 0xFFu) > bound;
+                        if (det) {
+                            fw |= 1u << j;
+                            if (do_corr) v[j] = range_flip ? rangecheck_flip(v[j], bound) : rangecheck_max(v[j], bound);
+                        }
+                    }
+                    if (c0 + 32 > (uint32_t)p.N) fw &= c0 < (uint32_t)p.N ? (1u << ((uint32_t)p.N - c0)) - 1u : 0u;
+                }
                 if (do_bound) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {

@@ -21,6 +21,10 @@ struct GemmParams {
     float *C;
     const mpgemmfi_site *sites;
     uint32_t *flags;
+    // output-level range check (null when not requested): row exponent maxima of A and Bt, ceil(log2 K)
+    const uint32_t *exp_a;
+    const uint32_t *exp_b;
+    int log2_k;
 };
 
 // shared-memory pipeline depth used for an output tile that is bn columns wide

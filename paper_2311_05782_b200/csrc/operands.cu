@@ -1,0 +1,51 @@
+// Per-row exponent maxima of an operand matrix (input of the output-level range check).
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "checks.cuh"
+#include "operands.cuh"
+
+namespace mpg {
+
+namespace {
+
+// One warp per row; 16-byte loads; the maximum of the biased FP32 exponent fields of the widened values.
+__global__ void __launch_bounds__(256) exponent_max_kernel(int dtype, int rows, int K, const void *X, uint32_t *out)
+{
+    const int lane = threadIdx.x & 31;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int n_warps = (gridDim.x * blockDim.x) >> 5;
+    const int es = esize_of(dtype);
+    const int vecs = K * es / 16;                       // K * es is a multiple of 16
+    for (int r = warp; r < rows; r += n_warps) {
+        const uint4 *row = reinterpret_cast<const uint4 *>(reinterpret_cast<const unsigned char *>(X) + (size_t)r * K * es);
+        uint32_t e = 0;
+        for (int v = lane; v < vecs; v += 32) {
+            const uint4 x = __ldg(row + v);
+            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (es == 4) {
+                    e = max(e, (w[i] >> 23) & 0xFFu);
+                } else {
+                    e = max(e, (f32_bits(widen_operand(dtype, w[i] & 0xFFFFu)) >> 23) & 0xFFu);
+                    e = max(e, (f32_bits(widen_operand(dtype, w[i] >> 16)) >> 23) & 0xFFu);
+                }
+            }
+        }
+        e = __reduce_max_sync(0xFFFFFFFFu, e);
+        if (lane == 0) out[r] = e;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_operand_exponents(int dtype, int rows, int K, const void *X, uint32_t *out, int num_sms,
+                                     cudaStream_t stream)
+{
+    const int grid = max(1, min((rows + 7) / 8, 8 * num_sms));
+    exponent_max_kernel<<<grid, 256, 0, stream>>>(dtype, rows, K, X, out);
+    return cudaGetLastError();
+}
+
+}  // namespace mpg

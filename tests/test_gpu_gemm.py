@@ -269,3 +269,70 @@ def test_degenerate_shapes_and_special_values(dtype, tile_policy):
         info = [(int(i), int(w), hex(int(bm[i, w])), hex(int(bm_o[i, w])), Cg[i, 32 * w:32 * w + 32][:12].tolist(), Co[i, 32 * w:32 * w + 32][:12].tolist()) for i, w in d[:3]]
         assert np.array_equal(bm, bm_o) and hdr[1] == hdr_o[1], info      # NaN, Inf and huge values are flagged alike
         assert (Cg[20][np.isfinite(tol[20])] == 0).all() and (Cg[:, 6][np.isfinite(tol[:, 6])] == 0).all()
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_output_level_range_check(dtype, tile_policy):
+    """RangeCheck extended to output elements (exponent maxima of the clean operands): clean runs flag nothing,
+    operand / output / accumulator faults that push an exponent over the bound are flagged and corrected as the oracle says."""
+    kt = synth.kstep(dtype)
+    M, N, K = 300, 330, 4 * kt + 8
+    rng = np.random.default_rng(71)
+    a = (rng.standard_normal((M, K)) * np.exp2(rng.integers(-6, 6, (M, 1)))).astype(np.float32)
+    b = (rng.standard_normal((N, K)) * np.exp2(rng.integers(-6, 6, (N, 1)))).astype(np.float32)
+    A, Bt = synth.round_to_storage(a, dtype), synth.round_to_storage(b, dtype)
+    # exponent maxima kernel against the oracle
+    ea = torch.empty(M, dtype=torch.int32, device="cuda"); eb = torch.empty(N, dtype=torch.int32, device="cuda")
+    da, db = to_dev(A, dtype), to_dev(Bt, dtype)
+    st = torch.cuda.current_stream().cuda_stream
+    assert mpg.mpgemmfi_operand_exponents(dtype, M, K, da.data_ptr(), ea.data_ptr(), st) == 0
+    assert mpg.mpgemmfi_operand_exponents(dtype, N, K, db.data_ptr(), eb.data_ptr(), st) == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(ea.cpu().numpy().view(np.uint32), orc.operand_exponents(dtype, A))
+    assert np.array_equal(eb.cpu().numpy().view(np.uint32), orc.operand_exponents(dtype, Bt))
+    width = 19 if dtype == orc.TF32 else 16
+    sites = np.concatenate([
+        site(orc.KIND_A, 17, 0, 5, 1 << (width - 2)), site(orc.KIND_B, 0, 200, kt + 3, 1 << (width - 2)),
+        site(orc.KIND_OUT, 299, 329, 0, 1 << 30), site(orc.KIND_OUT, 150, 31, 0, 1 << 29), site(orc.KIND_OUT, 3, 64, 0, 1 << 23),
+        site(orc.KIND_ACC, 250, 100, 2 * kt, 1 << 30), site(orc.KIND_TERM, 40, 40, 3 * kt + 1, 1 << 30),
+    ])
+    for mode in (orc.T_RMAX | orc.OUTPUT_RANGE, orc.T_RMAX | orc.CORRECT | orc.OUTPUT_RANGE, orc.T_RFLIP | orc.CORRECT | orc.OUTPUT_RANGE):
+        Cg, hdr, log, bm = run_gpu_gemm(dtype, A, Bt, None, mode)
+        assert hdr[0] == 0 and hdr[1] == 0 and not bm.any()           # no false positive on a clean product
+        Cg, hdr, log, bm = run_gpu_gemm(dtype, A, Bt, sites, mode)
+        Co, hdr_o, log_o, bm_o = orc.gemm(dtype, A, Bt, sites, mode)
+        assert hdr[0] == 0 and hdr[3] == len(sites)
+        # flags: exact, except where an element sits within rounding of a binade edge that the bound happens to be
+        diff = bm ^ bm_o
+        assert sum(bin(int(x)).count("1") for x in diff.reshape(-1)) <= 2
+        assert hdr[1] > N // 2                                          # the faulty A element shows in most of its row
+        assert abs(int(hdr[1]) - int(hdr_o[1])) <= 2
+        from parity import faulted_operands
+        A2, B2 = faulted_operands(dtype, A, Bt, sites)
+        tol = TOL * orc.absprod(dtype, A2, B2)
+        touched = np.zeros((M, N), dtype=bool)
+        for s_ in sites:
+            if s_["kind"] in (orc.KIND_OUT, orc.KIND_ACC, orc.KIND_TERM):
+                touched[s_["row"], s_["col"]] = True
+        unflagged = np.zeros((M, N), dtype=bool)
+        for i in range(M):
+            for w in range(bm.shape[1]):
+                both = ~(bm[i, w] | bm_o[i, w])
+                for j in range(32 * w, min(N, 32 * w + 32)):
+                    unflagged[i, j] = (both >> (j % 32)) & 1
+        assert (close(Cg, Co, tol) | touched | ~unflagged).all()
+        if mode & orc.CORRECT:
+            # every stored exponent respects its bound
+            EA, EB = orc.operand_exponents(dtype, A), orc.operand_exponents(dtype, Bt)
+            L = int(np.ceil(np.log2(K)))
+            bound = np.clip(EA[:, None].astype(np.int64) + EB[None, :].astype(np.int64) - 126 + L, 0, 255)
+            assert (((Cg.view(np.uint32) >> 23) & 0xFF).astype(np.int64) <= bound).all()
+    # the plain entry point refuses the flag; the ranged one refuses it with BoundCheck or without maxima
+    c = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    f = torch.empty(mpg.mpgemmfi_flags_bytes(M, N, 0) // 4, dtype=torch.int32, device="cuda")
+    args = (dtype, M, N, K, da.data_ptr(), db.data_ptr(), c.data_ptr(), None, 0)
+    assert mpg.mpgemmfi_gemm(*args, orc.T_RMAX | orc.OUTPUT_RANGE, f.data_ptr(), st) == -1
+    assert mpg.mpgemmfi_gemm_ranged(*args, orc.T_BOUND | orc.OUTPUT_RANGE, f.data_ptr(), ea.data_ptr(), eb.data_ptr(), st) == -1
+    assert mpg.mpgemmfi_gemm_ranged(*args, orc.T_RMAX | orc.OUTPUT_RANGE, f.data_ptr(), None, eb.data_ptr(), st) == -1
+    assert mpg.mpgemmfi_gemm_ranged(*args, orc.T_RMAX, f.data_ptr(), None, None, st) == 0
+    torch.cuda.synchronize()
