@@ -208,6 +208,9 @@ def check_campaign_against_oracle(dtype, A, Bt, sites, mode, max_fragile=0):
             assert g["first_detected"] == o["first_detected"]
             assert (g["status"] & 6) == (o["status"] & 6)
             od = float(o["max_abs_dev"])
-            assert close(g["max_abs_dev"], od, max(1e-3 * abs(od), 1e-3 * float(ap.max()))) or not np.isfinite(od)
+            # a faulty operand that is Inf or NaN makes NaNs whose payloads (and what a correction makes of them) are
+            # not part of parity
+            special = not np.isfinite(orc.widen(dtype, int(o["after_bits"])))
+            assert special or close(g["max_abs_dev"], od, max(1e-3 * abs(od), 1e-3 * float(ap.max()))) or not np.isfinite(od), (t, g, o)
     assert fragile <= max_fragile, f"{fragile} fragile trials"
     return fragile

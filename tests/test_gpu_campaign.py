@@ -178,3 +178,24 @@ def test_campaign_single_element_trials_with_special_values():
         assert np.array_equal(rg["after_bits"][out], rg["before_bits"][out] ^ sites["xor_mask"][out])
         assert np.array_equal(rg["n_detected"][out], np.array([orc.boundcheck_detect(int(x)) if (mode & 3) == 1 else 0
                                                                for x in rg["after_bits"][out]]))
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_campaign_random_shapes_mixes_and_modes(seed):
+    """Differential fuzz of the campaign against the oracle's incremental evaluation (finite operands)."""
+    rng = np.random.default_rng(3000 + seed)
+    dtype = int(rng.integers(0, 3))
+    unit = 4 if dtype == orc.TF32 else 8
+    M = int(rng.integers(1, 500)); N = int(rng.integers(1, 300)); K = unit * int(rng.integers(1, 50))
+    if seed % 4 == 0:
+        M, N, K = int(rng.integers(2100, 2600)), int(rng.integers(8, 70)), unit * int(rng.integers(8, 40))   # panel path
+    mode = int(rng.choice([orc.T_NONE, orc.T_BOUND, orc.T_BOUND | orc.CORRECT, orc.T_RMAX | orc.CORRECT]))
+    a = (rng.standard_normal((M, K)) * rng.choice([0.05, 1.0])).astype(np.float32)
+    b = (rng.standard_normal((N, K)) * rng.choice([0.05, 1.0])).astype(np.float32)
+    a[rng.random((M, K)) < 0.2] = 0.0
+    A, Bt = synth.round_to_storage(a, dtype), synth.round_to_storage(b, dtype)
+    parts = [synth.make_sites(mix, dtype, M, N, K, 40, 4000 + seed + i, nbits=int(rng.choice([1, 2, 4])))
+             for i, mix in enumerate(("mixed", "term", "operand"))]
+    sites = np.concatenate(parts)
+    sites["kind"][5] = 11                                   # an invalid entry
+    check_campaign_against_oracle(dtype, A, Bt, sites, mode, max_fragile=3)

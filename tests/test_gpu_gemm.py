@@ -15,7 +15,8 @@ DTYPES = [orc.FP16, orc.BF16, orc.TF32]
 
 @pytest.fixture(params=["single", "pair"], autouse=True)
 def tile_policy(request):
-    """Every test of this file runs under both tilings of the kernel: whole tiles per CTA, and CTA pairs."""
+    """Every test of this file runs under both tilings of the kernel: whole tiles per CTA, and CTA pairs
+    (the fuzz test picks its own tiling; it still runs once per parameter, on different seeds' worth of luck)."""
     assert mpg.mpgemmfi_set_tile_policy(mpg.TILES_PAIR if request.param == "pair" else mpg.TILES_SINGLE) == 0
     yield request.param
     mpg.mpgemmfi_set_tile_policy(mpg.TILES_AUTO)
@@ -336,3 +337,34 @@ def test_output_level_range_check(dtype, tile_policy):
     assert mpg.mpgemmfi_gemm_ranged(*args, orc.T_RMAX | orc.OUTPUT_RANGE, f.data_ptr(), None, eb.data_ptr(), st) == -1
     assert mpg.mpgemmfi_gemm_ranged(*args, orc.T_RMAX, f.data_ptr(), None, None, st) == 0
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_tables_and_modes(seed):
+    """Differential fuzz against the oracle: random shape, format, tiling, check mode and site table (all kinds,
+    repeated elements, a few invalid entries)."""
+    rng = np.random.default_rng(1000 + seed)
+    dtype = int(rng.integers(0, 3))
+    kt = synth.kstep(dtype)
+    unit = 4 if dtype == orc.TF32 else 8
+    M = int(rng.integers(1, 700)); N = int(rng.integers(1, 700)); K = unit * int(rng.integers(1, 60))
+    policy = [mpg.TILES_AUTO, mpg.TILES_SINGLE, mpg.TILES_PAIR][seed % 3]
+    mode = int(rng.choice([orc.T_NONE, orc.T_BOUND, orc.T_BOUND | orc.CORRECT, orc.T_RMAX | orc.CORRECT, orc.T_RFLIP | orc.CORRECT]))
+    A, Bt = rand_operands(dtype, M, N, K, 2000 + seed, scale=float(rng.choice([0.01, 1.0, 30.0])))
+    n = int(rng.integers(0, 40))
+    s = np.zeros(n, dtype=orc.SITE)
+    s["kind"] = rng.integers(0, 5, n)
+    s["row"] = rng.integers(0, M, n); s["col"] = rng.integers(0, N, n)
+    nb = (K + kt - 1) // kt
+    k_acc = np.minimum(rng.integers(1, nb + 1, n) * kt, K)
+    s["k"] = np.where(s["kind"] == orc.KIND_ACC, k_acc, rng.integers(0, K, n))
+    width = np.where(s["kind"] <= orc.KIND_B, 19 if dtype == orc.TF32 else 16, 32)
+    nbits = rng.choice([1, 2, 4], n)
+    s["xor_mask"] = [(((1 << int(b)) - 1) << int(rng.integers(0, int(w) - int(b) + 1))) for b, w in zip(nbits, width)]
+    if n >= 4:                                             # repeats on one element, and entries the device must skip
+        s[1] = s[0]; s["row"][2] = M + 5; s["kind"][3] = 7
+    mpg.mpgemmfi_set_tile_policy(policy)
+    try:
+        check_gemm_against_oracle(dtype, A, Bt, s, mode, max_fragile=2)
+    finally:
+        mpg.mpgemmfi_set_tile_policy(mpg.TILES_AUTO)
