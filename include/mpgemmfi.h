@@ -135,7 +135,9 @@ enum {
 /*
  * flags_out layout (uint32 words):
  *   [0 .. 16)            header: [0] status, [1] n_detected, [2] n_corrected,
- *                        [3] sites applied, [4] sites skipped, rest reserved (0)
+ *                        [3] sites applied, [4] sites skipped, [5] number of runs of k-steps the
+ *                        tiles of the last round were cut into (0: whole tiles, see
+ *                        mpgemmfi_set_split_policy), rest reserved (0)
  *   [16 .. 16+4*n_faults) site log, one entry per table entry (the paper logs the sum
  *                        before and after injection the same way, Section V-B):
  *                        {before_bits, after_bits, final_bits, status}
@@ -314,6 +316,30 @@ enum {
     MPGEMMFI_TILES_PAIR = 2
 };
 int mpgemmfi_set_tile_policy(int policy);
+
+/*
+ * Tuning knob (no counterpart in the paper): what happens to the last round of tiles when the
+ * tile count is not a multiple of the number of tile walkers (CTAs or CTA pairs), so that the last
+ * round would leave walkers idle.
+ *   AUTO   the library cuts that round's tiles along K when that shortens the launch (default)
+ *   OFF    every tile is computed whole by one walker
+ *   ON     cut whenever the shape allows it (more tiles than walkers, at most half as many tiles left
+ *          over as walkers, C and N fit 16-byte accesses), also where it does not pay: for tests
+ * A cut tile is run as two to four consecutive runs of k-steps by different walkers at different
+ * times; the unfinished FP32 accumulators wait in the tile's place in C and go back into the
+ * tensor core's accumulator memory before the next run, so every element is still one FP32
+ * accumulation in increasing k, bit-identical to the uncut tile, and accumulator / term sites meet
+ * the same running sum. While the launch runs, C therefore holds intermediate values in those
+ * tiles. The hand-over between walkers uses 160 KB of static device memory of the library,
+ * tagged per launch. Process-wide, not thread-safe against concurrent launches.
+ * Returns MPGEMMFI_OK or MPGEMMFI_ERR_ARG.
+ */
+enum {
+    MPGEMMFI_SPLIT_AUTO = 0,
+    MPGEMMFI_SPLIT_OFF = 1,
+    MPGEMMFI_SPLIT_ON = 2
+};
+int mpgemmfi_set_split_policy(int policy);
 
 /* k elements between two accumulator boundaries: 64 (FP16, BF16), 32 (TF32); 0 for a bad dtype. */
 int mpgemmfi_kstep(int dtype);

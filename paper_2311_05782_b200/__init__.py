@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP, CORRECT, TERM_HMMA_STEP, OUTPUT_RANGE,
     STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT, MAX_FAULTS, HEADER_WORDS, STATIC_MAX_TRIALS,
     TILES_AUTO, TILES_SINGLE, TILES_PAIR, mpgemmfi_set_tile_policy,
+    SPLIT_AUTO, SPLIT_OFF, SPLIT_ON, mpgemmfi_set_split_policy,
     SITE_DTYPE, SITE_LOG_DTYPE, RECORD_DTYPE, SUMMARY_DTYPE,
     MpgemmfiError, library_path, load_library, exported_symbols,
     mpgemmfi_gemm, mpgemmfi_campaign, mpgemmfi_campaign_static, mpgemmfi_kstep, mpgemmfi_flags_bytes,

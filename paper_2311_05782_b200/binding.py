@@ -22,6 +22,7 @@ STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT = 1, 2
 MAX_FAULTS = 4096
 STATIC_MAX_TRIALS = 65536
 TILES_AUTO, TILES_SINGLE, TILES_PAIR = 0, 1, 2
+SPLIT_AUTO, SPLIT_OFF, SPLIT_ON = 0, 1, 2
 HEADER_WORDS = 16
 
 SITE_DTYPE = np.dtype([("kind", "<u4"), ("row", "<u4"), ("col", "<u4"), ("k", "<u4"),
@@ -43,7 +44,7 @@ _SYMBOLS = [
     "mpgemmfi_gemm", "mpgemmfi_campaign", "mpgemmfi_kstep", "mpgemmfi_flags_bytes",
     "mpgemmfi_flags_bitmap_offset", "mpgemmfi_campaign_workspace_bytes", "mpgemmfi_validate_sites",
     "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version", "mpgemmfi_campaign_static",
-    "mpgemmfi_set_tile_policy", "mpgemmfi_campaign_summary", "mpgemmfi_operand_exponents", "mpgemmfi_gemm_ranged",
+    "mpgemmfi_set_tile_policy", "mpgemmfi_set_split_policy", "mpgemmfi_campaign_summary", "mpgemmfi_operand_exponents", "mpgemmfi_gemm_ranged",
 ]
 
 
@@ -88,6 +89,8 @@ def load_library():
     L.mpgemmfi_campaign_summary.argtypes = [vp, i, vp, vp]
     L.mpgemmfi_set_tile_policy.restype = i
     L.mpgemmfi_set_tile_policy.argtypes = [i]
+    L.mpgemmfi_set_split_policy.restype = i
+    L.mpgemmfi_set_split_policy.argtypes = [i]
     L.mpgemmfi_kstep.restype = i
     L.mpgemmfi_kstep.argtypes = [i]
     L.mpgemmfi_flags_bytes.restype = sz
@@ -157,6 +160,11 @@ def campaign_summary(records, stream=None):
 def mpgemmfi_set_tile_policy(policy):
     """TILES_AUTO (0), TILES_SINGLE (1) or TILES_PAIR (2); process-wide."""
     return load_library().mpgemmfi_set_tile_policy(policy)
+
+
+def mpgemmfi_set_split_policy(policy):
+    """SPLIT_AUTO (0), SPLIT_OFF (1) or SPLIT_ON (2); process-wide."""
+    return load_library().mpgemmfi_set_split_policy(policy)
 
 
 def mpgemmfi_kstep(dtype):

@@ -86,6 +86,30 @@ int encode_operand_map(CUtensorMap *map, int dtype, const void *base, int rows, 
 }
 
 int g_tile_policy = MPGEMMFI_TILES_AUTO;
+int g_split_policy = MPGEMMFI_SPLIT_AUTO;
+
+// Split schedule for `tiles` tiles on `walkers` tile walkers: fills the three schedule fields of p.
+// Off unless there is at least one full round, the left-over tiles number at most half the walkers,
+// every part keeps at least four k-tiles, and (policy AUTO) the launch gets visibly shorter.
+void choose_split(mpg::GemmParams &p, int walkers)
+{
+    p.split_parts = 0; p.full_rounds = 0; p.left_tiles = 0;
+    if (g_split_policy == MPGEMMFI_SPLIT_OFF || !p.c_vec_ok) return;
+    const int rounds = p.num_tiles / walkers, left = p.num_tiles % walkers;
+    if (rounds < 1 || left == 0 || left * 16 > mpg::SPLIT_SIGNAL_WORDS) return;
+    int parts = walkers / left;
+    if (parts > 4) parts = 4;
+    if (parts > rounds + 1) parts = rounds + 1;
+    while (parts >= 2 && p.num_kt / parts < 4) --parts;
+    if (parts < 2) return;
+    if (g_split_policy == MPGEMMFI_SPLIT_AUTO) {
+        // a cut tile costs its walkers one more pass of accumulators through C (measured: about 5 us); it
+        // pays when the k-tiles saved (0.35 us each) outweigh that and are a visible share of the launch
+        const int saved = p.num_kt - (p.num_kt + parts - 1) / parts;
+        if (saved < 24 || saved < 0.03 * (rounds + 1) * p.num_kt) return;
+    }
+    p.split_parts = parts; p.full_rounds = rounds; p.left_tiles = left;
+}
 
 // widest tile that still gives every SM a tile; narrow outputs get narrow tiles
 int choose_bn(int M, int N, int num_sms)
@@ -156,6 +180,12 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
         if (e != cudaSuccess) return cuda_fail(e);
     }
     const int walkers = pair ? max_pairs : di.num_sms;
+    p.epoch = 0; p.signals = nullptr;
+    choose_split(p, walkers);
+    if (p.split_parts > 1) {
+        const cudaError_t es = mpg::gemm_split_signals(&p.epoch, &p.signals);
+        if (es != cudaSuccess) return cuda_fail(es);
+    }
     const int grid = (p.num_tiles < walkers ? p.num_tiles : walkers) * (pair ? 2 : 1);
     const cudaError_t e = mpg::launch_gemm(bn, pair, tm_a, tm_b, p, grid, stream);
     return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
@@ -295,6 +325,14 @@ int mpgemmfi_set_tile_policy(int policy)
     if (policy != MPGEMMFI_TILES_AUTO && policy != MPGEMMFI_TILES_SINGLE && policy != MPGEMMFI_TILES_PAIR)
         return MPGEMMFI_ERR_ARG;
     g_tile_policy = policy;
+    return MPGEMMFI_OK;
+}
+
+int mpgemmfi_set_split_policy(int policy)
+{
+    if (policy != MPGEMMFI_SPLIT_AUTO && policy != MPGEMMFI_SPLIT_OFF && policy != MPGEMMFI_SPLIT_ON)
+        return MPGEMMFI_ERR_ARG;
+    g_split_policy = policy;
     return MPGEMMFI_OK;
 }
 

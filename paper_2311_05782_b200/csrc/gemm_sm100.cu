@@ -20,7 +20,19 @@
 // both CTAs' shared memory and fill both CTAs' TMEM, and each CTA runs the epilogue of its own
 // 128 rows. Halving the Bt bytes each SM has to pull per MMA is what lifts the main loop off
 // the SM's shared-memory fill rate.
+//
+// Tile schedule. Tiles are dealt out round-robin to the tile walkers (CTAs or CTA pairs). When the
+// last round would leave many walkers idle, its tiles are cut along K into parts that different
+// walkers run at different times: the walker of part 0 runs it before its full tiles and leaves the
+// raw accumulators in the tile's place in C; the walker of the last part runs after its full tiles,
+// loads those accumulators back into TMEM and carries on with the next k-tile, so every element
+// still sees one FP32 accumulation in increasing k, bit for bit the one of an uncut tile, and an
+// accumulator site still meets the running sum. Parts in between sit after the walker's g-th full
+// tile. A part's hand-over is one flag word per epilogue warp in a per-launch slot of a static
+// device array; the waits on it are bounded like every other wait here.
+#include <atomic>
 #include <cstdint>
+#include <type_traits>
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -33,6 +45,8 @@ namespace mpg {
 namespace {
 
 constexpr uint32_t NONE = 0xFFFFFFFFu;
+// check modes of the epilogue: none, BoundCheck (detect), BoundCheck + correction, output-level range check
+enum { EPI_PLAIN = 0, EPI_BOUND = 1, EPI_BOUND_CORRECT = 2, EPI_RANGE = 3 };
 constexpr int BM = 128;
 constexpr int NUM_THREADS = 384;     // 4 control warps + 8 epilogue warps
 constexpr int EPI_WARPS = 8;
@@ -60,6 +74,7 @@ struct alignas(16) Control {
     uint64_t acc_empty[2];
     uint64_t pause_full;
     uint64_t pause_done;
+    uint64_t acc_loaded;      // the accumulators of a continued tile part are back in TMEM
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t site_count;
@@ -285,24 +300,156 @@ __device__ __forceinline__ uint32_t tile_number(const GemmParams &p, uint32_t tm
     return band * (uint32_t)p.group_m * (uint32_t)p.tiles_n + tn * rows + (tm - band * (uint32_t)p.group_m);
 }
 
+// One piece of work of a tile walker: k-tiles [kt0, kt1) of one output tile. `load`: the
+// accumulators of k-tiles [0, kt0) come from C (left there by the walker of the previous part);
+// `save`: the tile is not finished here, the raw accumulators go to C for the next part.
+struct Segment {
+    uint32_t tile, kt0, kt1, part;
+    bool load, save;
+};
+
+// i-th segment of walker `gid`. Plain schedule (split_parts <= 1): tiles gid, gid + groups, ...,
+// each whole. Split schedule: `full_rounds` whole tiles dealt out the same way, and the
+// `left_tiles` tiles of the last round cut into `split_parts` equal runs of k-tiles; part g of
+// left-over tile j belongs to walker g * left_tiles + j, which runs it after its g-th whole tile
+// (the last part: after all of them), so that part g is finished long before part g + 1 starts.
+__device__ __forceinline__ bool get_segment(const GemmParams &p, uint32_t gid, uint32_t groups, uint32_t i, Segment &sg)
+{
+    const uint32_t nkt = (uint32_t)p.num_kt;
+    if (p.split_parts <= 1) {
+        sg.tile = gid + i * groups;
+        sg.kt0 = 0; sg.kt1 = nkt; sg.part = 0; sg.load = false; sg.save = false;
+        return sg.tile < (uint32_t)p.num_tiles;
+    }
+    const uint32_t left = (uint32_t)p.left_tiles, parts = (uint32_t)p.split_parts, rounds = (uint32_t)p.full_rounds;
+    const uint32_t g = gid / left;
+    const bool has_part = g < parts;
+    const uint32_t pos = g + 1 < parts ? g : rounds;
+    if (i >= rounds + (has_part ? 1u : 0u)) return false;
+    if (has_part && i == pos) {
+        sg.tile = groups * rounds + gid % left;
+        sg.kt0 = g * nkt / parts; sg.kt1 = (g + 1) * nkt / parts; sg.part = g;
+        sg.load = g > 0; sg.save = g + 1 < parts;
+        return true;
+    }
+    sg.tile = gid + ((has_part && i > pos) ? i - 1 : i) * groups;
+    sg.kt0 = 0; sg.kt1 = nkt; sg.part = 0; sg.load = false; sg.save = false;
+    return true;
+}
+
+// does walker `gid` run tile t, whole or in part?
+__device__ __forceinline__ bool walker_has_tile(const GemmParams &p, uint32_t t, uint32_t gid, uint32_t groups)
+{
+    if (p.split_parts > 1 && t >= groups * (uint32_t)p.full_rounds) {
+        const uint32_t j = t - groups * (uint32_t)p.full_rounds;
+        return gid % (uint32_t)p.left_tiles == j && gid / (uint32_t)p.left_tiles < (uint32_t)p.split_parts;
+    }
+    return t % groups == gid;
+}
+
 // Does a site touch a tile walked by tile-walker `gid` of `groups` (a CTA, or a CTA pair)?
-// Tiles are TM x BN and are dealt out round-robin by tile number.
+// Tiles are TM x BN.
 template <int TM, int BN>
 __device__ bool site_touches_group(const mpgemmfi_site &s, const GemmParams &p, uint32_t gid, uint32_t groups)
 {
     if (s.kind == MPGEMMFI_SITE_A) {
         const uint32_t tm = s.row / TM;
         for (uint32_t tn = 0; tn < (uint32_t)p.tiles_n; ++tn)
-            if (tile_number(p, tm, tn) % groups == gid) return true;
+            if (walker_has_tile(p, tile_number(p, tm, tn), gid, groups)) return true;
         return false;
     }
     if (s.kind == MPGEMMFI_SITE_B) {
         const uint32_t tn = s.col / BN;
         for (uint32_t tm = 0; tm < (uint32_t)p.tiles_m; ++tm)
-            if (tile_number(p, tm, tn) % groups == gid) return true;
+            if (walker_has_tile(p, tile_number(p, tm, tn), gid, groups)) return true;
         return false;
     }
-    return tile_number(p, s.row / TM, s.col / BN) % groups == gid;
+    return walker_has_tile(p, tile_number(p, s.row / TM, s.col / BN), gid, groups);
+}
+
+// Hand-over of a tile part between walkers: one word per epilogue warp of the walker.
+__device__ __forceinline__ void signal_store_release(uint32_t *ptr, uint32_t v)
+{
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ uint32_t signal_load_acquire(const uint32_t *ptr)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
+
+// bounded wait for *ptr == want; same give-up rules as mbar_wait
+__device__ __forceinline__ bool signal_wait(const uint32_t *ptr, uint32_t want, volatile uint32_t *abort_flag,
+                                            uint64_t limit_ns = 4000000000ull)
+{
+    if (signal_load_acquire(ptr) == want) return true;
+    uint64_t t0 = 0;
+    for (uint32_t it = 1;; ++it) {
+        if (signal_load_acquire(ptr) == want) return true;
+        __nanosleep(64);
+        if ((it & 0x3Fu) == 0) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) { *abort_flag = 1; return false; }
+        }
+    }
+}
+
+// One epilogue warp, for a continued tile part that its walker runs later: wait for the warp of the
+// previous part's walker that owns the same rows and columns (hand-over word *sig == want), then copy
+// rows row0..row0+31, columns col0..col0+32*pieces-1 of the accumulators it left in C back into TMEM
+// (this warp's lanes, columns from t_dst on). `park` is the warp's 2 KB of shared-memory staging.
+// The store transpose of the epilogue run backwards: every load instruction reads whole 128-byte rows
+// of C (lane l: 16-byte piece l % 8 of rows l / 8 + 4 it) and parks them in shared memory, then the
+// threads of one half-warp pick up their own rows. (One 128-byte row per thread instead: 11 us per
+// tile, during which the main loop next to it stood still.) Returns false when the wait gave up.
+__device__ __forceinline__ bool load_partial(const float *C, uint32_t M, uint32_t N, const uint32_t *sig, uint32_t want,
+                                             volatile uint32_t *abort_flag, uint32_t row0, uint32_t col0, int pieces,
+                                             uint32_t t_dst, uint8_t *park, int lane)
+{
+    bool got = true;
+    if (lane == 0) got = signal_wait(sig, want, abort_flag);
+    got = __shfl_sync(0xFFFFFFFFu, got, 0);
+    if (!got) return false;
+    __threadfence();
+    const uint32_t j = (uint32_t)lane & 7u;
+#pragma unroll 1
+    for (int i = 0; i < pieces; ++i) {
+        const uint32_t col = col0 + (uint32_t)(32 * i) + 4 * j;
+        uint32_t v[32];
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            uint4 x[4];
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+                const uint32_t grow = row0 + (uint32_t)(16 * half + 4 * it) + ((uint32_t)lane >> 3);
+                x[it] = make_uint4(0u, 0u, 0u, 0u);
+                if (grow < M && col < N) x[it] = __ldcg(reinterpret_cast<const uint4 *>(C + (size_t)grow * N + col));
+            }
+            __syncwarp();                               // the rows parked before have been picked up
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+                const uint32_t r = (uint32_t)(4 * it) + ((uint32_t)lane >> 3);
+                *reinterpret_cast<uint4 *>(park + r * 128 + ((j ^ (r & 7u)) << 4)) = x[it];
+            }
+            __syncwarp();
+            if ((lane >> 4) == half) {
+                const uint8_t *srow = park + (lane & 15) * 128;
+#pragma unroll
+                for (int jj = 0; jj < 8; ++jj) {
+                    const uint4 y = *reinterpret_cast<const uint4 *>(srow + ((jj ^ (lane & 7)) << 4));
+                    v[4 * jj] = y.x; v[4 * jj + 1] = y.y; v[4 * jj + 2] = y.z; v[4 * jj + 3] = y.w;
+                }
+            }
+        }
+        tmem_st_32x32(t_dst + (uint32_t)(i * 32), v);
+    }
+    __syncwarp();
+    tmem_wait_st();
+    return true;
 }
 
 // Slice of the site table that one warp examines when the CTA builds its list.
@@ -407,7 +554,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     volatile uint32_t *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t num_kt = (uint32_t)p.num_kt;
     const uint32_t rank = kPair ? cluster_cta_rank() : 0u;          // 0 = leader of the pair
     const uint32_t gid = kPair ? blockIdx.x >> 1 : blockIdx.x;      // tile walker id
     const uint32_t groups = kPair ? gridDim.x >> 1 : gridDim.x;
@@ -429,6 +575,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->acc_full[s]), 1); mbar_init(smem_u32(&ctl->acc_empty[s]), EPI_ARRIVALS); }
         mbar_init(smem_u32(&ctl->pause_full), 1);
         mbar_init(smem_u32(&ctl->pause_done), EPI_ARRIVALS);
+        mbar_init(smem_u32(&ctl->acc_loaded), EPI_ARRIVALS);
         ctl->abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tm_a);
@@ -458,6 +605,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     // barriers of the leader CTA that this CTA's warps arrive on
     const uint32_t lead_acc_empty0 = kPair ? map_to_cta(smem_u32(&ctl->acc_empty[0]), 0) : smem_u32(&ctl->acc_empty[0]);
     const uint32_t lead_pause_done = kPair ? map_to_cta(smem_u32(&ctl->pause_done), 0) : smem_u32(&ctl->pause_done);
+    const uint32_t lead_acc_loaded = kPair ? map_to_cta(smem_u32(&ctl->acc_loaded), 0) : smem_u32(&ctl->acc_loaded);
+    Segment sg;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -468,11 +617,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         uint32_t stage = 0, phase = 0, armed = 0, armed_parity = 0;
         const uint32_t lead_full0 = kPair ? map_to_cta(smem_u32(&ctl->full[0]), 0) : 0u;
         bool ok = true;
-        for (uint32_t t = gid; ok && t < (uint32_t)p.num_tiles; t += groups) {
-            set_tile(t);
+        for (uint32_t si = 0; ok && get_segment(p, gid, groups, si, sg); ++si) {
+            set_tile(sg.tile);
             uint32_t next_op = NONE;
-            if (kPair && !leader && has_sites) next_op = scan_next_operand(tc, 0, lane);
-            for (uint32_t kt = 0; kt < num_kt; ++kt) {
+            if (kPair && !leader && has_sites) next_op = scan_next_operand(tc, sg.kt0, lane);
+            for (uint32_t kt = sg.kt0; kt < sg.kt1; ++kt) {
                 const bool own_barrier = !kPair || leader || kt == next_op;
                 if (kPair && kt == next_op) next_op = scan_next_operand(tc, kt + 1, lane);
                 if (lane == 0) {
@@ -511,14 +660,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         // ------------------------------------------------------------ pair mode, non-leader CTA: no MMAs to
         // issue; only the stages that carry one of this CTA's operand sites need attention
         if (has_sites) {
-            uint32_t lt = 0, own_phase = 0;     // own_phase: bit s = parity of this CTA's full[s]
+            uint32_t steps_before = 0, own_phase = 0;     // own_phase: bit s = parity of this CTA's full[s]
             bool ok = true;
             const uint32_t lead_full0 = map_to_cta(smem_u32(&ctl->full[0]), 0);
-            for (uint32_t t = gid; ok && t < (uint32_t)p.num_tiles; t += groups, ++lt) {
-                set_tile(t);
-                uint32_t kt = scan_next_operand(tc, 0, lane);
-                while (kt != NONE) {
-                    const uint32_t g = lt * num_kt + kt, stage = g % STAGES;
+            for (uint32_t si = 0; ok && get_segment(p, gid, groups, si, sg); steps_before += sg.kt1 - sg.kt0, ++si) {
+                set_tile(sg.tile);
+                uint32_t kt = scan_next_operand(tc, sg.kt0, lane);
+                while (kt < sg.kt1) {          // NONE is larger than any k-tile
+                    const uint32_t g = steps_before + (kt - sg.kt0), stage = g % STAGES;
                     ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->full[stage]), (own_phase >> stage) & 1u, abort_flag));
                     if (!ok) break;
                     own_phase ^= 1u << stage;
@@ -536,18 +685,54 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         const uint32_t idesc = umma_instr_desc((uint32_t)p.dtype, TM, BN);
-        uint32_t stage = 0, phase = 0, lt = 0, pause_phase = 0;
+        uint32_t stage = 0, phase = 0, pause_phase = 0, loaded_phase = 0;
         bool ok = true;
-        for (uint32_t t = gid; ok && t < (uint32_t)p.num_tiles; t += groups, ++lt) {
+        for (uint32_t lt = 0; ok && get_segment(p, gid, groups, lt, sg); ++lt) {
             const uint32_t as = lt & 1u, ap = (lt >> 1) & 1u;
-            set_tile(t);
+            set_tile(sg.tile);
             uint32_t next_op = NONE, next_b = NONE;
-            if (has_sites) { next_op = scan_next_operand(tc, 0, lane); next_b = scan_next_boundary(tc, 1, lane); }
+            if (has_sites) { next_op = scan_next_operand(tc, sg.kt0, lane); next_b = scan_next_boundary(tc, sg.kt0 + 1, lane); }
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_empty[as]), ap ^ 1u, abort_flag));
             if (!ok) break;
+            if (sg.load) {
+                // continued tile: the epilogue warps put the earlier k-tiles' accumulators back first
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_loaded), loaded_phase, abort_flag));
+                if (!ok) break;
+                loaded_phase ^= 1u;
+            }
             tc_fence_after_sync();
             const uint32_t d_tmem = tmem_base + as * BN;
-            for (uint32_t kt = 0; kt < num_kt; ++kt) {
+            const uint32_t fresh_kt = sg.load ? NONE : sg.kt0;      // the k-tile whose first MMA overwrites the accumulator
+            if (next_op >= sg.kt1 && next_b > sg.kt1) {
+                // no operand, accumulator or term site in these k-tiles (the usual case): one thread
+                // runs the whole loop, with no warp-wide step in it, so that issuing a k-tile's MMAs
+                // takes less time than the tensor core needs to run them
+                if (lane == 0) {
+                    const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+                    const uint64_t desc0 = umma_smem_desc_sw128(smem_u32(smem));
+                    uint32_t accumulate = sg.load ? 1u : 0u;
+                    for (uint32_t kt = sg.kt0; kt < sg.kt1; ++kt) {
+                        if (!mbar_wait(full0 + stage * 8u, phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        // the address field counts 16-byte units: stage s starts s * STAGE_BYTES / 16 further on
+                        const uint64_t a_desc = desc0 + (uint64_t)(stage * (uint32_t)(C::STAGE_BYTES >> 4));
+                        const uint64_t b_desc = a_desc + (uint64_t)(C::A_BYTES >> 4);
+#pragma unroll
+                        for (uint32_t k = 0; k < 4; ++k) {
+                            if constexpr (kPair) umma_ss_pair<kTF32>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, accumulate);
+                            else umma_ss<kTF32>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, accumulate);
+                            accumulate = 1u;
+                        }
+                        if constexpr (kPair) umma_commit_pair(empty0 + stage * 8u, 3);
+                        else umma_commit(empty0 + stage * 8u);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                }
+                ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                stage = __shfl_sync(0xFFFFFFFFu, stage, 0);
+                phase = __shfl_sync(0xFFFFFFFFu, phase, 0);
+            } else
+            for (uint32_t kt = sg.kt0; kt < sg.kt1; ++kt) {
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag));
                 if (!ok) break;
                 tc_fence_after_sync();
@@ -565,8 +750,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     const uint64_t b_desc = umma_smem_desc_sw128(smem_u32(sa + C::A_BYTES));
 #pragma unroll
                     for (uint32_t k = 0; k < 4; ++k) {   // 4 x 32 bytes along K inside the swizzle row
-                        if constexpr (kPair) umma_ss_pair<kTF32>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kt | k) != 0 ? 1u : 0u);
-                        else umma_ss<kTF32>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kt | k) != 0 ? 1u : 0u);
+                        const uint32_t accumulate = (kt == fresh_kt && k == 0) ? 0u : 1u;
+                        if constexpr (kPair) umma_ss_pair<kTF32>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, accumulate);
+                        else umma_ss<kTF32>(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, accumulate);
                     }
                     if constexpr (kPair) umma_commit_pair(smem_u32(&ctl->empty[stage]), 3);
                     else umma_commit(smem_u32(&ctl->empty[stage]));
@@ -599,23 +785,53 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         const int q = warp & 3;               // TMEM lane quarter this warp may access
         const int h = (warp - 4) >> 2;        // column half of the tile this warp handles
         const int tech = p.detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK;
-        const bool do_bound = tech == MPGEMMFI_DETECT_BOUNDCHECK;
-        const bool do_range = (p.detect_mode & MPGEMMFI_OUTPUT_RANGE) && p.exp_a != nullptr &&
-                              (tech == MPGEMMFI_DETECT_RANGE_MAX || tech == MPGEMMFI_DETECT_RANGE_FLIP);
+        const bool want_bound = tech == MPGEMMFI_DETECT_BOUNDCHECK;
+        const bool want_range = (p.detect_mode & MPGEMMFI_OUTPUT_RANGE) && p.exp_a != nullptr &&
+                                (tech == MPGEMMFI_DETECT_RANGE_MAX || tech == MPGEMMFI_DETECT_RANGE_FLIP);
         const bool range_flip = tech == MPGEMMFI_DETECT_RANGE_FLIP;
-        const bool do_corr = (do_bound || do_range) && (p.detect_mode & MPGEMMFI_CORRECT);
-        uint32_t lt = 0, pause_phase = 0, n_det = 0;
+        const bool want_corr = (want_bound || want_range) && (p.detect_mode & MPGEMMFI_CORRECT);
+        // The per-element work of a tile is compiled once per check mode (EPI_*), so that the 32-element
+        // loops carry no mode tests: left to itself the compiler does not always pull them out of the
+        // tile loop (when it did not, a launch ran a quarter more instructions).
+        const int epi_mode = want_range ? EPI_RANGE : (want_bound ? (want_corr ? EPI_BOUND_CORRECT : EPI_BOUND) : EPI_PLAIN);
+        uint32_t pause_phase = 0, n_det = 0;
         uint32_t *bitmap = p.flags ? p.flags + MPGEMMFI_HEADER_WORDS + 4 * (size_t)p.n_faults : nullptr;
         uint8_t *my_out = stage_out + (warp - 4) * (16 * 128);
+        constexpr int MY_PIECES = BN / 64;          // 32-column pieces per warp (half the tile's columns)
+        const int first = h * MY_PIECES;
+        // hand-over words of this warp for left-over tile j: signals[j * 16 + my_signal]
+        const uint32_t my_signal = rank * EPI_WARPS + (uint32_t)(warp - 4);
+        const uint32_t first_left = groups * (uint32_t)p.full_rounds;
         bool ok = true;
-        for (uint32_t t = gid; ok && t < (uint32_t)p.num_tiles; t += groups, ++lt) {
+        for (uint32_t lt = 0; ok && get_segment(p, gid, groups, lt, sg); ++lt) {
             const uint32_t as = lt & 1u, ap = (lt >> 1) & 1u;
-            set_tile(t);
+            if (p.split_parts > 1) {
+                // the other TMEM buffer is free (this warp has read its share of the segment before this
+                // one): if the next segment continues a tile, fetch its accumulators while this one runs
+                Segment nx;
+                if (get_segment(p, gid, groups, lt + 1, nx) && nx.load) {
+                    uint32_t tm, tn;
+                    tile_coords(p, nx.tile, tm, tn);
+                    const uint32_t *sig = p.signals + (size_t)(nx.tile - first_left) * 16 + my_signal;
+                    const uint32_t t_dst = tmem_base + ((lt + 1) & 1u) * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)(first * 32);
+                    ok = load_partial(p.C, (uint32_t)p.M, (uint32_t)p.N, sig, (p.epoch << 3) | nx.part, abort_flag,
+                                      tm * TM + rank * BM + (uint32_t)(q * 32), tn * BN + (uint32_t)(first * 32), MY_PIECES,
+                                      t_dst, my_out, lane);
+                    if (!ok) break;
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if constexpr (kPair) mbar_arrive_cluster(lead_acc_loaded);
+                        else mbar_arrive(lead_acc_loaded);
+                    }
+                }
+            }
+            set_tile(sg.tile);
             const uint32_t tmem_acc = tmem_base + as * BN;
             bool tile_has_out = false;
             if (has_sites) {
-                uint32_t b = scan_next_boundary(tc, 1, lane);
-                while (b != NONE) {
+                uint32_t b = scan_next_boundary(tc, sg.kt0 + 1, lane);
+                while (b <= sg.kt1) {          // boundaries of this segment's k-tiles (NONE is larger than any)
                     ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->pause_full), pause_phase, abort_flag));
                     if (!ok) break;
                     pause_phase ^= 1u;
@@ -630,7 +846,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     b = scan_next_boundary(tc, b + 1, lane);
                 }
                 if (!ok) break;
-                tile_has_out = scan_has_out(tc, lane);
+                tile_has_out = !sg.save && scan_has_out(tc, lane);
             }
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_full[as]), ap, abort_flag));
             if (!ok) break;
@@ -639,48 +855,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             const uint32_t row = tc.m0 + (uint32_t)(q * 32 + lane);
             const uint32_t row0 = tc.m0 + (uint32_t)(q * 32);
             const bool row_ok = row < (uint32_t)p.M;
-            const uint32_t row_e = (do_range && row_ok) ? __ldg(p.exp_a + row) : 0u;
             float *crow = p.C + (size_t)row * p.N;
-            const uint32_t t_lane = tmem_acc + ((uint32_t)(q * 32) << 16);
-            constexpr int MY_PIECES = BN / 64;          // 32-column pieces per warp (half the tile's columns)
-            const int first = h * MY_PIECES;
-            uint32_t flagw[MY_PIECES];
+            const uint32_t t_first = tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(first * 32);
 
-            // One 32-column piece of this thread's row: output sites, check, flags, store.
-            auto finish_piece = [&](uint32_t (&v)[32], int i) {
-                const uint32_t c0 = tc.n0 + (uint32_t)((first + i) * 32);
-                // output-level range check: this lane fetches the exponent maximum of column c0 + lane early
-                uint32_t col_e = 0;
-                if (do_range && c0 + (uint32_t)lane < (uint32_t)p.N) col_e = __ldg(p.exp_b + c0 + lane);
-                if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 0);
-                uint32_t fw = 0;
-                if (do_range) {
-                    const int row_part = (int)row_e - 126 + p.log2_k;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int bound = min(255, max(0, row_part + (int)__shfl_sync(0xFFFFFFFFu, col_e, j)));
-                        const bool det = (int)((v[j] >> 23) & 0xFFu) > bound;
-                        if (det) {
-                            fw |= 1u << j;
-                            if (do_corr) v[j] = range_flip ? rangecheck_flip(v[j], bound) : rangecheck_max(v[j], bound);
-                        }
-                    }
-                    if (c0 + 32 > (uint32_t)p.N) fw &= c0 < (uint32_t)p.N ? (1u << ((uint32_t)p.N - c0)) - 1u : 0u;
-                }
-                if (do_bound) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        // exponent field >= 0x90 <=> not (|value| < 131072); NaN compares false, so it is caught
-                        const bool det = !(fabsf(bits_f32(v[j])) < 131072.0f);
-                        if (det) fw |= 1u << j;
-                        if (do_corr && det) v[j] = boundcheck_clear(v[j]);
-                    }
-                    // columns past N are not part of C (their zero-filled Bt rows still give NaN against an
-                    // Inf or NaN in A): their flag bits stay 0
-                    if (c0 + 32 > (uint32_t)p.N) fw &= c0 < (uint32_t)p.N ? (1u << ((uint32_t)p.N - c0)) - 1u : 0u;
-                }
-                if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 1);
-                flagw[i] = fw;
+            // stores of one 32-column piece (this thread's row, columns c0..c0+31) to C
+            auto store_piece = [&](uint32_t (&v)[32], uint32_t c0) {
                 if (p.c_vec_ok) {
                     // Transpose through shared memory so that every store instruction writes whole
                     // 128-byte rows, 16 rows at a time: threads of one half-warp park their rows
@@ -725,43 +904,114 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 }
             };
 
-            // software pipeline: the TMEM read of the next piece is in flight while this one is finished
-            uint32_t va[32], vb[32];
-            const uint32_t t_first = t_lane + (uint32_t)(first * 32);
-            tmem_ld_32x32(t_first, va);
-#pragma unroll
-            for (int i = 0; i < MY_PIECES; i += 2) {
-                tmem_wait_ld();
-                if (i + 1 < MY_PIECES) tmem_ld_32x32(t_first + (uint32_t)((i + 1) * 32), vb);
-                else release_acc();
-                finish_piece(va, i);
-                if (i + 1 < MY_PIECES) {
+            if (sg.save) {
+                // unfinished tile: the raw accumulators go to the tile's place in C (no output site, no check),
+                // then the walker of the next part is told that this warp's share is there
+#pragma unroll 1
+                for (int i = 0; i < MY_PIECES; ++i) {
+                    uint32_t raw[32];
+                    tmem_ld_32x32(t_first + (uint32_t)(i * 32), raw);
                     tmem_wait_ld();
-                    if (i + 2 < MY_PIECES) tmem_ld_32x32(t_first + (uint32_t)((i + 2) * 32), va);
-                    else release_acc();
-                    finish_piece(vb, i + 1);
+                    store_piece(raw, tc.n0 + (uint32_t)((first + i) * 32));
                 }
+                release_acc();
+                __threadfence();
+                __syncwarp();
+                if (lane == 0)
+                    signal_store_release(p.signals + (size_t)(sg.tile - first_left) * 16 + my_signal, (p.epoch << 3) | (sg.part + 1u));
+                continue;
             }
-            if (bitmap && row_ok) {
-                const uint32_t w0 = tc.n0 / 32 + (uint32_t)first;
-                uint32_t *frow = bitmap + (size_t)row * p.wpr + w0;
-                if (MY_PIECES == 4 && (p.wpr & 3) == 0) {       // this thread's 4 words are 16-byte aligned
-                    if (w0 < (uint32_t)p.wpr)
-                    *reinterpret_cast<uint4 *>(frow) = make_uint4(flagw[0], flagw[MY_PIECES > 1 ? 1 : 0],
-                                                                   flagw[MY_PIECES > 2 ? 2 : 0], flagw[MY_PIECES > 3 ? 3 : 0]);
-                } else {
+
+            // The finished tile under check mode kMode (a compile-time constant inside).
+            auto finish_tile = [&](auto mode_tag) {
+                constexpr int kMode = decltype(mode_tag)::value;
+                constexpr bool do_bound = kMode == EPI_BOUND || kMode == EPI_BOUND_CORRECT;
+                constexpr bool do_range = kMode == EPI_RANGE;
+                const bool do_corr = kMode == EPI_BOUND_CORRECT || (kMode == EPI_RANGE && want_corr);
+                const uint32_t row_e = (do_range && row_ok) ? __ldg(p.exp_a + row) : 0u;
+                uint32_t flagw[MY_PIECES];
+
+                // One 32-column piece of this thread's row: output sites, check, flags, store.
+                auto finish_piece = [&](uint32_t (&v)[32], int i) {
+                    const uint32_t c0 = tc.n0 + (uint32_t)((first + i) * 32);
+                    // output-level range check: this lane fetches the exponent maximum of column c0 + lane early
+                    uint32_t col_e = 0;
+                    if (do_range && c0 + (uint32_t)lane < (uint32_t)p.N) col_e = __ldg(p.exp_b + c0 + lane);
+                    if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 0);
+                    uint32_t fw = 0;
+                    if constexpr (do_range) {
+                        const int row_part = (int)row_e - 126 + p.log2_k;
 #pragma unroll
-                    for (int i = 0; i < MY_PIECES; ++i)
-                        if (w0 + i < (uint32_t)p.wpr) frow[i] = flagw[i];
+                        for (int j = 0; j < 32; ++j) {
+                            const int bound = min(255, max(0, row_part + (int)__shfl_sync(0xFFFFFFFFu, col_e, j)));
+                            const bool det = (int)((v[j] >> 23) & 0xFFu) > bound;
+                            if (det) {
+                                fw |= 1u << j;
+                                if (do_corr) v[j] = range_flip ? rangecheck_flip(v[j], bound) : rangecheck_max(v[j], bound);
+                            }
+                        }
+                        if (c0 + 32 > (uint32_t)p.N) fw &= c0 < (uint32_t)p.N ? (1u << ((uint32_t)p.N - c0)) - 1u : 0u;
+                    }
+                    if constexpr (do_bound) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            // exponent field >= 0x90 <=> not (|value| < 131072); NaN compares false, so it is caught
+                            const bool det = !(fabsf(bits_f32(v[j])) < 131072.0f);
+                            if (det) fw |= 1u << j;
+                            if (kMode == EPI_BOUND_CORRECT && det) v[j] = boundcheck_clear(v[j]);
+                        }
+                        // columns past N are not part of C (their zero-filled Bt rows still give NaN against an
+                        // Inf or NaN in A): their flag bits stay 0
+                        if (c0 + 32 > (uint32_t)p.N) fw &= c0 < (uint32_t)p.N ? (1u << ((uint32_t)p.N - c0)) - 1u : 0u;
+                    }
+                    if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 1);
+                    flagw[i] = fw;
+                    store_piece(v, c0);
+                };
+
+                // software pipeline: the TMEM read of the next piece is in flight while this one is finished
+                uint32_t va[32], vb[32];
+                tmem_ld_32x32(t_first, va);
+#pragma unroll
+                for (int i = 0; i < MY_PIECES; i += 2) {
+                    tmem_wait_ld();
+                    if (i + 1 < MY_PIECES) tmem_ld_32x32(t_first + (uint32_t)((i + 1) * 32), vb);
+                    else release_acc();
+                    finish_piece(va, i);
+                    if (i + 1 < MY_PIECES) {
+                        tmem_wait_ld();
+                        if (i + 2 < MY_PIECES) tmem_ld_32x32(t_first + (uint32_t)((i + 2) * 32), va);
+                        else release_acc();
+                        finish_piece(vb, i + 1);
+                    }
                 }
+                if (bitmap && row_ok) {
+                    const uint32_t w0 = tc.n0 / 32 + (uint32_t)first;
+                    uint32_t *frow = bitmap + (size_t)row * p.wpr + w0;
+                    if (MY_PIECES == 4 && (p.wpr & 3) == 0) {       // this thread's 4 words are 16-byte aligned
+                        if (w0 < (uint32_t)p.wpr)
+                            *reinterpret_cast<uint4 *>(frow) = make_uint4(flagw[0], flagw[MY_PIECES > 1 ? 1 : 0],
+                                                                           flagw[MY_PIECES > 2 ? 2 : 0], flagw[MY_PIECES > 3 ? 3 : 0]);
+                    } else {
 #pragma unroll
-                for (int i = 0; i < MY_PIECES; ++i) n_det += __popc(flagw[i]);
+                        for (int i = 0; i < MY_PIECES; ++i)
+                            if (w0 + i < (uint32_t)p.wpr) frow[i] = flagw[i];
+                    }
+#pragma unroll
+                    for (int i = 0; i < MY_PIECES; ++i) n_det += __popc(flagw[i]);
+                }
+            };
+            switch (epi_mode) {
+            case EPI_PLAIN: finish_tile(std::integral_constant<int, EPI_PLAIN>{}); break;
+            case EPI_BOUND: finish_tile(std::integral_constant<int, EPI_BOUND>{}); break;
+            case EPI_BOUND_CORRECT: finish_tile(std::integral_constant<int, EPI_BOUND_CORRECT>{}); break;
+            default: finish_tile(std::integral_constant<int, EPI_RANGE>{}); break;
             }
         }
         n_det = __reduce_add_sync(0xFFFFFFFFu, n_det);
         if (lane == 0 && n_det && p.flags) {
             atomicAdd(&p.flags[1], n_det);
-            if (do_corr) atomicAdd(&p.flags[2], n_det);
+            if (want_corr) atomicAdd(&p.flags[2], n_det);
         }
     }
 
@@ -774,6 +1024,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         else tmem_dealloc(tmem_base, C::TMEM_COLS);
     }
     if (threadIdx.x == 0 && ctl->abort_flag && p.flags) atomicOr(&p.flags[0], MPGEMMFI_STATUS_WAIT_LIMIT);
+    if (threadIdx.x == 0 && blockIdx.x == 0 && p.flags && p.split_parts > 1) p.flags[5] = (uint32_t)p.split_parts;
 }
 
 template <int BN, bool kTF32, bool kPair>
@@ -835,6 +1086,30 @@ int gemm_max_resident_pairs(int dtype)
         cache[dev][tf] = n > 0 ? n : -1;
     }
     return cache[dev][tf] > 0 ? cache[dev][tf] : 0;
+}
+
+namespace {
+__device__ uint32_t g_split_signals[SPLIT_SIGNAL_SLOTS][SPLIT_SIGNAL_WORDS];
+}
+
+cudaError_t gemm_split_signals(uint32_t *epoch, uint32_t **signals)
+{
+    static uint32_t *base[64] = {};
+    static std::atomic<uint32_t> counter{0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!base[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_split_signals);
+        if (e != cudaSuccess) return e;
+        base[dev] = static_cast<uint32_t *>(ptr);
+    }
+    const uint32_t n = counter.fetch_add(1u) + 1u;
+    *epoch = n & 0x1FFFFFFFu ? n & 0x1FFFFFFFu : 1u;     // 29 bits (3 more carry the part number), never 0
+    *signals = base[dev] + (size_t)(n % SPLIT_SIGNAL_SLOTS) * SPLIT_SIGNAL_WORDS;
+    return cudaSuccess;
 }
 
 int gemm_stage_count(int bn, bool pair)

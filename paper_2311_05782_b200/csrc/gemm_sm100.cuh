@@ -25,7 +25,23 @@ struct GemmParams {
     const uint32_t *exp_a;
     const uint32_t *exp_b;
     int log2_k;
+    // Split schedule of the last round of tiles (split_parts <= 1: off). The tile walkers first share
+    // out `full_rounds` whole tiles each; the `left_tiles` tiles that remain are cut along K into
+    // `split_parts` parts run by different walkers, the accumulators travelling through C.
+    int split_parts, full_rounds, left_tiles;
+    uint32_t epoch;        // tag of this launch in the hand-over words
+    uint32_t *signals;     // SPLIT_SIGNAL_WORDS hand-over words of this launch (device memory)
 };
+
+// hand-over words one launch can use: 16 per left-over tile, fewer left-over tiles than walkers
+constexpr int SPLIT_MAX_WALKERS = 160;
+constexpr int SPLIT_SIGNAL_WORDS = SPLIT_MAX_WALKERS * 16;
+
+// Gives a launch that uses the split schedule its tag and its hand-over words: a slot of a static
+// device array, slots handed out in turn (a slot comes round again after SPLIT_SIGNAL_SLOTS launches;
+// the tag keeps a launch from reading what an earlier one left there).
+constexpr int SPLIT_SIGNAL_SLOTS = 16;
+cudaError_t gemm_split_signals(uint32_t *epoch, uint32_t **signals);
 
 // shared-memory pipeline depth used for an output tile that is bn columns wide
 int gemm_stage_count(int bn, bool pair);

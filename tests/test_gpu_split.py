@@ -1,0 +1,111 @@
+"""GPU tests of the split schedule of the last round of tiles (mpgemmfi_set_split_policy).
+
+A cut tile must come out bit for bit as the whole tile does (same accumulation order, sites on the same
+running sums), so the first test compares the two schedules with each other on C, the site log and the
+flags; the second compares the split schedule with the oracle like any other GEMM.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2311_05782_b200 as mpg
+import synth
+from parity import check_gemm_against_oracle, run_gpu_gemm, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def rand_operands(dtype, M, N, K, seed):
+    rng = np.random.default_rng(seed)
+    a = rng.standard_normal((M, K)).astype(np.float32)
+    b = rng.standard_normal((N, K)).astype(np.float32)
+    return synth.round_to_storage(a, dtype), synth.round_to_storage(b, dtype)
+
+
+def site_table(dtype, M, N, K, n, seed):
+    """All five kinds, uniformly placed; accumulator sites on every boundary, so that some fall inside the first
+    run of a cut tile, some on the cut and some after it."""
+    rng = np.random.default_rng(seed)
+    kt = synth.kstep(dtype)
+    s = np.zeros(n, dtype=orc.SITE)
+    s["kind"] = rng.integers(0, 5, n)
+    s["row"] = rng.integers(0, M, n); s["col"] = rng.integers(0, N, n)
+    nb = (K + kt - 1) // kt
+    k_acc = np.minimum(rng.integers(1, nb + 1, n) * kt, K)
+    s["k"] = np.where(s["kind"] == orc.KIND_ACC, k_acc, rng.integers(0, K, n))
+    width = np.where(s["kind"] <= orc.KIND_B, 19 if dtype == orc.TF32 else 16, 32)
+    s["xor_mask"] = [1 << int(rng.integers(0, int(w))) for w in width]
+    return s
+
+
+# (tile policy, dtype, M, N, K): more tiles than tile walkers, few tiles left over for the last round
+#   pair tiles are 256 x 256 on 74 CTA pairs, single tiles 128 x 256 on 148 CTAs (a B200)
+CASES = [
+    (mpg.TILES_PAIR, orc.BF16, 2304, 2300, 520),      # 81 tiles: 7 left over, two runs each, ragged N and K
+    (mpg.TILES_PAIR, orc.FP16, 3328, 2048, 512),      # 104 tiles: 30 left over, two runs
+    (mpg.TILES_PAIR, orc.TF32, 3584, 3072, 264),      # 168 tiles: 20 left over after two rounds, three runs
+    (mpg.TILES_SINGLE, orc.FP16, 1500, 3328, 512),    # 156 tiles of 128 x 256: 8 left over, ragged M
+]
+
+
+@pytest.fixture
+def policies():
+    yield
+    mpg.mpgemmfi_set_tile_policy(mpg.TILES_AUTO)
+    mpg.mpgemmfi_set_split_policy(mpg.SPLIT_AUTO)
+
+
+@pytest.mark.parametrize("case", CASES)
+@pytest.mark.parametrize("mode", [orc.T_NONE, orc.T_BOUND | orc.CORRECT, orc.T_RFLIP | orc.CORRECT])
+def test_split_schedule_is_bit_identical(case, mode, policies):
+    tiles, dtype, M, N, K = case
+    A, Bt = rand_operands(dtype, M, N, K, 77)
+    sites = site_table(dtype, M, N, K, 600, 78)
+    assert mpg.mpgemmfi_set_tile_policy(tiles) == 0
+    out = {}
+    for name, pol in (("whole", mpg.SPLIT_OFF), ("split", mpg.SPLIT_ON)):
+        assert mpg.mpgemmfi_set_split_policy(pol) == 0
+        out[name] = run_gpu_gemm(dtype, A, Bt, sites, mode)
+    Cw, hw, lw, bw = out["whole"]
+    Cs, hs, ls, bs = out["split"]
+    assert hw[5] == 0 and hs[5] >= 2, "the split schedule did not engage on this device"
+    assert hs[0] == hw[0] and not (hs[0] & mpg.STATUS_WAIT_LIMIT)
+    same = Cw.view(np.uint32) == Cs.view(np.uint32)
+    assert same.all(), f"{(~same).sum()} elements differ, first at {np.argwhere(~same)[:5].tolist()}"
+    assert np.array_equal(hw[1:5], hs[1:5])
+    for f in lw.dtype.names:
+        assert np.array_equal(lw[f], ls[f]), f
+    assert np.array_equal(bw, bs)
+
+
+def test_split_schedule_without_flags_buffer(policies):
+    """The plain product (no sites, no check, no flags buffer) under both schedules, twice under the split one."""
+    dtype, M, N, K = orc.BF16, 2304, 2304, 1024
+    A, Bt = rand_operands(dtype, M, N, K, 5)
+    a, b = to_dev(A, dtype), to_dev(Bt, dtype)
+    st = torch.cuda.current_stream().cuda_stream
+    mpg.mpgemmfi_set_tile_policy(mpg.TILES_PAIR)
+    res = []
+    for pol in (mpg.SPLIT_OFF, mpg.SPLIT_ON, mpg.SPLIT_ON):
+        mpg.mpgemmfi_set_split_policy(pol)
+        c = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        assert mpg.mpgemmfi_gemm(dtype, M, N, K, a.data_ptr(), b.data_ptr(), c.data_ptr(), None, 0, 0, None, st) == 0
+        torch.cuda.synchronize()
+        res.append(c.cpu().numpy().view(np.uint32))
+    assert np.array_equal(res[0], res[1]) and np.array_equal(res[0], res[2])
+
+
+@pytest.mark.parametrize("case", CASES[:2] + CASES[3:])
+def test_split_schedule_against_oracle(case, policies):
+    tiles, dtype, M, N, K = case
+    A, Bt = rand_operands(dtype, M, N, K, 91)
+    sites = site_table(dtype, M, N, K, 300, 92)
+    mpg.mpgemmfi_set_tile_policy(tiles)
+    mpg.mpgemmfi_set_split_policy(mpg.SPLIT_ON)
+    check_gemm_against_oracle(dtype, A, Bt, sites, orc.T_BOUND | orc.CORRECT, max_fragile=2)
+
+
+def test_split_policy_argument():
+    assert mpg.mpgemmfi_set_split_policy(3) == -1
+    assert mpg.mpgemmfi_set_split_policy(mpg.SPLIT_AUTO) == 0
