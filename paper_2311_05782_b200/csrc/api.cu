@@ -175,15 +175,12 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
     p.exp_a = exp_a; p.exp_b = exp_bt;
     p.log2_k = 0;
     while ((1 << p.log2_k) < K) ++p.log2_k;
-    if (flags) {
-        const cudaError_t e = cudaMemsetAsync(flags, 0, sizeof(uint32_t) * (MPGEMMFI_HEADER_WORDS + 4 * (size_t)n_faults), stream);
-        if (e != cudaSuccess) return cuda_fail(e);
-    }
     const int walkers = pair ? max_pairs : di.num_sms;
-    p.epoch = 0; p.signals = nullptr;
+    p.epoch = 0; p.signals = nullptr; p.ready = nullptr;
     choose_split(p, walkers);
-    if (p.split_parts > 1) {
-        const cudaError_t es = mpg::gemm_split_signals(&p.epoch, &p.signals);
+    if (p.split_parts > 1 || flags) {
+        // (the header and the site log of `flags` are cleared by the kernel itself)
+        const cudaError_t es = mpg::gemm_launch_slot(&p.epoch, &p.signals, &p.ready);
         if (es != cudaSuccess) return cuda_fail(es);
     }
     const int grid = (p.num_tiles < walkers ? p.num_tiles : walkers) * (pair ? 2 : 1);

@@ -566,6 +566,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         if (sl.beg + lane < sl.end) first_site = load_site(p.sites, sl.beg + lane);
     }
 
+    if (blockIdx.x == 0 && p.flags) {
+        // header and site log start at zero: cleared here rather than by a memset in front of every launch
+        // (2.5 us each); the other CTAs learn through *p.ready that it has been done
+        for (uint32_t i = threadIdx.x; i < (uint32_t)(MPGEMMFI_HEADER_WORDS + 4 * p.n_faults); i += NUM_THREADS) p.flags[i] = 0u;
+        __syncthreads();
+        if (threadIdx.x == 0) { __threadfence(); signal_store_release(p.ready, p.epoch); }
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             // pair mode, leader CTA: one arrival per CTA of the pair (each announces its own bytes)
@@ -586,6 +593,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         else { tmem_alloc(smem_u32(&ctl->tmem_base), C::TMEM_COLS); tmem_relinquish(); }
     }
     build_site_list<TM, BN>(p, ctl, gid, groups, first_site);
+    // a CTA with sites writes log entries as it goes: not before CTA 0 has cleared the log
+    if (threadIdx.x == 0 && blockIdx.x != 0 && p.flags && ctl->site_count != 0) signal_wait(p.ready, p.epoch, abort_flag);
     tc_fence_before_sync();
     if constexpr (kPair) cluster_sync_all(); else __syncthreads();
     tc_fence_after_sync();
@@ -1009,7 +1018,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             }
         }
         n_det = __reduce_add_sync(0xFFFFFFFFu, n_det);
-        if (lane == 0 && n_det && p.flags) {
+        if (lane == 0 && n_det && p.flags && (blockIdx.x == 0 || signal_wait(p.ready, p.epoch, abort_flag))) {
             atomicAdd(&p.flags[1], n_det);
             if (want_corr) atomicAdd(&p.flags[2], n_det);
         }
@@ -1023,7 +1032,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         if constexpr (kPair) tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
         else tmem_dealloc(tmem_base, C::TMEM_COLS);
     }
-    if (threadIdx.x == 0 && ctl->abort_flag && p.flags) atomicOr(&p.flags[0], MPGEMMFI_STATUS_WAIT_LIMIT);
+    if (threadIdx.x == 0 && ctl->abort_flag && p.flags) {
+        if (blockIdx.x != 0) { volatile uint32_t never = 0; signal_wait(p.ready, p.epoch, &never, 1000000000ull); }
+        atomicOr(&p.flags[0], MPGEMMFI_STATUS_WAIT_LIMIT);
+    }
     if (threadIdx.x == 0 && blockIdx.x == 0 && p.flags && p.split_parts > 1) p.flags[5] = (uint32_t)p.split_parts;
 }
 
@@ -1089,10 +1101,10 @@ int gemm_max_resident_pairs(int dtype)
 }
 
 namespace {
-__device__ uint32_t g_split_signals[SPLIT_SIGNAL_SLOTS][SPLIT_SIGNAL_WORDS];
+__device__ uint32_t g_launch_slots[LAUNCH_SLOTS][LAUNCH_SLOT_WORDS];
 }
 
-cudaError_t gemm_split_signals(uint32_t *epoch, uint32_t **signals)
+cudaError_t gemm_launch_slot(uint32_t *epoch, uint32_t **signals, uint32_t **ready)
 {
     static uint32_t *base[64] = {};
     static std::atomic<uint32_t> counter{0};
@@ -1102,13 +1114,14 @@ cudaError_t gemm_split_signals(uint32_t *epoch, uint32_t **signals)
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!base[dev]) {
         void *ptr = nullptr;
-        e = cudaGetSymbolAddress(&ptr, g_split_signals);
+        e = cudaGetSymbolAddress(&ptr, g_launch_slots);
         if (e != cudaSuccess) return e;
         base[dev] = static_cast<uint32_t *>(ptr);
     }
     const uint32_t n = counter.fetch_add(1u) + 1u;
     *epoch = n & 0x1FFFFFFFu ? n & 0x1FFFFFFFu : 1u;     // 29 bits (3 more carry the part number), never 0
-    *signals = base[dev] + (size_t)(n % SPLIT_SIGNAL_SLOTS) * SPLIT_SIGNAL_WORDS;
+    *signals = base[dev] + (size_t)(n % LAUNCH_SLOTS) * LAUNCH_SLOT_WORDS;
+    *ready = *signals + SPLIT_SIGNAL_WORDS;
     return cudaSuccess;
 }
 

@@ -29,19 +29,23 @@ struct GemmParams {
     // out `full_rounds` whole tiles each; the `left_tiles` tiles that remain are cut along K into
     // `split_parts` parts run by different walkers, the accumulators travelling through C.
     int split_parts, full_rounds, left_tiles;
-    uint32_t epoch;        // tag of this launch in the hand-over words
+    uint32_t epoch;        // tag of this launch in the hand-over words and in *ready
     uint32_t *signals;     // SPLIT_SIGNAL_WORDS hand-over words of this launch (device memory)
+    // With a flags buffer: CTA 0 clears the header and the site log when it starts, then stores `epoch`
+    // here (release); any other CTA reads it (acquire, bounded wait) before it touches header or log.
+    uint32_t *ready;
 };
 
 // hand-over words one launch can use: 16 per left-over tile, fewer left-over tiles than walkers
 constexpr int SPLIT_MAX_WALKERS = 160;
 constexpr int SPLIT_SIGNAL_WORDS = SPLIT_MAX_WALKERS * 16;
 
-// Gives a launch that uses the split schedule its tag and its hand-over words: a slot of a static
-// device array, slots handed out in turn (a slot comes round again after SPLIT_SIGNAL_SLOTS launches;
-// the tag keeps a launch from reading what an earlier one left there).
-constexpr int SPLIT_SIGNAL_SLOTS = 16;
-cudaError_t gemm_split_signals(uint32_t *epoch, uint32_t **signals);
+// Gives a launch its tag, its hand-over words and its ready word: a slot of a static device array,
+// slots handed out in turn (a slot comes round again after LAUNCH_SLOTS launches; the tag keeps a
+// launch from reading what an earlier one left there).
+constexpr int LAUNCH_SLOTS = 16;
+constexpr int LAUNCH_SLOT_WORDS = SPLIT_SIGNAL_WORDS + 16;
+cudaError_t gemm_launch_slot(uint32_t *epoch, uint32_t **signals, uint32_t **ready);
 
 // shared-memory pipeline depth used for an output tile that is bn columns wide
 int gemm_stage_count(int bn, bool pair);
