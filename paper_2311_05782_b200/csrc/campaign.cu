@@ -200,18 +200,18 @@ __global__ void __launch_bounds__(256) element_kernel(CampaignParams p)
 
 // ---------------------------------------------------------------- operand trials (one CTA each)
 
-// which = 0: A-site trials (row i fixed, walk the N columns); which = 1: B-site trials
-// (column j fixed, walk the M rows).
-__global__ void __launch_bounds__(VEC_THREADS) vector_kernel(CampaignParams p, int which)
+// A-site trials (row i fixed, walk the N columns) and, when with_b is set, B-site trials (column j
+// fixed, walk the M rows) in one launch: one CTA per trial, the A list first.
+__global__ void __launch_bounds__(VEC_THREADS) vector_kernel(CampaignParams p, int with_b)
 {
     __shared__ Stats warp_stats[VEC_THREADS / 32];
-    const uint32_t count = p.counters[which];
-    const uint32_t *list = which == 0 ? p.list_a : p.list_b;
+    const uint32_t count_a = p.counters[0];
+    const uint32_t count = count_a + (with_b ? p.counters[1] : 0u);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (uint32_t w = blockIdx.x; w < count; w += gridDim.x) {
-        const uint32_t t = list[w];
+        const bool is_a = w < count_a;
+        const uint32_t t = is_a ? p.list_a[w] : p.list_b[w - count_a];
         const mpgemmfi_site s = load_site(p.sites, t);
-        const bool is_a = which == 0;
         const size_t pos = (size_t)(is_a ? s.row : s.col) * p.K + s.k;
         const uint32_t w_clean = load_operand(p.dtype, is_a ? p.A : p.Bt, pos);
         const float x = widen_operand(p.dtype, w_clean);
@@ -220,13 +220,31 @@ __global__ void __launch_bounds__(VEC_THREADS) vector_kernel(CampaignParams p, i
         const void *other = is_a ? p.Bt : p.A;
         Stats st;
         stats_init(st);
-        for (uint32_t o = threadIdx.x; o < n_other; o += VEC_THREADS) {
-            const float y = widen_operand(p.dtype, load_operand(p.dtype, other, (size_t)o * p.K + s.k));
-            const uint32_t lin = is_a ? s.row * (uint32_t)p.N + o : o * (uint32_t)p.N + s.col;
-            const float c = p.C[lin];
-            const float rep = __fsub_rn(c, __fmul_rn(x, y));        // Eq. 1 on the finished sum
-            const float cf = __fadd_rn(rep, __fmul_rn(xf, y));      // Eq. 2
-            stats_account(st, p.detect_mode, f32_bits(cf), f32_bits(c), lin);
+        // four elements per thread and round: their (strided, L2-latency-bound) loads are all in flight
+        // before the first is used
+        constexpr int UNROLL = 4;
+        for (uint32_t o0 = threadIdx.x; o0 < n_other; o0 += UNROLL * VEC_THREADS) {
+            uint32_t yw[UNROLL];
+            float c[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const uint32_t o = o0 + (uint32_t)(u * VEC_THREADS);
+                if (o < n_other) {
+                    yw[u] = load_operand(p.dtype, other, (size_t)o * p.K + s.k);
+                    c[u] = p.C[is_a ? s.row * (uint32_t)p.N + o : o * (uint32_t)p.N + s.col];
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const uint32_t o = o0 + (uint32_t)(u * VEC_THREADS);
+                if (o < n_other) {
+                    const float y = widen_operand(p.dtype, yw[u]);
+                    const uint32_t lin = is_a ? s.row * (uint32_t)p.N + o : o * (uint32_t)p.N + s.col;
+                    const float rep = __fsub_rn(c[u], __fmul_rn(x, y));        // Eq. 1 on the finished sum
+                    const float cf = __fadd_rn(rep, __fmul_rn(xf, y));         // Eq. 2
+                    stats_account(st, p.detect_mode, f32_bits(cf), f32_bits(c[u]), lin);
+                }
+            }
         }
         stats_warp_reduce(st);
         if (lane == 0) warp_stats[warp] = st;
@@ -530,10 +548,12 @@ cudaError_t launch_campaign_trials(const CampaignParams &p, int num_sms, cudaStr
     const int grid_e = min((p.n_trials + 7) / 8, max_ctas);
     element_kernel<<<grid_e, 256, 0, stream>>>(p);
     const int grid_v = min(p.n_trials, max_ctas);
-    vector_kernel<<<grid_v, VEC_THREADS, 0, stream>>>(p, 0);
-    // B-site trials: by row panel when a useful panel fits in shared memory and the columns are long
+    // B-site trials: by row panel when a useful panel fits in shared memory and the columns are long;
+    // otherwise one CTA per trial, in the same launch as the A-site trials
     const PanelShape ps = panel_shape(p.dtype, p.N, p.K, 227 * 1024);
-    if (ps.rows >= 64 && p.M >= 16 * ps.rows) {
+    const bool by_panel = ps.rows >= 64 && p.M >= 16 * ps.rows;
+    vector_kernel<<<grid_v, VEC_THREADS, 0, stream>>>(p, by_panel ? 0 : 1);
+    if (by_panel) {
         static bool configured[64] = {};
         int dev = 0;
         e = cudaGetDevice(&dev);
@@ -544,8 +564,6 @@ cudaError_t launch_campaign_trials(const CampaignParams &p, int num_sms, cudaStr
             if (dev >= 0 && dev < 64) configured[dev] = true;
         }
         panel_kernel<<<num_sms, PANEL_THREADS, ps.smem, stream>>>(p, ps);
-    } else {
-        vector_kernel<<<grid_v, VEC_THREADS, 0, stream>>>(p, 1);
     }
     return cudaGetLastError();
 }

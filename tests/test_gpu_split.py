@@ -109,3 +109,42 @@ def test_split_schedule_against_oracle(case, policies):
 def test_split_policy_argument():
     assert mpg.mpgemmfi_set_split_policy(3) == -1
     assert mpg.mpgemmfi_set_split_policy(mpg.SPLIT_AUTO) == 0
+
+
+def test_two_streams_at_once(policies):
+    """Two split-schedule GEMMs with flags buffers in flight on two streams (each launch has its own hand-over slot
+    and tag): every result equals the one of the same GEMM run alone."""
+    dtype = orc.BF16
+    shapes = [(2304, 2304, 1024), (3328, 2048, 512)]
+    mpg.mpgemmfi_set_tile_policy(mpg.TILES_PAIR)
+    mpg.mpgemmfi_set_split_policy(mpg.SPLIT_ON)
+    ops, alone = [], []
+    for i, (M, N, K) in enumerate(shapes):
+        A, Bt = rand_operands(dtype, M, N, K, 40 + i)
+        sites = site_table(dtype, M, N, K, 64, 50 + i)
+        a, b = to_dev(A, dtype), to_dev(Bt, dtype)
+        sd = torch.from_numpy(sites.view(np.int32).reshape(-1, 8)).cuda()
+        ops.append((M, N, K, a, b, sd))
+        Cg, flags = mpg.gemm(dtype, a, b, sites, orc.T_BOUND | orc.CORRECT)
+        torch.cuda.synchronize()
+        alone.append((Cg.cpu().numpy().view(np.uint32), flags.cpu().numpy()))
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = []
+    for (M, N, K, a, b, sd) in ops:
+        c = torch.empty((M, N), dtype=torch.float32, device="cuda")
+        f = torch.empty(mpg.mpgemmfi_flags_bytes(M, N, 64) // 4, dtype=torch.int32, device="cuda")
+        outs.append((c, f))
+    torch.cuda.synchronize()
+    for rep in range(6):
+        for k, (M, N, K, a, b, sd) in enumerate(ops):
+            c, f = outs[k]
+            rc = mpg.mpgemmfi_gemm(dtype, M, N, K, a.data_ptr(), b.data_ptr(), c.data_ptr(), sd.data_ptr(), 64,
+                                   orc.T_BOUND | orc.CORRECT, f.data_ptr(), streams[k].cuda_stream)
+            assert rc == 0
+    torch.cuda.synchronize()
+    for k in range(2):
+        c, f = outs[k]
+        fg = f.cpu().numpy()
+        assert not (int(fg[0]) & mpg.STATUS_WAIT_LIMIT)
+        assert np.array_equal(c.cpu().numpy().view(np.uint32), alone[k][0])
+        assert np.array_equal(fg, alone[k][1])
