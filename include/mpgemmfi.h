@@ -9,6 +9,11 @@
  * Problems found on the device (a site outside the matrices, a wait that ran into
  * its time limit) never trap: they set bits in the status word of the flags header
  * (or the trial record) and the offending site is skipped.
+ * A GEMM launch that has a flags buffer, or whose last round of tiles is cut (see
+ * mpgemmfi_set_split_policy), carries a tag drawn from a counter when the entry point is
+ * called, and uses one of 16 slots of a 160 KB static device array for the words its CTAs
+ * hand to each other: launches on several streams may overlap, but a launch recorded once
+ * and replayed (a CUDA graph) would reuse its tag and is not supported.
  *
  * Operation (paper Section II-B, IV-C): D = A x B with A (M x K) and B (K x N) in a
  * low-precision format -- FP16 (1/5/10), BF16 (1/8/7) or TF32 (1/8/10 held in a

@@ -36,6 +36,9 @@ def test_host_helpers():
     assert mpg.mpgemmfi_campaign_workspace_bytes(0, 8, 8, 8, 1000) % 256 == 0
     assert mpg.mpgemmfi_campaign_workspace_bytes(0, 8, 8, 8, 1000) >= 12000
     assert "align" in mpg.mpgemmfi_strerror(-3)
+    # tuning knobs: argument checks need no device
+    assert mpg.mpgemmfi_set_tile_policy(7) == -1 and mpg.mpgemmfi_set_tile_policy(mpg.TILES_AUTO) == 0
+    assert mpg.mpgemmfi_set_split_policy(-1) == -1 and mpg.mpgemmfi_set_split_policy(mpg.SPLIT_AUTO) == 0
     # struct sizes the ABI promises
     assert mpg.SITE_DTYPE.itemsize == 32 and mpg.SITE_LOG_DTYPE.itemsize == 16 and mpg.RECORD_DTYPE.itemsize == 48
 
