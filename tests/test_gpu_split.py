@@ -148,3 +148,22 @@ def test_two_streams_at_once(policies):
         assert not (int(fg[0]) & mpg.STATUS_WAIT_LIMIT)
         assert np.array_equal(c.cpu().numpy().view(np.uint32), alone[k][0])
         assert np.array_equal(fg, alone[k][1])
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_shapes_under_split_schedule(seed, policies):
+    """Differential fuzz against the oracle with the split schedule forced on: random shape (enough tiles for a
+    left-over round under either tiling), format, check mode and site table (all kinds, a repeat, invalid entries)."""
+    rng = np.random.default_rng(7000 + seed)
+    dtype = int(rng.integers(0, 3))
+    kt = synth.kstep(dtype)
+    unit = 4 if dtype == orc.TF32 else 8
+    M = int(rng.integers(2100, 3700)); N = int(rng.integers(2100, 3700)); K = unit * int(rng.integers(40, 80))
+    N -= N % 4                                    # the split schedule needs 16-byte rows of C
+    mode = int(rng.choice([orc.T_NONE, orc.T_BOUND, orc.T_BOUND | orc.CORRECT, orc.T_RMAX | orc.CORRECT, orc.T_RFLIP | orc.CORRECT]))
+    A, Bt = rand_operands(dtype, M, N, K, 7100 + seed)
+    s = site_table(dtype, M, N, K, 48, 7200 + seed)
+    s[1] = s[0]; s["row"][2] = M + 5; s["kind"][3] = 7
+    mpg.mpgemmfi_set_tile_policy([mpg.TILES_PAIR, mpg.TILES_SINGLE][seed % 2])
+    mpg.mpgemmfi_set_split_policy(mpg.SPLIT_ON)
+    check_gemm_against_oracle(dtype, A, Bt, s, mode, max_fragile=2)
