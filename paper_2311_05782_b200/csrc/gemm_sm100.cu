@@ -712,15 +712,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             tc_fence_after_sync();
             const uint32_t d_tmem = tmem_base + as * BN;
             const uint32_t fresh_kt = sg.load ? NONE : sg.kt0;      // the k-tile whose first MMA overwrites the accumulator
-            if (next_op >= sg.kt1 && next_b > sg.kt1) {
-                // no operand, accumulator or term site in these k-tiles (the usual case): one thread
-                // runs the whole loop, with no warp-wide step in it, so that issuing a k-tile's MMAs
-                // takes less time than the tensor core needs to run them
+            uint32_t kt = sg.kt0;
+            while (kt < sg.kt1) {
+              // k-tiles up to the next one with a site (an operand site in it, or an accumulator / term site
+              // at the boundary behind it) -- usually all of them: one thread runs the loop, with no
+              // warp-wide step in it, so that issuing a k-tile's MMAs takes less time than the tensor core
+              // needs to run them
+              const uint32_t stop = min(sg.kt1, min(next_op, next_b - 1u));
+              if (kt < stop) {
                 if (lane == 0) {
                     const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
                     const uint64_t desc0 = umma_smem_desc_sw128(smem_u32(smem));
-                    uint32_t accumulate = sg.load ? 1u : 0u;
-                    for (uint32_t kt = sg.kt0; kt < sg.kt1; ++kt) {
+                    uint32_t accumulate = kt == fresh_kt ? 0u : 1u;
+                    for (; kt < stop; ++kt) {
                         if (!mbar_wait(full0 + stage * 8u, phase, abort_flag)) { ok = false; break; }
                         tc_fence_after_sync();
                         // the address field counts 16-byte units: stage s starts s * STAGE_BYTES / 16 further on
@@ -740,8 +744,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
                 stage = __shfl_sync(0xFFFFFFFFu, stage, 0);
                 phase = __shfl_sync(0xFFFFFFFFu, phase, 0);
-            } else
-            for (uint32_t kt = sg.kt0; kt < sg.kt1; ++kt) {
+                if (!ok) break;
+                kt = stop;
+                continue;
+              }
+              // one k-tile with a site, by the whole warp
+              {
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag));
                 if (!ok) break;
                 tc_fence_after_sync();
@@ -781,6 +789,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     next_b = scan_next_boundary(tc, kt + 2, lane);
                 }
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                ++kt;
+              }
             }
             if (!ok) break;
             if (lane == 0) {
