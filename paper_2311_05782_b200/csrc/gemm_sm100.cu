@@ -972,12 +972,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                         if (c0 + 32 > (uint32_t)p.N) fw &= c0 < (uint32_t)p.N ? (1u << ((uint32_t)p.N - c0)) - 1u : 0u;
                     }
                     if constexpr (do_bound) {
+                        // A flagged element has exponent bit 7 (word bit 30) set. The OR of the 32 words costs a
+                        // third of the per-element test and settles the usual case (every |value| < 2) at once.
+                        uint32_t any = 0;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            // exponent field >= 0x90 <=> not (|value| < 131072); NaN compares false, so it is caught
-                            const bool det = !(fabsf(bits_f32(v[j])) < 131072.0f);
-                            if (det) fw |= 1u << j;
-                            if (kMode == EPI_BOUND_CORRECT && det) v[j] = boundcheck_clear(v[j]);
+                        for (int j = 0; j < 32; ++j) any |= v[j];
+                        if (any & 0x40000000u) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                // exponent field >= 0x90 <=> not (|value| < 131072); NaN compares false, so it is caught
+                                const bool det = !(fabsf(bits_f32(v[j])) < 131072.0f);
+                                if (det) fw |= 1u << j;
+                                if (kMode == EPI_BOUND_CORRECT && det) v[j] = boundcheck_clear(v[j]);
+                            }
                         }
                         // columns past N are not part of C (their zero-filled Bt rows still give NaN against an
                         // Inf or NaN in A): their flag bits stay 0
