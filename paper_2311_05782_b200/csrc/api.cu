@@ -85,6 +85,22 @@ int encode_operand_map(CUtensorMap *map, int dtype, const void *base, int rows, 
     return MPGEMMFI_OK;
 }
 
+// C as an M x N FP32 tensor; box = 32 columns (one 128-byte swizzle row) x 16 rows: what one epilogue warp
+// hands to the TMA engine per store
+int encode_output_map(CUtensorMap *map, float *C, int M, int N)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return cuda_fail(cudaErrorUnknown);
+    const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)N * 4u};
+    const cuuint32_t box[2] = {32, 16};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return MPGEMMFI_ERR_CUDA; }
+    return MPGEMMFI_OK;
+}
+
 int g_tile_policy = MPGEMMFI_TILES_AUTO;
 int g_split_policy = MPGEMMFI_SPLIT_AUTO;
 
@@ -171,6 +187,12 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
     p.num_kt = (K + ks - 1) / ks;
     p.wpr = (N + 31) / 32;
     p.c_vec_ok = (N % 4 == 0) && (((uintptr_t)C & 15) == 0);
+    CUtensorMap tm_c;
+    memset(&tm_c, 0, sizeof(tm_c));
+    if (p.c_vec_ok) {
+        rc = encode_output_map(&tm_c, C, M, N);
+        if (rc) return rc;
+    }
     p.A = A; p.Bt = Bt; p.C = C; p.sites = sites; p.flags = flags;
     p.exp_a = exp_a; p.exp_b = exp_bt;
     p.log2_k = 0;
@@ -184,7 +206,7 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
         if (es != cudaSuccess) return cuda_fail(es);
     }
     const int grid = (p.num_tiles < walkers ? p.num_tiles : walkers) * (pair ? 2 : 1);
-    const cudaError_t e = mpg::launch_gemm(bn, pair, tm_a, tm_b, p, grid, stream);
+    const cudaError_t e = mpg::launch_gemm(bn, pair, tm_a, tm_b, tm_c, p, grid, stream);
     return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
 }
 

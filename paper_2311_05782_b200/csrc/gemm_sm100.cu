@@ -539,7 +539,8 @@ __device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid,
 // kPair = true : grid of CTA pairs (cluster dimension 2), tiles 256 x BN, BN = 256.
 template <int BN, bool kTF32, bool kPair>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, const GemmParams p)
+gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+            const __grid_constant__ CUtensorMap tm_c, const GemmParams p)
 {
     using C = Cfg<BN, kPair>;
     constexpr int KT = kTF32 ? 32 : 64;      // elements per 128-byte row
@@ -587,6 +588,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         mbar_fence_init();
         tma_prefetch_desc(&tm_a);
         tma_prefetch_desc(&tm_b);
+        if (p.c_vec_ok) tma_prefetch_desc(&tm_c);
     }
     if (warp == 2) {
         if constexpr (kPair) { tmem_alloc_pair(smem_u32(&ctl->tmem_base), C::TMEM_COLS); tmem_relinquish_pair(); }
@@ -831,6 +833,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 if (get_segment(p, gid, groups, lt + 1, nx) && nx.load) {
                     uint32_t tm, tn;
                     tile_coords(p, nx.tile, tm, tn);
+                    if (lane == 0) bulk_wait_read_all();       // the staging rows are free again
+                    __syncwarp();
                     const uint32_t *sig = p.signals + (size_t)(nx.tile - first_left) * 16 + my_signal;
                     const uint32_t t_dst = tmem_base + ((lt + 1) & 1u) * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)(first * 32);
                     ok = load_partial(p.C, (uint32_t)p.M, (uint32_t)p.N, sig, (p.epoch << 3) | nx.part, abort_flag,
@@ -912,6 +916,33 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                         if (c0 + jj < (uint32_t)p.N) crow[c0 + jj] = bits_f32(v[jj]);
                 }
             };
+            // The same for a finished tile when C allows 16-byte accesses: the rows are parked in the layout
+            // of the 128-byte swizzle and one thread hands them to the TMA engine (16 rows x 128 bytes a
+            // store). The warp does not wait for the store, only -- before it parks the next rows -- for
+            // its staging to have been read: the SM's write port (about 32 bytes a cycle) then drains one
+            // warp's rows while the other warps check and park theirs, instead of all eight warps
+            // checking together and then queueing behind the port together.
+            auto store_piece_tma = [&](uint32_t (&v)[32], uint32_t c0) {
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    if (lane == 0) bulk_wait_read_all();
+                    __syncwarp();
+                    if ((lane >> 4) == half) {
+                        uint8_t *srow = my_out + (lane & 15) * 128;
+#pragma unroll
+                        for (int jj = 0; jj < 8; ++jj)
+                            *reinterpret_cast<uint4 *>(srow + ((jj ^ (lane & 7)) << 4)) =
+                                make_uint4(v[4 * jj], v[4 * jj + 1], v[4 * jj + 2], v[4 * jj + 3]);
+                        fence_proxy_async_smem();
+                    }
+                    __syncwarp();
+                    const uint32_t r0 = row0 + (uint32_t)(16 * half);
+                    if (lane == 0 && r0 < (uint32_t)p.M && c0 < (uint32_t)p.N) {
+                        tma_store_2d(&tm_c, smem_u32(my_out), (int)c0, (int)r0);
+                        bulk_commit_group();
+                    }
+                }
+            };
             // accumulator columns of this warp fully read: one arrival towards handing the TMEM
             // buffer back to the MMA warp
             auto release_acc = [&]() {
@@ -926,6 +957,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             if (sg.save) {
                 // unfinished tile: the raw accumulators go to the tile's place in C (no output site, no check),
                 // then the walker of the next part is told that this warp's share is there
+                if (lane == 0) bulk_wait_read_all();
+                __syncwarp();
 #pragma unroll 1
                 for (int i = 0; i < MY_PIECES; ++i) {
                     uint32_t raw[32];
@@ -992,7 +1025,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     }
                     if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 1);
                     flagw[i] = fw;
-                    store_piece(v, c0);
+                    if (p.c_vec_ok) store_piece_tma(v, c0);
+                    else store_piece(v, c0);
                 };
 
                 // software pipeline: the TMEM read of the next piece is in flight while this one is finished
@@ -1034,6 +1068,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             default: finish_tile(std::integral_constant<int, EPI_RANGE>{}); break;
             }
         }
+        if (lane == 0) bulk_wait_read_all();       // shared memory stays until the last store has read it
         n_det = __reduce_add_sync(0xFFFFFFFFu, n_det);
         if (lane == 0 && n_det && p.flags && (blockIdx.x == 0 || signal_wait(p.ready, p.epoch, abort_flag))) {
             atomicAdd(&p.flags[1], n_det);
@@ -1057,8 +1092,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
 }
 
 template <int BN, bool kTF32, bool kPair>
-cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p, int grid,
-                       cudaStream_t stream)
+cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c, const GemmParams &p,
+                       int grid, cudaStream_t stream)
 {
     using C = Cfg<BN, kPair>;
     const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024;
@@ -1083,7 +1118,7 @@ cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const G
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, kTF32, kPair>, tm_a, tm_b, p);
+    return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, kTF32, kPair>, tm_a, tm_b, tm_c, p);
 }
 
 }  // namespace
@@ -1148,17 +1183,17 @@ int gemm_stage_count(int bn, bool pair)
     return bn == 256 ? Cfg<256, false>::STAGES : (bn == 128 ? Cfg<128, false>::STAGES : Cfg<64, false>::STAGES);
 }
 
-cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p,
-                        int grid, cudaStream_t stream)
+cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c,
+                        const GemmParams &p, int grid, cudaStream_t stream)
 {
     const bool tf32 = p.dtype == MPGEMMFI_TF32;
     if (pair)
-        return tf32 ? launch_one<256, true, true>(tm_a, tm_b, p, grid, stream)
-                    : launch_one<256, false, true>(tm_a, tm_b, p, grid, stream);
+        return tf32 ? launch_one<256, true, true>(tm_a, tm_b, tm_c, p, grid, stream)
+                    : launch_one<256, false, true>(tm_a, tm_b, tm_c, p, grid, stream);
     switch (bn) {
-    case 256: return tf32 ? launch_one<256, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<256, false, false>(tm_a, tm_b, p, grid, stream);
-    case 128: return tf32 ? launch_one<128, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<128, false, false>(tm_a, tm_b, p, grid, stream);
-    default:  return tf32 ? launch_one<64, true, false>(tm_a, tm_b, p, grid, stream) : launch_one<64, false, false>(tm_a, tm_b, p, grid, stream);
+    case 256: return tf32 ? launch_one<256, true, false>(tm_a, tm_b, tm_c, p, grid, stream) : launch_one<256, false, false>(tm_a, tm_b, tm_c, p, grid, stream);
+    case 128: return tf32 ? launch_one<128, true, false>(tm_a, tm_b, tm_c, p, grid, stream) : launch_one<128, false, false>(tm_a, tm_b, tm_c, p, grid, stream);
+    default:  return tf32 ? launch_one<64, true, false>(tm_a, tm_b, tm_c, p, grid, stream) : launch_one<64, false, false>(tm_a, tm_b, tm_c, p, grid, stream);
     }
 }
 

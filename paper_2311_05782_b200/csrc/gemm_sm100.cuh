@@ -56,8 +56,10 @@ int gemm_stage_count(int bn, bool pair);
 // Pair mode (pair = true): 256 x 256 tiles walked by CTA pairs; tm_b box is (128 bytes x 128 rows);
 // `grid` is even (two CTAs per pair); p.tiles_m counts 256-row tiles.
 // tm_a always has a box of (128 bytes x 128 rows). Both maps use the 128-byte swizzle.
-cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const GemmParams &p,
-                        int grid, cudaStream_t stream);
+// tm_c covers C (FP32, box 32 columns x 16 rows, 128-byte swizzle) and is used for the stores of finished
+// tiles when p.c_vec_ok is set; otherwise its contents do not matter.
+cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c,
+                        const GemmParams &p, int grid, cudaStream_t stream);
 
 // how many CTA pairs of the pair-mode kernel can be resident at once on the current device (0 if none)
 int gemm_max_resident_pairs(int dtype);

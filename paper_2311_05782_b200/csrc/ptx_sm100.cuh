@@ -189,6 +189,26 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const CUtens
         : "memory");
 }
 
+// 2-D tiled store shared -> global (bulk async group of the issuing thread). c0 is the innermost
+// coordinate and must address a 16-byte boundary; neither coordinate may be negative. Elements that
+// fall outside the tensor are not written.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *m, uint32_t src_smem, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src_smem), "r"(c0), "r"(c1) : "memory");
+}
+
+__device__ __forceinline__ void bulk_commit_group()
+{
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+// the issuing thread's bulk stores have read their shared-memory source (it may be overwritten)
+__device__ __forceinline__ void bulk_wait_read_all()
+{
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+
 // ---------------------------------------------------------------- tensor memory
 
 // whole warp; writes the TMEM base address of the allocation to *dst_smem
