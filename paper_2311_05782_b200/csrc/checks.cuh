@@ -15,6 +15,8 @@ __device__ __forceinline__ uint32_t f32_bits(float f) { return __float_as_uint(f
 __device__ __forceinline__ float bits_f32(uint32_t u) { return __uint_as_float(u); }
 
 MPG_HD int kstep_of(int dtype) { return dtype == MPGEMMFI_TF32 ? 32 : 64; }
+// log2 of the k-step (the k-step is a power of two: shifts instead of integer divisions on the device)
+MPG_HD uint32_t kshift_of(int dtype) { return dtype == MPGEMMFI_TF32 ? 5u : 6u; }
 MPG_HD int esize_of(int dtype) { return dtype == MPGEMMFI_TF32 ? 4 : 2; }
 
 // XOR a mask into an operand storage word. 16-bit formats: mask bits 0..15.
@@ -48,7 +50,7 @@ MPG_HD bool site_valid(const mpgemmfi_site &s, int dtype, int M, int N, int K)
     case MPGEMMFI_SITE_B: return s.col < (uint32_t)N && s.k < (uint32_t)K;
     case MPGEMMFI_SITE_ACC:
         return s.row < (uint32_t)M && s.col < (uint32_t)N && s.k >= 1 && s.k <= (uint32_t)K &&
-               (s.k % ks == 0 || s.k == (uint32_t)K);
+               ((s.k & (ks - 1u)) == 0 || s.k == (uint32_t)K);
     case MPGEMMFI_SITE_OUT: return s.row < (uint32_t)M && s.col < (uint32_t)N;
     case MPGEMMFI_SITE_TERM: return s.row < (uint32_t)M && s.col < (uint32_t)N && s.k < (uint32_t)K;
     default: return false;
@@ -59,9 +61,10 @@ MPG_HD bool site_valid(const mpgemmfi_site &s, int dtype, int M, int N, int K)
 MPG_HD uint32_t site_boundary(const mpgemmfi_site &s, int dtype, int K)
 {
     const uint32_t ks = static_cast<uint32_t>(kstep_of(dtype));
-    const uint32_t nkt = ((uint32_t)K + ks - 1) / ks;
-    if (s.kind == MPGEMMFI_SITE_ACC) return s.k == (uint32_t)K ? nkt : s.k / ks;
-    return s.k / ks + 1;   // TERM: the boundary that ends the k-step containing k
+    const uint32_t sh = kshift_of(dtype);
+    const uint32_t nkt = ((uint32_t)K + ks - 1) >> sh;
+    if (s.kind == MPGEMMFI_SITE_ACC) return s.k == (uint32_t)K ? nkt : s.k >> sh;
+    return (s.k >> sh) + 1;   // TERM: the boundary that ends the k-step containing k
 }
 
 // ---- BoundCheck: exponent bit 7 set and any of exponent bits 6..4 set ("1eeexxxx"), i.e. an

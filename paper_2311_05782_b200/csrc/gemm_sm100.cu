@@ -110,13 +110,13 @@ __device__ __forceinline__ mpgemmfi_site listed_site(const TileCtx &c, uint32_t 
 // smallest k-tile >= kt_from in which this tile has an operand site (warp-wide)
 __device__ uint32_t scan_next_operand(const TileCtx &c, uint32_t kt_from, int lane)
 {
-    const uint32_t ks = (uint32_t)kstep_of(c.p->dtype);
+    const uint32_t sh = kshift_of(c.p->dtype);
     uint32_t best = NONE;
     for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
         const mpgemmfi_site s = listed_site(c, i);
         const bool hit = (s.kind == MPGEMMFI_SITE_A && in_own_rows(c, s.row)) ||
                          (s.kind == MPGEMMFI_SITE_B && in_own_b(c, s.col));
-        if (hit && s.k / ks >= kt_from) best = min(best, s.k / ks);
+        if (hit && (s.k >> sh) >= kt_from) best = min(best, s.k >> sh);
     }
     return __reduce_min_sync(0xFFFFFFFFu, best);
 }
@@ -168,7 +168,7 @@ __device__ __forceinline__ uint32_t swizzled_offset(uint32_t r, uint32_t kb)
 __device__ void apply_operand_sites(const TileCtx &c, uint32_t kt, uint8_t *smem_a, uint8_t *smem_b)
 {
     const GemmParams &p = *c.p;
-    const uint32_t ks = (uint32_t)kstep_of(p.dtype);
+    const uint32_t sh = kshift_of(p.dtype);
     const uint32_t es = (uint32_t)esize_of(p.dtype);
     for (uint32_t i = 0; i < c.ctl->site_count; ++i) {
         const uint32_t idx = c.ctl->site_idx[i];
@@ -179,8 +179,8 @@ __device__ void apply_operand_sites(const TileCtx &c, uint32_t kt, uint8_t *smem
         if (s.kind == MPGEMMFI_SITE_A && in_own_rows(c, s.row)) { tile = smem_a; r = s.row - c.m0; log_here = c.n0 == 0; }
         else if (s.kind == MPGEMMFI_SITE_B && in_own_b(c, s.col)) { tile = smem_b; r = s.col - c.b0; log_here = c.tile_m0 == 0; }
         else continue;
-        if (s.k / ks != kt) continue;
-        uint8_t *ptr = tile + swizzled_offset(r, (s.k % ks) * es);
+        if ((s.k >> sh) != kt) continue;
+        uint8_t *ptr = tile + swizzled_offset(r, (s.k & ((1u << sh) - 1u)) * es);
         uint32_t before, after;
         if (es == 2) {
             unsigned short *w = reinterpret_cast<unsigned short *>(ptr);
@@ -762,7 +762,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                         fence_proxy_async_smem();
                     }
                     __syncwarp();
-                    next_op = scan_next_operand(tc, kt + 1, lane);
                 }
                 if (lane == 0) {
                     const uint64_t a_desc = umma_smem_desc_sw128(smem_u32(sa));
@@ -777,6 +776,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     else umma_commit(smem_u32(&ctl->empty[stage]));
                 }
                 __syncwarp();
+                if (kt == next_op) next_op = scan_next_operand(tc, kt + 1, lane);     // (after the MMAs are on their way)
                 if (kt + 1 == next_b) {
                     // an accumulator / term site takes effect here: let the epilogue warps edit TMEM
                     if (lane == 0) {
