@@ -273,14 +273,14 @@ __global__ void __launch_bounds__(VEC_THREADS) vector_kernel(CampaignParams p, i
 // are evaluated panel by panel: a CTA loads a panel once and applies a whole group of trials to
 // it, so A and C are streamed once per GROUP of trials instead of once per trial (each trial
 // alone would pull one 32-byte sector per row out of both matrices).
-// Work item = (group of up to PANEL_GROUP trials) x (contiguous chunk of panels); partial
-// statistics are kept in shared memory per trial and merged into the records with atomics.
+// Work item = (group of up to PANEL_GROUP trials) x (contiguous chunk of panels); a thread keeps its
+// trial's partial statistics in registers and merges them into the record with atomics at the end.
 constexpr int PANEL_GROUP = 1024;
 constexpr int PANEL_THREADS = 1024;
 
 struct PanelShape {
-    int rows;        // R, multiple of 32
-    int a_words;     // 32-bit words per staged A row (odd: conflict-free column reads)
+    int rows;        // R, multiple of 8
+    int a_words;     // 32-bit words per staged A row (odd, so that rows start in different banks)
     int c_words;     // 32-bit words per staged C row (odd)
     size_t smem;
 };
@@ -291,18 +291,66 @@ __host__ __device__ inline PanelShape panel_shape(int dtype, int N, int K, size_
     s.a_words = (K * esize_of(dtype) + 3) / 4;
     s.a_words |= 1;
     s.c_words = N | 1;
-    const size_t fixed = (size_t)PANEL_GROUP * (5 * 4 + 4 * 4 + 8) + 1024;    // trial parameters + statistics
+    const size_t fixed = (size_t)PANEL_GROUP * (6 * 4) + 256;    // trial parameters and sort keys
     const size_t row_bytes = 4 * (size_t)(s.a_words + s.c_words);
     long long r = smem_limit > fixed ? (long long)((smem_limit - fixed) / row_bytes) : 0;
-    r = r / 32 * 32;
+    r = r / 8 * 8;
     if (r > 256) r = 256;
     s.rows = (int)r;
     s.smem = fixed + row_bytes * (size_t)(r > 0 ? r : 0);
     return s;
 }
 
+// One thread per trial of the group (PANEL_GROUP == PANEL_THREADS): it walks the rows of the staged panel
+// with its own column j of C and its own element k of every A row, and keeps its trial's statistics in
+// registers over the whole chunk of panels -- no warp-wide reduction, one merge into the record per item.
+// The trials of a group are ordered by k first, so that the threads of a warp read the same or
+// neighbouring words of an A row (broadcast, or distinct banks) instead of 32 random ones.
+template <int kDtype>
+__device__ __forceinline__ void panel_rows(const uint32_t *As, const uint32_t *Cs, const PanelShape &ps, uint32_t rows,
+                                           uint32_t lin_base, uint32_t n_cols, uint32_t j, uint32_t k, float b, float bf,
+                                           bool do_bound, bool do_corr, uint32_t &n_det, uint32_t &first,
+                                           unsigned long long &hash, float &maxdev, uint32_t &changed)
+{
+    constexpr bool two_byte = kDtype != MPGEMMFI_TF32;
+    // the trial's element of the first row: a 16-bit half of a word (byte selector for PRMT) or a word
+    const uint32_t *a_ptr = As + (two_byte ? (k >> 1) : k);
+    const uint32_t a_sel = (k & 1u) ? 0x4432u : 0x4410u;          // bytes 2,3 or 0,1 into the low half, zeros above
+    const uint32_t *c_ptr = Cs + j;
+    const uint32_t a_step = (uint32_t)ps.a_words, c_step = (uint32_t)ps.c_words;
+#pragma unroll 4
+    for (uint32_t r = 0; r < rows; ++r, a_ptr += a_step, c_ptr += c_step) {
+        uint32_t aw = *a_ptr;
+        if (two_byte) aw = __byte_perm(aw, 0u, a_sel);
+        const float a = widen_operand(kDtype, aw);
+        const uint32_t c_bits = *c_ptr;
+        const float c = bits_f32(c_bits);
+        const float rep = __fsub_rn(c, __fmul_rn(a, b));          // Eq. 1 on the finished sum
+        const float cf = __fadd_rn(rep, __fmul_rn(a, bf));        // Eq. 2
+        uint32_t fin = f32_bits(cf);
+        if (!(fabsf(cf) < 131072.0f)) {
+            // rare: exponent field >= 0x90 (what BoundCheck flags), infinities and NaNs
+            if (do_bound) {
+                const uint32_t lin = lin_base + r * n_cols;
+                ++n_det;
+                hash += ((unsigned long long)lin + 1ull) * HASH_MUL;
+                first = min(first, lin);
+                if (do_corr) fin = boundcheck_clear(fin);
+            }
+            // a NaN deviation counts as +inf (fmaxf below would drop it)
+            const float d = fabsf(__fsub_rn(bits_f32(fin), c));
+            if (d != d) maxdev = __uint_as_float(0x7F800000u);
+        }
+        changed |= fin ^ c_bits;
+        // a finite cf and a NaN or infinite clean value cannot meet (cf would not be finite), so outside the
+        // branch above the deviation is never NaN
+        maxdev = fmaxf(maxdev, fabsf(__fsub_rn(bits_f32(fin), c)));
+    }
+}
+
 __global__ void __launch_bounds__(PANEL_THREADS) panel_kernel(CampaignParams p, PanelShape ps)
 {
+    static_assert(PANEL_GROUP == PANEL_THREADS, "one thread per trial of a group");
     extern __shared__ __align__(16) unsigned char panel_smem[];
     uint32_t *As = reinterpret_cast<uint32_t *>(panel_smem);
     uint32_t *Cs = As + (size_t)ps.rows * ps.a_words;
@@ -311,16 +359,11 @@ __global__ void __launch_bounds__(PANEL_THREADS) panel_kernel(CampaignParams p, 
     uint32_t *t_k = t_j + PANEL_GROUP;
     float *t_b = reinterpret_cast<float *>(t_k + PANEL_GROUP);
     float *t_bf = t_b + PANEL_GROUP;
-    uint32_t *s_ndet = reinterpret_cast<uint32_t *>(t_bf + PANEL_GROUP);
-    uint32_t *s_first = s_ndet + PANEL_GROUP;
-    uint32_t *s_maxdev = s_first + PANEL_GROUP;
-    uint32_t *s_changed = s_maxdev + PANEL_GROUP;
-    unsigned long long *s_hash = reinterpret_cast<unsigned long long *>(
-        (reinterpret_cast<uintptr_t>(s_changed + PANEL_GROUP) + 7) & ~uintptr_t(7));
+    uint32_t *t_key = reinterpret_cast<uint32_t *>(t_bf + PANEL_GROUP);
 
     const uint32_t count = p.counters[1];
     if (count == 0) return;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t tid = threadIdx.x;
     const int es = esize_of(p.dtype);
     const uint32_t n_groups = (count + PANEL_GROUP - 1) / PANEL_GROUP;
     const uint32_t n_panels = ((uint32_t)p.M + ps.rows - 1) / ps.rows;
@@ -328,120 +371,85 @@ __global__ void __launch_bounds__(PANEL_THREADS) panel_kernel(CampaignParams p, 
     uint32_t n_chunks = (2 * gridDim.x + n_groups - 1) / n_groups;
     n_chunks = max(1u, min(n_chunks, (n_panels + 3) / 4));
     const uint32_t panels_per_chunk = (n_panels + n_chunks - 1) / n_chunks;
+    const bool do_bound = (p.detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK) == MPGEMMFI_DETECT_BOUNDCHECK;
+    const bool do_corr = do_bound && (p.detect_mode & MPGEMMFI_CORRECT);
 
     for (uint32_t item = blockIdx.x; item < n_groups * n_chunks; item += gridDim.x) {
         const uint32_t g = item / n_chunks, ch = item % n_chunks;
         const uint32_t g_beg = g * PANEL_GROUP, g_n = min((uint32_t)PANEL_GROUP, count - g_beg);
-        __syncthreads();
-        for (uint32_t i = threadIdx.x; i < g_n; i += PANEL_THREADS) {
-            const uint32_t t = p.list_b[g_beg + i];
-            const mpgemmfi_site s = load_site(p.sites, t);
-            const uint32_t w_clean = load_operand(p.dtype, p.Bt, (size_t)s.col * p.K + s.k);
-            t_id[i] = t; t_j[i] = s.col; t_k[i] = s.k;
-            t_b[i] = widen_operand(p.dtype, w_clean);
-            t_bf[i] = widen_operand(p.dtype, flip_operand(p.dtype, w_clean, s.xor_mask));
-            s_ndet[i] = 0; s_first[i] = 0xFFFFFFFFu; s_maxdev[i] = 0; s_changed[i] = 0; s_hash[i] = 0ull;
+        __syncthreads();                       // the tables of the previous item are no longer read
+        // the group's trials, ordered by k (rank by counting: g_n <= 1024 keys in shared memory)
+        {
+            uint32_t t = 0, j = 0, k = 0xFFFFFFFFu;
+            float b = 0.0f, bf = 0.0f;
+            if (tid < g_n) {
+                t = p.list_b[g_beg + tid];
+                const mpgemmfi_site s = load_site(p.sites, t);
+                const uint32_t w_clean = load_operand(p.dtype, p.Bt, (size_t)s.col * p.K + s.k);
+                j = s.col; k = s.k;
+                b = widen_operand(p.dtype, w_clean);
+                bf = widen_operand(p.dtype, flip_operand(p.dtype, w_clean, s.xor_mask));
+            }
+            t_key[tid] = k;
+            __syncthreads();
+            if (tid < g_n) {
+                uint32_t rank = 0;
+                for (uint32_t i = 0; i < g_n; ++i) {
+                    const uint32_t ki = t_key[i];
+                    rank += (ki < k || (ki == k && i < tid)) ? 1u : 0u;
+                }
+                t_id[rank] = t; t_j[rank] = j; t_k[rank] = k; t_b[rank] = b; t_bf[rank] = bf;
+            }
+            __syncthreads();
         }
+        const bool have = tid < g_n;
+        const uint32_t my_t = have ? t_id[tid] : 0u, my_j = have ? t_j[tid] : 0u, my_k = have ? t_k[tid] : 0u;
+        const float my_b = have ? t_b[tid] : 0.0f, my_bf = have ? t_bf[tid] : 0.0f;
+        uint32_t n_det = 0, first = 0xFFFFFFFFu, changed = 0;
+        float maxdev = 0.0f;                   // non-negative or +inf
+        unsigned long long hash = 0ull;
+
         const uint32_t p_beg = ch * panels_per_chunk, p_end = min(n_panels, p_beg + panels_per_chunk);
         for (uint32_t pn = p_beg; pn < p_end; ++pn) {
             const uint32_t row0 = pn * (uint32_t)ps.rows;
             const uint32_t rows = min((uint32_t)ps.rows, (uint32_t)p.M - row0);
-            __syncthreads();       // the previous panel is no longer read; the trial tables are written
+            __syncthreads();       // the previous panel is no longer read
             // stage the A and C rows of this panel (global reads in 16-byte pieces, rows padded in smem)
             const uint32_t a_vec = (uint32_t)(p.K * es) / 16;     // K * es is a multiple of 16
             const uint4 *Ag = reinterpret_cast<const uint4 *>(reinterpret_cast<const unsigned char *>(p.A) + (size_t)row0 * p.K * es);
-            for (uint32_t i = threadIdx.x; i < rows * a_vec; i += PANEL_THREADS) {
+            for (uint32_t i = tid; i < rows * a_vec; i += PANEL_THREADS) {
                 const uint32_t r = i / a_vec, v = i % a_vec;
                 const uint4 x = __ldg(Ag + (size_t)r * a_vec + v);
                 uint32_t *dst = As + (size_t)r * ps.a_words + 4 * v;
                 dst[0] = x.x; dst[1] = x.y; dst[2] = x.z; dst[3] = x.w;
             }
             const float *Cg = p.C + (size_t)row0 * p.N;
-            for (uint32_t i = threadIdx.x; i < rows * (uint32_t)p.N; i += PANEL_THREADS) {
+            for (uint32_t i = tid; i < rows * (uint32_t)p.N; i += PANEL_THREADS) {
                 const uint32_t r = i / (uint32_t)p.N, c = i % (uint32_t)p.N;
                 Cs[(size_t)r * ps.c_words + c] = f32_bits(Cg[i]);
             }
             __syncthreads();
-            // trials of the group: warp w takes trials w, w + 32, ...; every lane evaluates 4 rows per
-            // 128-row pass. Row addresses do not depend on the trial: hoist them.
-            const bool do_bound = (p.detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK) == MPGEMMFI_DETECT_BOUNDCHECK;
-            const bool do_corr = do_bound && (p.detect_mode & MPGEMMFI_CORRECT);
-            for (uint32_t rb = 0; rb < rows; rb += 128) {
-                const uint32_t *a_row[4];
-                const uint32_t *c_row[4];
-                bool live[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const uint32_t r = rb + (uint32_t)(32 * u) + (uint32_t)lane;
-                    live[u] = r < rows;
-                    const uint32_t rr = live[u] ? r : 0u;           // dead lanes read row 0 and discard
-                    a_row[u] = As + rr * (uint32_t)ps.a_words;
-                    c_row[u] = Cs + rr * (uint32_t)ps.c_words;
-                }
-                const uint32_t lin0 = (row0 + rb + (uint32_t)lane) * (uint32_t)p.N;
-                for (uint32_t i = warp; i < g_n; i += PANEL_THREADS / 32) {
-                    const uint32_t j = t_j[i], k = t_k[i];
-                    const float b = t_b[i], bf = t_bf[i];
-                    uint32_t maxdev = 0, changed = 0, det_mask = 0;
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const uint32_t aw = es == 2 ? (uint32_t)reinterpret_cast<const unsigned short *>(a_row[u])[k] : a_row[u][k];
-                        const float a = widen_operand(p.dtype, aw);
-                        const uint32_t c_bits = c_row[u][j];
-                        const float rep = __fsub_rn(bits_f32(c_bits), __fmul_rn(a, b));      // Eq. 1 on the finished sum
-                        const float cf = __fadd_rn(rep, __fmul_rn(a, bf));                    // Eq. 2
-                        uint32_t fin = f32_bits(cf);
-                        const bool det = do_bound && live[u] && !(fabsf(cf) < 131072.0f);      // exponent field >= 0x90
-                        if (det) { det_mask |= 1u << u; if (do_corr) fin = boundcheck_clear(fin); }
-                        if (live[u]) {
-                            changed |= fin ^ c_bits;
-                            // |deviation| as raw bits: NaN patterns sort above +inf and are clamped to it below
-                            maxdev = max(maxdev, f32_bits(fabsf(__fsub_rn(bits_f32(fin), bits_f32(c_bits)))));
-                        }
-                    }
-                    if (__any_sync(0xFFFFFFFFu, det_mask != 0)) {
-                        // rare: fold the flagged elements of these rows
-                        unsigned long long h = 0ull;
-                        uint32_t first = 0xFFFFFFFFu;
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (det_mask & (1u << u)) {
-                                const uint32_t lin = lin0 + (uint32_t)(32 * u) * (uint32_t)p.N + j;
-                                h += ((unsigned long long)lin + 1ull) * HASH_MUL;
-                                first = min(first, lin);
-                            }
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) h += __shfl_xor_sync(0xFFFFFFFFu, h, o);
-                        first = __reduce_min_sync(0xFFFFFFFFu, first);
-                        const uint32_t n = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)__popc(det_mask));
-                        if (lane == 0) {
-                            s_ndet[i] += n;
-                            s_hash[i] += h;
-                            s_first[i] = min(s_first[i], first);
-                        }
-                    }
-                    maxdev = min(__reduce_max_sync(0xFFFFFFFFu, maxdev), 0x7F800000u);
-                    changed = __reduce_or_sync(0xFFFFFFFFu, changed);
-                    if (lane == 0) {
-                        if (maxdev > s_maxdev[i]) s_maxdev[i] = maxdev;
-                        if (changed) s_changed[i] = 1;
-                    }
-                }
+            if (have) {
+                const uint32_t lin_base = row0 * (uint32_t)p.N + my_j;
+                if (p.dtype == MPGEMMFI_FP16)
+                    panel_rows<MPGEMMFI_FP16>(As, Cs, ps, rows, lin_base, (uint32_t)p.N, my_j, my_k, my_b, my_bf, do_bound, do_corr, n_det, first, hash, maxdev, changed);
+                else if (p.dtype == MPGEMMFI_BF16)
+                    panel_rows<MPGEMMFI_BF16>(As, Cs, ps, rows, lin_base, (uint32_t)p.N, my_j, my_k, my_b, my_bf, do_bound, do_corr, n_det, first, hash, maxdev, changed);
+                else
+                    panel_rows<MPGEMMFI_TF32>(As, Cs, ps, rows, lin_base, (uint32_t)p.N, my_j, my_k, my_b, my_bf, do_bound, do_corr, n_det, first, hash, maxdev, changed);
             }
         }
-        __syncthreads();
-        // merge this item's partial statistics into the records
-        const bool corr = (p.detect_mode & MPGEMMFI_CORRECT) &&
-                          (p.detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK) == MPGEMMFI_DETECT_BOUNDCHECK;
-        for (uint32_t i = threadIdx.x; i < g_n; i += PANEL_THREADS) {
-            mpgemmfi_trial_record *r = &p.records[t_id[i]];
-            if (s_ndet[i]) {
-                atomicAdd(&r->n_detected, s_ndet[i]);
-                atomicAdd(reinterpret_cast<unsigned long long *>(&r->idx_hash), s_hash[i]);
-                atomicMin(&r->first_detected, s_first[i]);
+        // merge this item's statistics into the trial's record
+        if (have) {
+            mpgemmfi_trial_record *r = &p.records[my_t];
+            const uint32_t maxdev_bits = f32_bits(maxdev);     // non-negative floats order like their bit patterns
+            if (n_det) {
+                atomicAdd(&r->n_detected, n_det);
+                atomicAdd(reinterpret_cast<unsigned long long *>(&r->idx_hash), hash);
+                atomicMin(&r->first_detected, first);
             }
-            if (s_maxdev[i]) atomicMax(reinterpret_cast<uint32_t *>(&r->max_abs_dev), s_maxdev[i]);
-            const uint32_t st = (s_changed[i] ? 1u : 0u) | (s_ndet[i] ? 2u : 0u) | ((s_ndet[i] && corr) ? 4u : 0u);
+            if (maxdev_bits) atomicMax(reinterpret_cast<uint32_t *>(&r->max_abs_dev), maxdev_bits);
+            const uint32_t st = (changed ? 1u : 0u) | (n_det ? 2u : 0u) | ((n_det && do_corr) ? 4u : 0u);
             if (st) atomicOr(&r->status, st);
         }
     }
