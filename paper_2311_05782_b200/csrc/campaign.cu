@@ -306,6 +306,14 @@ __host__ __device__ inline PanelShape panel_shape(int dtype, int N, int K, size_
 // registers over the whole chunk of panels -- no warp-wide reduction, one merge into the record per item.
 // The trials of a group are ordered by k first, so that the threads of a warp read the same or
 // neighbouring words of an A row (broadcast, or distinct banks) instead of 32 random ones.
+// 32-bit word of shared memory at a 32-bit shared-space address (address arithmetic stays 32-bit)
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
 template <int kDtype>
 __device__ __forceinline__ void panel_rows(const uint32_t *As, const uint32_t *Cs, const PanelShape &ps, uint32_t rows,
                                            uint32_t lin_base, uint32_t n_cols, uint32_t j, uint32_t k, float b, float bf,
@@ -314,38 +322,59 @@ __device__ __forceinline__ void panel_rows(const uint32_t *As, const uint32_t *C
 {
     constexpr bool two_byte = kDtype != MPGEMMFI_TF32;
     // the trial's element of the first row: a 16-bit half of a word (byte selector for PRMT) or a word
-    const uint32_t *a_ptr = As + (two_byte ? (k >> 1) : k);
+    uint32_t a_addr = (uint32_t)__cvta_generic_to_shared(As + (two_byte ? (k >> 1) : k));
+    uint32_t c_addr = (uint32_t)__cvta_generic_to_shared(Cs + j);
     const uint32_t a_sel = (k & 1u) ? 0x4432u : 0x4410u;          // bytes 2,3 or 0,1 into the low half, zeros above
-    const uint32_t *c_ptr = Cs + j;
-    const uint32_t a_step = (uint32_t)ps.a_words, c_step = (uint32_t)ps.c_words;
-#pragma unroll 4
-    for (uint32_t r = 0; r < rows; ++r, a_ptr += a_step, c_ptr += c_step) {
-        uint32_t aw = *a_ptr;
+    const uint32_t a_step = 4u * (uint32_t)ps.a_words, c_step = 4u * (uint32_t)ps.c_words;
+
+    // one row, every case handled (flagged values, infinities, NaNs)
+    auto exact_row = [&](uint32_t r, uint32_t aw, uint32_t c_bits) {
         if (two_byte) aw = __byte_perm(aw, 0u, a_sel);
         const float a = widen_operand(kDtype, aw);
-        const uint32_t c_bits = *c_ptr;
         const float c = bits_f32(c_bits);
         const float rep = __fsub_rn(c, __fmul_rn(a, b));          // Eq. 1 on the finished sum
         const float cf = __fadd_rn(rep, __fmul_rn(a, bf));        // Eq. 2
         uint32_t fin = f32_bits(cf);
-        if (!(fabsf(cf) < 131072.0f)) {
-            // rare: exponent field >= 0x90 (what BoundCheck flags), infinities and NaNs
-            if (do_bound) {
-                const uint32_t lin = lin_base + r * n_cols;
-                ++n_det;
-                hash += ((unsigned long long)lin + 1ull) * HASH_MUL;
-                first = min(first, lin);
-                if (do_corr) fin = boundcheck_clear(fin);
-            }
-            // a NaN deviation counts as +inf (fmaxf below would drop it)
-            const float d = fabsf(__fsub_rn(bits_f32(fin), c));
-            if (d != d) maxdev = __uint_as_float(0x7F800000u);
+        if (do_bound && !(fabsf(cf) < 131072.0f)) {               // exponent field >= 0x90
+            const uint32_t lin = lin_base + r * n_cols;
+            ++n_det;
+            hash += ((unsigned long long)lin + 1ull) * HASH_MUL;
+            first = min(first, lin);
+            if (do_corr) fin = boundcheck_clear(fin);
         }
         changed |= fin ^ c_bits;
-        // a finite cf and a NaN or infinite clean value cannot meet (cf would not be finite), so outside the
-        // branch above the deviation is never NaN
-        maxdev = fmaxf(maxdev, fabsf(__fsub_rn(bits_f32(fin), c)));
+        const float d = fabsf(__fsub_rn(bits_f32(fin), c));
+        maxdev = d != d ? __uint_as_float(0x7F800000u) : fmaxf(maxdev, d);      // a NaN deviation counts as +inf
+    };
+
+    uint32_t r = 0;
+    for (; r + 4 <= rows; r += 4, a_addr += 4 * a_step, c_addr += 4 * c_step) {
+        // Four rows at once on the assumption that nothing is flagged and nothing is infinite or NaN (one
+        // compare per row, folded into one branch per four rows); otherwise the four rows are done again, exactly.
+        uint32_t aw[4], cb[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { aw[u] = lds_u32(a_addr + u * a_step); cb[u] = lds_u32(c_addr + u * c_step); }
+        bool plain = true;
+        uint32_t ch = 0;
+        float md = 0.0f;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float a = widen_operand(kDtype, two_byte ? __byte_perm(aw[u], 0u, a_sel) : aw[u]);
+            const float c = bits_f32(cb[u]);
+            const float cf = __fadd_rn(__fsub_rn(c, __fmul_rn(a, b)), __fmul_rn(a, bf));     // Eq. 1, Eq. 2
+            plain = plain && (fabsf(cf) < 131072.0f);
+            ch |= f32_bits(cf) ^ cb[u];
+            md = fmaxf(md, fabsf(__fsub_rn(cf, c)));        // cf finite and below the bound: never NaN (c is finite too)
+        }
+        if (plain) {
+            changed |= ch;
+            maxdev = fmaxf(maxdev, md);
+        } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) exact_row(r + u, aw[u], cb[u]);
+        }
     }
+    for (; r < rows; ++r, a_addr += a_step, c_addr += c_step) exact_row(r, lds_u32(a_addr), lds_u32(c_addr));
 }
 
 __global__ void __launch_bounds__(PANEL_THREADS) panel_kernel(CampaignParams p, PanelShape ps)
