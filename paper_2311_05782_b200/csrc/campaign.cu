@@ -279,25 +279,24 @@ constexpr int PANEL_GROUP = 1024;
 constexpr int PANEL_THREADS = 1024;
 
 struct PanelShape {
-    int rows;        // R, multiple of 8
-    int a_words;     // 32-bit words per staged A row (odd, so that rows start in different banks)
-    int c_words;     // 32-bit words per staged C row (odd)
+    int rows;        // R, rows of one staged panel (two panels are resident: one evaluated, one arriving), multiple of 8
+    int a_words;     // 32-bit words per staged A row (the row as it is in global memory: K * element size / 4)
+    int c_words;     // 32-bit words per staged C row (N)
     size_t smem;
 };
 
 __host__ __device__ inline PanelShape panel_shape(int dtype, int N, int K, size_t smem_limit)
 {
     PanelShape s;
-    s.a_words = (K * esize_of(dtype) + 3) / 4;
-    s.a_words |= 1;
-    s.c_words = N | 1;
+    s.a_words = K * esize_of(dtype) / 4;       // K * element size is a multiple of 16 bytes
+    s.c_words = N;
     const size_t fixed = (size_t)PANEL_GROUP * (6 * 4) + 256;    // trial parameters and sort keys
     const size_t row_bytes = 4 * (size_t)(s.a_words + s.c_words);
-    long long r = smem_limit > fixed ? (long long)((smem_limit - fixed) / row_bytes) : 0;
+    long long r = smem_limit > fixed ? (long long)((smem_limit - fixed) / (2 * row_bytes)) : 0;
     r = r / 8 * 8;
-    if (r > 256) r = 256;
+    if (r > 128) r = 128;
     s.rows = (int)r;
-    s.smem = fixed + row_bytes * (size_t)(r > 0 ? r : 0);
+    s.smem = fixed + 2 * row_bytes * (size_t)(r > 0 ? r : 0);
     return s;
 }
 
@@ -306,6 +305,21 @@ __host__ __device__ inline PanelShape panel_shape(int dtype, int N, int K, size_
 // registers over the whole chunk of panels -- no warp-wide reduction, one merge into the record per item.
 // The trials of a group are ordered by k first, so that the threads of a warp read the same or
 // neighbouring words of an A row (broadcast, or distinct banks) instead of 32 random ones.
+// asynchronous global -> shared copies (LSU path, no registers in between), grouped per panel
+__device__ __forceinline__ void cp_async_16(uint32_t dst_smem, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+
+__device__ __forceinline__ void cp_async_4(uint32_t dst_smem, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+
 // 32-bit word of shared memory at a 32-bit shared-space address (address arithmetic stays 32-bit)
 __device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
 {
@@ -381,9 +395,10 @@ __global__ void __launch_bounds__(PANEL_THREADS) panel_kernel(CampaignParams p, 
 {
     static_assert(PANEL_GROUP == PANEL_THREADS, "one thread per trial of a group");
     extern __shared__ __align__(16) unsigned char panel_smem[];
-    uint32_t *As = reinterpret_cast<uint32_t *>(panel_smem);
-    uint32_t *Cs = As + (size_t)ps.rows * ps.a_words;
-    uint32_t *t_id = Cs + (size_t)ps.rows * ps.c_words;
+    // two panels: A rows of both (16-byte aligned), then C rows of both
+    uint32_t *As2 = reinterpret_cast<uint32_t *>(panel_smem);
+    uint32_t *Cs2 = As2 + 2 * (size_t)ps.rows * ps.a_words;
+    uint32_t *t_id = Cs2 + 2 * (size_t)ps.rows * ps.c_words;
     uint32_t *t_j = t_id + PANEL_GROUP;
     uint32_t *t_k = t_j + PANEL_GROUP;
     float *t_b = reinterpret_cast<float *>(t_k + PANEL_GROUP);
@@ -439,26 +454,41 @@ __global__ void __launch_bounds__(PANEL_THREADS) panel_kernel(CampaignParams p, 
         unsigned long long hash = 0ull;
 
         const uint32_t p_beg = ch * panels_per_chunk, p_end = min(n_panels, p_beg + panels_per_chunk);
+        // Panel pn of A and C into buffer `buf`, asynchronously (cp.async, one group per panel). A panel's rows
+        // are contiguous in global memory and are kept that way in shared memory: a flat copy in 16-byte pieces
+        // (4-byte pieces for C when its panel does not start or end on a 16-byte boundary).
+        auto stage = [&](uint32_t pn, uint32_t buf) {
+            const uint32_t row0 = pn * (uint32_t)ps.rows;
+            if (row0 >= (uint32_t)p.M) return;                 // no such panel: nothing to copy
+            const uint32_t rows = min((uint32_t)ps.rows, (uint32_t)p.M - row0);
+            const unsigned char *Ag = reinterpret_cast<const unsigned char *>(p.A) + (size_t)row0 * p.K * es;
+            const uint32_t a_dst = (uint32_t)__cvta_generic_to_shared(As2 + (size_t)buf * ps.rows * ps.a_words);
+            const uint32_t a_pieces = rows * (uint32_t)ps.a_words / 4;
+            for (uint32_t i = tid; i < a_pieces; i += PANEL_THREADS) cp_async_16(a_dst + 16 * i, Ag + 16 * (size_t)i);
+            const float *Cg = p.C + (size_t)row0 * p.N;
+            const uint32_t c_dst = (uint32_t)__cvta_generic_to_shared(Cs2 + (size_t)buf * ps.rows * ps.c_words);
+            const uint32_t c_words = rows * (uint32_t)p.N;
+            if (((reinterpret_cast<uintptr_t>(Cg) | c_words * 4u) & 15u) == 0) {
+                for (uint32_t i = tid; i < c_words / 4; i += PANEL_THREADS) cp_async_16(c_dst + 16 * i, Cg + 4 * (size_t)i);
+            } else {
+                for (uint32_t i = tid; i < c_words; i += PANEL_THREADS) cp_async_4(c_dst + 4 * i, Cg + i);
+            }
+            cp_async_commit();
+        };
+        __syncthreads();           // nobody still reads the panels of the previous item
+        // (the chunk count is rounded up: the last items of a launch may have no panel at all)
+        if (p_beg < p_end) stage(p_beg, 0);
         for (uint32_t pn = p_beg; pn < p_end; ++pn) {
+            const uint32_t buf = (pn - p_beg) & 1u;
             const uint32_t row0 = pn * (uint32_t)ps.rows;
             const uint32_t rows = min((uint32_t)ps.rows, (uint32_t)p.M - row0);
-            __syncthreads();       // the previous panel is no longer read
-            // stage the A and C rows of this panel (global reads in 16-byte pieces, rows padded in smem)
-            const uint32_t a_vec = (uint32_t)(p.K * es) / 16;     // K * es is a multiple of 16
-            const uint4 *Ag = reinterpret_cast<const uint4 *>(reinterpret_cast<const unsigned char *>(p.A) + (size_t)row0 * p.K * es);
-            for (uint32_t i = tid; i < rows * a_vec; i += PANEL_THREADS) {
-                const uint32_t r = i / a_vec, v = i % a_vec;
-                const uint4 x = __ldg(Ag + (size_t)r * a_vec + v);
-                uint32_t *dst = As + (size_t)r * ps.a_words + 4 * v;
-                dst[0] = x.x; dst[1] = x.y; dst[2] = x.z; dst[3] = x.w;
-            }
-            const float *Cg = p.C + (size_t)row0 * p.N;
-            for (uint32_t i = tid; i < rows * (uint32_t)p.N; i += PANEL_THREADS) {
-                const uint32_t r = i / (uint32_t)p.N, c = i % (uint32_t)p.N;
-                Cs[(size_t)r * ps.c_words + c] = f32_bits(Cg[i]);
-            }
-            __syncthreads();
+            // the next panel starts to arrive in the other buffer (last read two panels ago) ...
+            if (pn + 1 < p_end) { stage(pn + 1, buf ^ 1u); cp_async_wait_all_but_one(); }
+            else cp_async_wait_all();
+            __syncthreads();       // ... and this one is complete for every thread
             if (have) {
+                const uint32_t *As = As2 + (size_t)buf * ps.rows * ps.a_words;
+                const uint32_t *Cs = Cs2 + (size_t)buf * ps.rows * ps.c_words;
                 const uint32_t lin_base = row0 * (uint32_t)p.N + my_j;
                 if (p.dtype == MPGEMMFI_FP16)
                     panel_rows<MPGEMMFI_FP16>(As, Cs, ps, rows, lin_base, (uint32_t)p.N, my_j, my_k, my_b, my_bf, do_bound, do_corr, n_det, first, hash, maxdev, changed);
@@ -467,6 +497,7 @@ __global__ void __launch_bounds__(PANEL_THREADS) panel_kernel(CampaignParams p, 
                 else
                     panel_rows<MPGEMMFI_TF32>(As, Cs, ps, rows, lin_base, (uint32_t)p.N, my_j, my_k, my_b, my_bf, do_bound, do_corr, n_det, first, hash, maxdev, changed);
             }
+            __syncthreads();       // this buffer may be overwritten by the panel after the next
         }
         // merge this item's statistics into the trial's record
         if (have) {
@@ -588,7 +619,7 @@ cudaError_t launch_campaign_trials(const CampaignParams &p, int num_sms, cudaStr
     // B-site trials: by row panel when a useful panel fits in shared memory and the columns are long;
     // otherwise one CTA per trial, in the same launch as the A-site trials
     const PanelShape ps = panel_shape(p.dtype, p.N, p.K, 227 * 1024);
-    const bool by_panel = ps.rows >= 64 && p.M >= 16 * ps.rows;
+    const bool by_panel = ps.rows >= 32 && p.M >= 16 * ps.rows;
     vector_kernel<<<grid_v, VEC_THREADS, 0, stream>>>(p, by_panel ? 0 : 1);
     if (by_panel) {
         static bool configured[64] = {};
