@@ -139,13 +139,29 @@ __global__ void __launch_bounds__(256) element_kernel(CampaignParams p)
             }
             float acc_c = 0.0f, acc_f = 0.0f;
             before = 0; after = 0;
-            // product of term k0 + lane, fetched one 32-term chunk ahead of its use
-            auto fetch = [&](uint32_t k0) -> float {
-                const uint32_t k = k0 + lane;
-                if (k >= (uint32_t)p.K) return 0.0f;
-                const float a = widen_operand(p.dtype, load_operand(p.dtype, p.A, (size_t)s.row * p.K + k));
-                const float b = widen_operand(p.dtype, load_operand(p.dtype, p.Bt, (size_t)s.col * p.K + k));
-                return __fmul_rn(a, b);
+            // Chunks of 128 terms: lane l holds terms k0 + 4 l .. k0 + 4 l + 3 (one 16- or 8-byte load per
+            // operand), fetched two chunks ahead of their use: the rows come from L2 or HBM, a microsecond
+            // away, and with a single 32-term chunk in flight that latency was the whole run time of a trial.
+            const bool wide = p.dtype == MPGEMMFI_TF32;
+            const unsigned char *a_row = reinterpret_cast<const unsigned char *>(p.A) + (size_t)s.row * p.K * (wide ? 4 : 2);
+            const unsigned char *b_row = reinterpret_cast<const unsigned char *>(p.Bt) + (size_t)s.col * p.K * (wide ? 4 : 2);
+            struct Raw { uint32_t a[4], b[4]; };
+            auto fetch = [&](uint32_t k0, Raw &r) {
+                const uint32_t k = k0 + 4u * (uint32_t)lane;
+                r.a[0] = r.a[1] = r.a[2] = r.a[3] = 0u;
+                r.b[0] = r.b[1] = r.b[2] = r.b[3] = 0u;
+                if (k >= (uint32_t)p.K) return;            // K is a multiple of 4 (16-byte rows): groups of 4 are whole
+                if (wide) {
+                    const uint4 x = __ldg(reinterpret_cast<const uint4 *>(a_row) + (k >> 2));
+                    const uint4 y = __ldg(reinterpret_cast<const uint4 *>(b_row) + (k >> 2));
+                    r.a[0] = x.x; r.a[1] = x.y; r.a[2] = x.z; r.a[3] = x.w;
+                    r.b[0] = y.x; r.b[1] = y.y; r.b[2] = y.z; r.b[3] = y.w;
+                } else {
+                    const uint2 x = __ldg(reinterpret_cast<const uint2 *>(a_row) + (k >> 2));
+                    const uint2 y = __ldg(reinterpret_cast<const uint2 *>(b_row) + (k >> 2));
+                    r.a[0] = x.x & 0xFFFFu; r.a[1] = x.x >> 16; r.a[2] = x.y & 0xFFFFu; r.a[3] = x.y >> 16;
+                    r.b[0] = y.x & 0xFFFFu; r.b[1] = y.x >> 16; r.b[2] = y.y & 0xFFFFu; r.b[3] = y.y >> 16;
+                }
             };
             auto site_hook = [&]() {
                 if (s.kind == MPGEMMFI_SITE_ACC) {
@@ -160,27 +176,38 @@ __global__ void __launch_bounds__(256) element_kernel(CampaignParams p)
                     acc_f = __fadd_rn(__fsub_rn(acc_f, re2), bits_f32(fin));
                 }
             };
-            float prod_next = fetch(0);
-            for (uint32_t k0 = 0; k0 < (uint32_t)p.K; k0 += 32) {
-                const float prod = prod_next;
-                prod_next = fetch(k0 + 32);
-                const uint32_t n_here = min(32u, (uint32_t)p.K - k0);
-                if (n_here == 32 && (kb <= k0 || kb > k0 + 32)) {
+            Raw r0, r1, r2;
+            fetch(0, r0);
+            fetch(128, r1);
+            for (uint32_t k0 = 0; k0 < (uint32_t)p.K; k0 += 128) {
+                fetch(k0 + 256, r2);
+                float pr[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) pr[q] = __fmul_rn(widen_operand(p.dtype, r0.a[q]), widen_operand(p.dtype, r0.b[q]));
+                const uint32_t n_here = min(128u, (uint32_t)p.K - k0);
+                if (n_here == 128 && (kb <= k0 || kb > k0 + 128)) {
                     // whole chunk, the site does not fall inside it: straight-line additions in k order
 #pragma unroll
                     for (uint32_t j = 0; j < 32; ++j) {
-                        const float pj = __shfl_sync(0xFFFFFFFFu, prod, j);
-                        acc_c = __fadd_rn(acc_c, pj);
-                        acc_f = __fadd_rn(acc_f, pj);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float pj = __shfl_sync(0xFFFFFFFFu, pr[q], j);
+                            acc_c = __fadd_rn(acc_c, pj);
+                            acc_f = __fadd_rn(acc_f, pj);
+                        }
                     }
                 } else {
-                    for (uint32_t j = 0; j < n_here; ++j) {
-                        const float pj = __shfl_sync(0xFFFFFFFFu, prod, j);
-                        acc_c = __fadd_rn(acc_c, pj);
-                        acc_f = __fadd_rn(acc_f, pj);
-                        if (k0 + j + 1 == kb) site_hook();
+                    for (uint32_t t4 = 0; t4 < n_here; t4 += 4) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float pj = __shfl_sync(0xFFFFFFFFu, pr[q], t4 >> 2);
+                            acc_c = __fadd_rn(acc_c, pj);
+                            acc_f = __fadd_rn(acc_f, pj);
+                            if (k0 + t4 + (uint32_t)q + 1 == kb) site_hook();
+                        }
                     }
                 }
+                r0 = r1; r1 = r2;
             }
             clean_bits = f32_bits(acc_c);
             value_bits = f32_bits(acc_f);
