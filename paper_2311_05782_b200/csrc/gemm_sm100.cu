@@ -111,6 +111,12 @@ __device__ __forceinline__ mpgemmfi_site listed_site(const TileCtx &c, uint32_t 
 __device__ uint32_t scan_next_operand(const TileCtx &c, uint32_t kt_from, int lane)
 {
     const uint32_t sh = kshift_of(c.p->dtype);
+    if (c.ctl->site_count == 1) {          // the usual table: one site, no loop and no warp-wide reduction
+        const mpgemmfi_site s = c.ctl->site_cache[0];
+        const bool hit = (s.kind == MPGEMMFI_SITE_A && in_own_rows(c, s.row)) ||
+                         (s.kind == MPGEMMFI_SITE_B && in_own_b(c, s.col));
+        return (hit && (s.k >> sh) >= kt_from) ? s.k >> sh : NONE;
+    }
     uint32_t best = NONE;
     for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
         const mpgemmfi_site s = listed_site(c, i);
@@ -124,6 +130,14 @@ __device__ uint32_t scan_next_operand(const TileCtx &c, uint32_t kt_from, int la
 // smallest boundary >= b_from at which this tile has an accumulator / term site (warp-wide)
 __device__ uint32_t scan_next_boundary(const TileCtx &c, uint32_t b_from, int lane)
 {
+    if (c.ctl->site_count == 1) {
+        const mpgemmfi_site s = c.ctl->site_cache[0];
+        if ((s.kind == MPGEMMFI_SITE_ACC || s.kind == MPGEMMFI_SITE_TERM) && in_tile_rows(c, s.row) && in_tile_cols(c, s.col)) {
+            const uint32_t b = site_boundary(s, c.p->dtype, c.p->K);
+            if (b >= b_from) return b;
+        }
+        return NONE;
+    }
     uint32_t best = NONE;
     for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
         const mpgemmfi_site s = listed_site(c, i);
@@ -138,6 +152,10 @@ __device__ uint32_t scan_next_boundary(const TileCtx &c, uint32_t b_from, int la
 
 __device__ bool scan_has_out(const TileCtx &c, int lane)
 {
+    if (c.ctl->site_count == 1) {
+        const mpgemmfi_site s = c.ctl->site_cache[0];
+        return s.kind == MPGEMMFI_SITE_OUT && in_own_rows(c, s.row) && in_tile_cols(c, s.col);
+    }
     bool any = false;
     for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
         const mpgemmfi_site s = listed_site(c, i);
