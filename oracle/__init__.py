@@ -71,6 +71,8 @@ def lib():
         vp = C.c_void_p
         L.orc_gemm.restype = C.c_int
         L.orc_gemm.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp, vp]
+        L.orc_gemm_addend.restype = C.c_int
+        L.orc_gemm_addend.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp, vp]
         L.orc_campaign.restype = C.c_int
         L.orc_campaign.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, vp]
         L.orc_sample.restype = C.c_int
@@ -149,8 +151,10 @@ def num_threads():
 
 # ---------------------------------------------------------------- matrix entry points
 
-def gemm(dtype, A, Bt, sites=None, detect_mode=0, kstep=None):
-    """Full-recompute fault-injected GEMM. Returns (C, header[16], site_log, bitmap[M, ceil(N/32)])."""
+def gemm(dtype, A, Bt, sites=None, detect_mode=0, kstep=None, addend=None):
+    """Full-recompute fault-injected GEMM. Returns (C, header[16], site_log, bitmap[M, ceil(N/32)]).
+
+    addend: optional M x N FP32 matrix, the C of D = A x B + C (Section II-B): every running sum starts from it."""
     A = _storage(A, dtype)
     Bt = _storage(Bt, dtype)
     M, K = A.shape
@@ -162,8 +166,14 @@ def gemm(dtype, A, Bt, sites=None, detect_mode=0, kstep=None):
     hdr = np.zeros(16, dtype=np.uint32)
     log = np.zeros(len(s), dtype=SITE_LOG)
     bitmap = np.zeros((M, (N + 31) // 32), dtype=np.uint32)
-    rc = lib().orc_gemm(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(Cm), _ptr(s), len(s), detect_mode, kstep,
-                        _ptr(hdr), _ptr(log), _ptr(bitmap))
+    if addend is None:
+        rc = lib().orc_gemm(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(Cm), _ptr(s), len(s), detect_mode, kstep,
+                            _ptr(hdr), _ptr(log), _ptr(bitmap))
+    else:
+        Cin = np.ascontiguousarray(addend, dtype=np.float32)
+        assert Cin.shape == (M, N)
+        rc = lib().orc_gemm_addend(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(Cin), _ptr(Cm), _ptr(s), len(s),
+                                   detect_mode, kstep, _ptr(hdr), _ptr(log), _ptr(bitmap))
     assert rc == 0
     return Cm, hdr, log, bitmap
 

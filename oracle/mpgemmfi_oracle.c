@@ -18,7 +18,7 @@
  * this file. It shares no code, header, table or constant with the CUDA path.
  *
  * Arithmetic: every element is accumulated as
- *     acc = +0;  for k = 0..K-1:  acc = fl32(acc + fl32(a_ik * b_kj))
+ *     acc = +0 (or the addend c_ij);  for k = 0..K-1:  acc = fl32(acc + fl32(a_ik * b_kj))
  * in IEEE binary32, round-to-nearest-even, no fused multiply-add (build with
  * -ffp-contract=off). There is no blocking of the k loop and no reordering of
  * the additions of one element; the only loop interchange is across
@@ -28,7 +28,8 @@
  * of Section V-B, exhaustive exponent sweeps of the three checks against
  * their Section VI-C bit-level forms, closed forms for bit flips, exact integer
  * GEMMs, linearity of operand faults, Eq. 1-2 exactness, brute-force flag
- * bitmaps. No function here is "parity unpinned".
+ * bitmaps; the addend form against a GEMM cut in two along k, exact integers
+ * and a per-element Python loop. No function here is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -186,11 +187,12 @@ static inline uint32_t term_boundary(uint32_t k, int kstep, int K)
  * sites of this element applied at their boundaries, in table order.
  * a[K], b[K]: widened operands (operand faults already applied).
  * idx[n_idx]: indices into sites[] of this element's ACC/TERM sites, ascending.
+ * acc0: what the running sum starts from (+0, or the addend c_ij of D = A x B + C, Section II-B).
  */
 static float element_with_sites(const float *a, const float *b, int K, int kstep, int detect_mode,
-                                const orc_site *sites, const int *idx, int n_idx, orc_site_log *log)
+                                const orc_site *sites, const int *idx, int n_idx, orc_site_log *log, float acc0)
 {
-    float acc = 0.0f;
+    float acc = acc0;
     for (int k = 0; k < K; ++k) {
         float p = a[k] * b[k];
         acc = acc + p;
@@ -319,16 +321,19 @@ static uint32_t output_check(int detect_mode, uint32_t bits, int bound, int *det
 /* ------------------------------------------------------------------ full GEMM (the definition) */
 
 /*
- * C = A x B with every site of the table applied (full recompute), then the
+ * C = A x B (+ addend) with every site of the table applied (full recompute), then the
  * output check. A: M x K, Bt: N x K (B stored K-major), C: M x N, FP32.
+ * addend (M x N FP32, or NULL): the C of D = A x B + C (Section II-B). On the paper's platform it is
+ * the accumulator the products are added to, so here every running sum starts from addend[i,j]
+ * instead of +0 and then takes the K products in k order as before.
  * hdr[16]: [0] status, [1] n_detected, [2] n_corrected, [3] sites applied,
  * [4] sites skipped. log[n_faults]. bitmap[M * ceil(N/32)]: bit j%32 of word
  * i*ceil(N/32) + j/32 set iff element (i,j) was detected.
  * Returns 0, or -1 on allocation failure.
  */
-int orc_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C,
-             const orc_site *sites, int n_faults, int detect_mode, int kstep,
-             uint32_t *hdr, orc_site_log *log, uint32_t *bitmap)
+static int gemm_impl(int dtype, int M, int N, int K, const void *A, const void *Bt, const float *addend, float *C,
+                     const orc_site *sites, int n_faults, int detect_mode, int kstep,
+                     uint32_t *hdr, orc_site_log *log, uint32_t *bitmap)
 {
     size_t wpr = ((size_t)N + 31) / 32;
     if (hdr) memset(hdr, 0, 16 * sizeof(uint32_t));
@@ -383,7 +388,7 @@ int orc_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
 #pragma omp parallel for schedule(dynamic, 4)
     for (int i = 0; i < M; ++i) {
         float *c = &C[(size_t)i * N];
-        for (int j = 0; j < N; ++j) c[j] = 0.0f;
+        for (int j = 0; j < N; ++j) c[j] = addend ? addend[(size_t)i * N + j] : 0.0f;
         for (int k = 0; k < K; ++k) {
             float a = Af[(size_t)i * K + k];
             const float *b = &BfT[(size_t)k * N];
@@ -408,7 +413,8 @@ int orc_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
         }
         C[(size_t)s->row * N + s->col] =
             element_with_sites(&Af[(size_t)s->row * K], &Bf[(size_t)s->col * K], K, kstep, detect_mode,
-                               sites, idx, n_idx, log);
+                               sites, idx, n_idx, log,
+                               addend ? addend[(size_t)s->row * N + s->col] : 0.0f);
     }
     free(idx); free(done);
 
@@ -456,6 +462,21 @@ int orc_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
     free(Af); free(Bf); free(BfT); free(EA); free(EB);
 #undef OUT_BOUND
     return 0;
+}
+
+int orc_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C,
+             const orc_site *sites, int n_faults, int detect_mode, int kstep,
+             uint32_t *hdr, orc_site_log *log, uint32_t *bitmap)
+{
+    return gemm_impl(dtype, M, N, K, A, Bt, NULL, C, sites, n_faults, detect_mode, kstep, hdr, log, bitmap);
+}
+
+/* D = A x B + C_in (Section II-B); C_in and D are M x N FP32 and must not overlap. */
+int orc_gemm_addend(int dtype, int M, int N, int K, const void *A, const void *Bt, const float *C_in, float *D,
+                    const orc_site *sites, int n_faults, int detect_mode, int kstep,
+                    uint32_t *hdr, orc_site_log *log, uint32_t *bitmap)
+{
+    return gemm_impl(dtype, M, N, K, A, Bt, C_in, D, sites, n_faults, detect_mode, kstep, hdr, log, bitmap);
 }
 
 /* ------------------------------------------------------------------ single trials (incremental mode) */
@@ -517,7 +538,7 @@ int orc_campaign(int dtype, int M, int N, int K, const void *A, const void *Bt, 
             orc_site_log lg; int idx0 = 0;
             orc_site one = *s;
             float v = element_with_sites(&Af[(size_t)s->row * K], &Bf[(size_t)s->col * K], K, kstep,
-                                         detect_mode, &one, &idx0, 1, &lg);
+                                         detect_mode, &one, &idx0, 1, &lg, 0.0f);
             r->primary_index = lin; r->before_bits = lg.before_bits; r->after_bits = lg.after_bits;
             trial_account(&ta, detect_mode, v, C_clean[lin], lin, &r->final_bits);
         } else {

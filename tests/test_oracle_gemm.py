@@ -326,3 +326,79 @@ def test_summary_bruteforce_and_bin_edges():
     r["max_abs_dev"] = [1.0, 1.9999999, 2.0, 2.0 ** -126, 2.0 ** -127, np.inf]
     h = orc.summary(r)[16:]
     assert h[127] == 2 and h[128] == 1 and h[1] == 1 and h[0] == 1 and h[255] == 1 and h.sum() == 6
+
+
+# ---------------------------------------------------------------- D = A x B + C (Section II-B)
+
+@pytest.mark.parametrize("dtype", [orc.FP16, orc.BF16, orc.TF32])
+def test_addend_exact_integers_and_zero_operand(dtype):
+    """Small integers: D = A x B + C exactly (a sign slip or a dropped addend shows); A = 0 gives D = C word for word."""
+    M, N, K = 5, 7, 11
+    a, b, A, Bt = int_operands(dtype, M, N, K, 21)
+    rng = np.random.default_rng(22)
+    cin = rng.integers(-100, 101, size=(M, N)).astype(np.float32)
+    D, hdr, _, bm = orc.gemm(dtype, A, Bt, addend=cin)
+    assert np.array_equal(D.astype(np.int64), a.astype(np.int64) @ b.astype(np.int64).T + cin.astype(np.int64))
+    assert hdr[1] == 0 and not bm.any()
+    cin = rng.standard_normal((M, N)).astype(np.float32)
+    D, *_ = orc.gemm(dtype, np.zeros_like(A), Bt, addend=cin)
+    assert np.array_equal(D.view(np.uint32), cin.view(np.uint32))
+
+
+@pytest.mark.parametrize("dtype", [orc.FP16, orc.BF16, orc.TF32])
+def test_addend_continues_an_accumulation(dtype):
+    """A GEMM cut in two along k, the second half taking the first half's output as its addend, is the uncut
+    GEMM bit for bit (one running sum in k order), and differs from summing the two halves separately."""
+    M, N, K, K1 = 6, 9, 96, 40
+    rng = np.random.default_rng(23)
+    A = synth.round_to_storage(rng.standard_normal((M, K)).astype(np.float32), dtype)
+    Bt = synth.round_to_storage(rng.standard_normal((N, K)).astype(np.float32), dtype)
+    whole, *_ = orc.gemm(dtype, A, Bt)
+    first, *_ = orc.gemm(dtype, np.ascontiguousarray(A[:, :K1]), np.ascontiguousarray(Bt[:, :K1]))
+    second, *_ = orc.gemm(dtype, np.ascontiguousarray(A[:, K1:]), np.ascontiguousarray(Bt[:, K1:]), addend=first)
+    assert np.array_equal(second.view(np.uint32), whole.view(np.uint32))
+    alone, *_ = orc.gemm(dtype, np.ascontiguousarray(A[:, K1:]), np.ascontiguousarray(Bt[:, K1:]))
+    assert not np.array_equal((first + alone).view(np.uint32), whole.view(np.uint32))
+
+
+def test_addend_scalar_loop_and_sites():
+    """Per-element Python loop in float32 starting from c_ij; an ACC site meets addend + partial sum, a TERM
+    site's write-back and an OUT site act on sums that include the addend."""
+    dtype, M, N, K = orc.BF16, 4, 5, 130
+    rng = np.random.default_rng(24)
+    A = synth.round_to_storage(rng.standard_normal((M, K)).astype(np.float32), dtype)
+    Bt = synth.round_to_storage(rng.standard_normal((N, K)).astype(np.float32), dtype)
+    cin = (rng.standard_normal((M, N)) * 3).astype(np.float32)
+    af = (A.astype(np.uint32) << 16).view(np.float32)
+    bf = (Bt.astype(np.uint32) << 16).view(np.float32)
+
+    def chain(i, j, upto):
+        acc = np.float32(cin[i, j])
+        for k in range(upto):
+            acc = np.float32(acc + np.float32(af[i, k] * bf[j, k]))
+        return acc
+
+    D, *_ = orc.gemm(dtype, A, Bt, addend=cin)
+    for i in range(M):
+        for j in range(N):
+            assert f32_bits(D[i, j]) == f32_bits(chain(i, j, K))
+    # ACC site at boundary 64 of element (1, 2): the word flipped is addend + 64 products
+    sites = np.concatenate([site(orc.KIND_ACC, 1, 2, 64, 1 << 20), site(orc.KIND_OUT, 3, 4, 0, 1 << 31),
+                            site(orc.KIND_TERM, 2, 0, 70, 1 << 22)])
+    D2, hdr, log, _ = orc.gemm(dtype, A, Bt, sites, addend=cin)
+    assert log[0]["before_bits"] == f32_bits(chain(1, 2, 64)) and log[0]["after_bits"] == log[0]["before_bits"] ^ (1 << 20)
+    acc = np.float32(bits_f32(int(log[0]["after_bits"])))
+    for k in range(64, K):
+        acc = np.float32(acc + np.float32(af[1, k] * bf[2, k]))
+    assert f32_bits(D2[1, 2]) == f32_bits(acc)
+    assert f32_bits(D2[3, 4]) == f32_bits(D[3, 4]) ^ (1 << 31)
+    # TERM site on term 70: written back at boundary 128 into addend + 128 products (Eq. 1-2)
+    p = np.float32(af[2, 70] * bf[0, 70])
+    pe = np.float32(bits_f32(f32_bits(p) ^ (1 << 22)))
+    acc = np.float32(np.float32(chain(2, 0, 128) - p) + pe)
+    for k in range(128, K):
+        acc = np.float32(acc + np.float32(af[2, k] * bf[0, k]))
+    assert f32_bits(D2[2, 0]) == f32_bits(acc)
+    untouched = np.ones((M, N), dtype=bool)
+    untouched[1, 2] = untouched[3, 4] = untouched[2, 0] = False
+    assert np.array_equal(D2[untouched].view(np.uint32), D[untouched].view(np.uint32)) and hdr[3] == 3
