@@ -207,6 +207,22 @@ int mpgemmfi_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt,
                   uint32_t *flags_out, mpgemmfi_stream stream);
 
 /*
+ * The same with an addend: D = A x B + C_in, the form the paper states the tensor-core operation in
+ * (Section II-B). C_in is the accumulator the products are added to: every running sum starts from
+ * c_in[i,j] instead of +0, so an ACC site at boundary k meets c_in[i,j] plus the first k products,
+ * a TERM site's write-back (Eq. 1-2) acts on a sum that holds the addend, and OUT sites and the
+ * output check see the finished d[i,j].
+ *   C_in   device pointer, M x N FP32 row-major, 4-byte aligned (16-byte alignment and N a
+ *          multiple of 4 let it be read 16 bytes at a time). It may be D itself (in place);
+ *          any other overlap of the two matrices is refused with ERR_ARG.
+ *   D      device pointer, M x N FP32 row-major, written in full.
+ * Everything else as for mpgemmfi_gemm. Campaigns take no addend.
+ */
+int mpgemmfi_gemm_addend(int dtype, int M, int N, int K, const void *A, const void *Bt, const float *C_in,
+                         float *D, const mpgemmfi_site *fault_sites, int n_faults, int detect_mode,
+                         uint32_t *flags_out, mpgemmfi_stream stream);
+
+/*
  * Largest FP32 exponent field of each row of a rows x K operand matrix (A, or Bt): out[r] in
  * 0..255; 0 for an all-zero row, 255 if the row holds Inf or NaN. X and out are device pointers
  * (X 16-byte aligned, K * element size a multiple of 16 bytes). Input of mpgemmfi_gemm_ranged.

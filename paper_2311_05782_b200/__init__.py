@@ -18,5 +18,5 @@ from .binding import (  # noqa: F401
     mpgemmfi_flags_bitmap_offset, mpgemmfi_campaign_workspace_bytes,
     mpgemmfi_validate_sites, mpgemmfi_strerror, mpgemmfi_last_cuda_error, mpgemmfi_version,
     gemm, campaign, split_flags, mpgemmfi_campaign_summary, campaign_summary,
-    mpgemmfi_operand_exponents, mpgemmfi_gemm_ranged,
+    mpgemmfi_operand_exponents, mpgemmfi_gemm_ranged, mpgemmfi_gemm_addend,
 )

@@ -45,6 +45,7 @@ _SYMBOLS = [
     "mpgemmfi_flags_bitmap_offset", "mpgemmfi_campaign_workspace_bytes", "mpgemmfi_validate_sites",
     "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version", "mpgemmfi_campaign_static",
     "mpgemmfi_set_tile_policy", "mpgemmfi_set_split_policy", "mpgemmfi_campaign_summary", "mpgemmfi_operand_exponents", "mpgemmfi_gemm_ranged",
+    "mpgemmfi_gemm_addend",
 ]
 
 
@@ -77,6 +78,8 @@ def load_library():
     vp, i, sz = C.c_void_p, C.c_int, C.c_size_t
     L.mpgemmfi_gemm.restype = i
     L.mpgemmfi_gemm.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp]
+    L.mpgemmfi_gemm_addend.restype = i
+    L.mpgemmfi_gemm_addend.argtypes = [i, i, i, i, vp, vp, vp, vp, vp, i, i, vp, vp]
     L.mpgemmfi_campaign.restype = i
     L.mpgemmfi_campaign.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp, sz, vp]
     L.mpgemmfi_campaign_static.restype = i
@@ -115,6 +118,12 @@ def mpgemmfi_gemm(dtype, M, N, K, A, Bt, C_out, fault_sites, n_faults, detect_mo
     """Raw call: every matrix argument is a device address (int), `stream` a cudaStream_t handle (int)."""
     return load_library().mpgemmfi_gemm(dtype, M, N, K, A, Bt, C_out, fault_sites, n_faults, detect_mode,
                                         flags_out, stream)
+
+
+def mpgemmfi_gemm_addend(dtype, M, N, K, A, Bt, C_in, D, fault_sites, n_faults, detect_mode, flags_out, stream):
+    """Raw call of D = A x B + C_in (device addresses; C_in may be D itself)."""
+    return load_library().mpgemmfi_gemm_addend(dtype, M, N, K, A, Bt, C_in, D, fault_sites, n_faults, detect_mode,
+                                               flags_out, stream)
 
 
 def mpgemmfi_campaign(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mode, records, workspace,
@@ -236,9 +245,10 @@ def _sites_tensor(sites, device):
     return (sites, sites.shape[0]) if sites.shape[0] else (None, 0)
 
 
-def gemm(dtype, A, Bt, sites=None, detect_mode=DETECT_NONE, C_out=None, flags_out=None, stream=None):
+def gemm(dtype, A, Bt, sites=None, detect_mode=DETECT_NONE, C_out=None, flags_out=None, stream=None, addend=None):
     """Fault-injected GEMM on CUDA tensors. Returns (C, flags) where flags is the raw uint32 buffer
-    (as an int32 tensor) laid out as documented in include/mpgemmfi.h; see split_flags()."""
+    (as an int32 tensor) laid out as documented in include/mpgemmfi.h; see split_flags().
+    addend: optional M x N float32 CUDA tensor, the C_in of D = A x B + C_in (it may be C_out itself)."""
     torch = _torch()
     _check_operand(A, dtype, "A")
     _check_operand(Bt, dtype, "Bt")
@@ -253,6 +263,8 @@ def gemm(dtype, A, Bt, sites=None, detect_mode=DETECT_NONE, C_out=None, flags_ou
         flags_out = torch.empty(mpgemmfi_flags_bytes(M, N, n_faults) // 4, dtype=torch.int32, device=A.device)
     stream_h = (torch.cuda.current_stream(A.device) if stream is None else stream).cuda_stream
     if detect_mode & OUTPUT_RANGE:
+        if addend is not None:
+            raise ValueError("the output-level range check takes no addend")
         # output-level range check: the exponent maxima of the (clean) operands come first
         ea = torch.empty(M, dtype=torch.int32, device=A.device)
         eb = torch.empty(N, dtype=torch.int32, device=A.device)
@@ -265,6 +277,15 @@ def gemm(dtype, A, Bt, sites=None, detect_mode=DETECT_NONE, C_out=None, flags_ou
                                   flags_out.data_ptr(), ea.data_ptr(), eb.data_ptr(), stream_h)
         if rc != 0:
             raise MpgemmfiError(rc, "mpgemmfi_gemm_ranged")
+        return C_out, flags_out
+    if addend is not None:
+        if addend.dtype != torch.float32 or tuple(addend.shape) != (M, N) or not addend.is_contiguous() or not addend.is_cuda:
+            raise ValueError("addend must be a contiguous M x N float32 CUDA tensor")
+        rc = mpgemmfi_gemm_addend(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), addend.data_ptr(), C_out.data_ptr(),
+                                  st.data_ptr() if st is not None else None, n_faults, detect_mode,
+                                  flags_out.data_ptr(), stream_h)
+        if rc != 0:
+            raise MpgemmfiError(rc, "mpgemmfi_gemm_addend")
         return C_out, flags_out
     rc = mpgemmfi_gemm(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), C_out.data_ptr(),
                        st.data_ptr() if st is not None else None, n_faults, detect_mode,

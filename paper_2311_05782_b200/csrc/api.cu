@@ -163,7 +163,7 @@ int check_common(int dtype, int M, int N, int K, const void *A, const void *Bt, 
 
 int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C, const mpgemmfi_site *sites,
              int n_faults, int detect_mode, uint32_t *flags, cudaStream_t stream, const DeviceInfo &di,
-             const uint32_t *exp_a = nullptr, const uint32_t *exp_bt = nullptr)
+             const uint32_t *exp_a = nullptr, const uint32_t *exp_bt = nullptr, const float *addend = nullptr)
 {
     int max_pairs = 0;
     const bool pair = choose_pair(dtype, M, N, &max_pairs);
@@ -195,6 +195,8 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
     }
     p.A = A; p.Bt = Bt; p.C = C; p.sites = sites; p.flags = flags;
     p.exp_a = exp_a; p.exp_b = exp_bt;
+    p.addend = addend;
+    p.addend_vec_ok = (N % 4 == 0) && (((uintptr_t)addend & 15) == 0);
     p.log2_k = 0;
     while ((1 << p.log2_k) < K) ++p.log2_k;
     const int walkers = pair ? max_pairs : di.num_sms;
@@ -255,6 +257,31 @@ int mpgemmfi_gemm_ranged(int dtype, int M, int N, int K, const void *A, const vo
     const bool ranged = (detect_mode & MPGEMMFI_OUTPUT_RANGE) != 0;
     return run_gemm(dtype, M, N, K, A, Bt, C, fault_sites, n_faults, detect_mode, flags_out,
                     static_cast<cudaStream_t>(stream), di, ranged ? exp_a : nullptr, ranged ? exp_bt : nullptr);
+}
+
+int mpgemmfi_gemm_addend(int dtype, int M, int N, int K, const void *A, const void *Bt, const float *C_in, float *D,
+                         const mpgemmfi_site *fault_sites, int n_faults, int detect_mode, uint32_t *flags_out,
+                         mpgemmfi_stream stream)
+{
+    int rc = check_common(dtype, M, N, K, A, Bt, D);
+    if (rc) return rc;
+    if (!C_in) return MPGEMMFI_ERR_ARG;
+    if ((uintptr_t)C_in & 3) return MPGEMMFI_ERR_ALIGN;
+    // in place (C_in == D) is fine: a tile's addend is read before anything of that tile is written;
+    // any other overlap would let one tile's stores reach another tile's addend
+    const uintptr_t c0 = (uintptr_t)C_in, d0 = (uintptr_t)D;
+    const size_t bytes = (size_t)M * (size_t)N * sizeof(float);
+    if (c0 != d0 && c0 < d0 + bytes && d0 < c0 + bytes) return MPGEMMFI_ERR_ARG;
+    if (n_faults < 0 || n_faults > MPGEMMFI_MAX_FAULTS || (n_faults > 0 && !fault_sites)) return MPGEMMFI_ERR_ARG;
+    if (detect_mode & ~(MPGEMMFI_DETECT_TECHNIQUE_MASK | MPGEMMFI_CORRECT)) return MPGEMMFI_ERR_ARG;
+    if (!flags_out && (n_faults > 0 || (detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK))) return MPGEMMFI_ERR_ARG;
+    if (((uintptr_t)fault_sites & 15) || ((uintptr_t)flags_out & 15)) return MPGEMMFI_ERR_ALIGN;
+    DeviceInfo di;
+    rc = device_info(di);
+    if (rc) return rc;
+    if (di.major != 10) return MPGEMMFI_ERR_ARCH;
+    return run_gemm(dtype, M, N, K, A, Bt, D, fault_sites, n_faults, detect_mode, flags_out,
+                    static_cast<cudaStream_t>(stream), di, nullptr, nullptr, C_in);
 }
 
 int mpgemmfi_operand_exponents(int dtype, int rows, int K, const void *X, uint32_t *out, mpgemmfi_stream stream)

@@ -74,7 +74,7 @@ struct alignas(16) Control {
     uint64_t acc_empty[2];
     uint64_t pause_full;
     uint64_t pause_done;
-    uint64_t acc_loaded;      // the accumulators of a continued tile part are back in TMEM
+    uint64_t acc_loaded[2];   // accumulator buffer s holds what its next segment starts from (a continued tile part, an addend)
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t site_count;
@@ -355,6 +355,13 @@ __device__ __forceinline__ bool get_segment(const GemmParams &p, uint32_t gid, u
     return true;
 }
 
+// Do the accumulators of this segment start from memory (the previous part's sums left in C, or the
+// addend of D = A x B + C at a tile's first k-tile) rather than from the first MMA's overwrite?
+__device__ __forceinline__ bool starts_from_memory(const GemmParams &p, const Segment &sg)
+{
+    return sg.load || (p.addend != nullptr && sg.kt0 == 0);
+}
+
 // does walker `gid` run tile t, whole or in part?
 __device__ __forceinline__ bool walker_has_tile(const GemmParams &p, uint32_t t, uint32_t gid, uint32_t groups)
 {
@@ -420,19 +427,23 @@ __device__ __forceinline__ bool signal_wait(const uint32_t *ptr, uint32_t want, 
 // previous part's walker that owns the same rows and columns (hand-over word *sig == want), then copy
 // rows row0..row0+31, columns col0..col0+32*pieces-1 of the accumulators it left in C back into TMEM
 // (this warp's lanes, columns from t_dst on). `park` is the warp's 2 KB of shared-memory staging.
+// With sig == nullptr nothing is waited for (an addend: the caller's matrix is there already); with
+// vec == false the source allows no 16-byte accesses and is read word by word.
 // The store transpose of the epilogue run backwards: every load instruction reads whole 128-byte rows
 // of C (lane l: 16-byte piece l % 8 of rows l / 8 + 4 it) and parks them in shared memory, then the
 // threads of one half-warp pick up their own rows. (One 128-byte row per thread instead: 11 us per
 // tile, during which the main loop next to it stood still.) Returns false when the wait gave up.
 __device__ __forceinline__ bool load_partial(const float *C, uint32_t M, uint32_t N, const uint32_t *sig, uint32_t want,
                                              volatile uint32_t *abort_flag, uint32_t row0, uint32_t col0, int pieces,
-                                             uint32_t t_dst, uint8_t *park, int lane)
+                                             uint32_t t_dst, uint8_t *park, int lane, bool vec = true)
 {
-    bool got = true;
-    if (lane == 0) got = signal_wait(sig, want, abort_flag);
-    got = __shfl_sync(0xFFFFFFFFu, got, 0);
-    if (!got) return false;
-    __threadfence();
+    if (sig) {
+        bool got = true;
+        if (lane == 0) got = signal_wait(sig, want, abort_flag);
+        got = __shfl_sync(0xFFFFFFFFu, got, 0);
+        if (!got) return false;
+        __threadfence();
+    }
     const uint32_t j = (uint32_t)lane & 7u;
 #pragma unroll 1
     for (int i = 0; i < pieces; ++i) {
@@ -445,7 +456,17 @@ __device__ __forceinline__ bool load_partial(const float *C, uint32_t M, uint32_
             for (int it = 0; it < 4; ++it) {
                 const uint32_t grow = row0 + (uint32_t)(16 * half + 4 * it) + ((uint32_t)lane >> 3);
                 x[it] = make_uint4(0u, 0u, 0u, 0u);
-                if (grow < M && col < N) x[it] = __ldcg(reinterpret_cast<const uint4 *>(C + (size_t)grow * N + col));
+                if (grow < M && col < N) {
+                    const float *src = C + (size_t)grow * N + col;
+                    if (vec) {
+                        x[it] = __ldcg(reinterpret_cast<const uint4 *>(src));
+                    } else {
+                        x[it].x = __float_as_uint(__ldcg(src));
+                        if (col + 1 < N) x[it].y = __float_as_uint(__ldcg(src + 1));
+                        if (col + 2 < N) x[it].z = __float_as_uint(__ldcg(src + 2));
+                        if (col + 3 < N) x[it].w = __float_as_uint(__ldcg(src + 3));
+                    }
+                }
             }
             __syncwarp();                               // the rows parked before have been picked up
 #pragma unroll
@@ -601,7 +622,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->acc_full[s]), 1); mbar_init(smem_u32(&ctl->acc_empty[s]), EPI_ARRIVALS); }
         mbar_init(smem_u32(&ctl->pause_full), 1);
         mbar_init(smem_u32(&ctl->pause_done), EPI_ARRIVALS);
-        mbar_init(smem_u32(&ctl->acc_loaded), EPI_ARRIVALS);
+        for (int s = 0; s < 2; ++s) mbar_init(smem_u32(&ctl->acc_loaded[s]), EPI_ARRIVALS);
         ctl->abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tm_a);
@@ -634,7 +655,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     // barriers of the leader CTA that this CTA's warps arrive on
     const uint32_t lead_acc_empty0 = kPair ? map_to_cta(smem_u32(&ctl->acc_empty[0]), 0) : smem_u32(&ctl->acc_empty[0]);
     const uint32_t lead_pause_done = kPair ? map_to_cta(smem_u32(&ctl->pause_done), 0) : smem_u32(&ctl->pause_done);
-    const uint32_t lead_acc_loaded = kPair ? map_to_cta(smem_u32(&ctl->acc_loaded), 0) : smem_u32(&ctl->acc_loaded);
+    const uint32_t lead_acc_loaded0 = kPair ? map_to_cta(smem_u32(&ctl->acc_loaded[0]), 0) : smem_u32(&ctl->acc_loaded[0]);
     Segment sg;
 
     if (warp == 0) {
@@ -723,15 +744,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             if (has_sites) { next_op = scan_next_operand(tc, sg.kt0, lane); next_b = scan_next_boundary(tc, sg.kt0 + 1, lane); }
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_empty[as]), ap ^ 1u, abort_flag));
             if (!ok) break;
-            if (sg.load) {
-                // continued tile: the epilogue warps put the earlier k-tiles' accumulators back first
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_loaded), loaded_phase, abort_flag));
+            const bool preloaded = starts_from_memory(p, sg);
+            if (preloaded) {
+                // continued tile or addend: the epilogue warps put the starting accumulators into TMEM first
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_loaded[as]), (loaded_phase >> as) & 1u, abort_flag));
                 if (!ok) break;
-                loaded_phase ^= 1u;
+                loaded_phase ^= 1u << as;
             }
             tc_fence_after_sync();
             const uint32_t d_tmem = tmem_base + as * BN;
-            const uint32_t fresh_kt = sg.load ? NONE : sg.kt0;      // the k-tile whose first MMA overwrites the accumulator
+            const uint32_t fresh_kt = preloaded ? NONE : sg.kt0;    // the k-tile whose first MMA overwrites the accumulator
             uint32_t kt = sg.kt0;
             while (kt < sg.kt1) {
               // k-tiles up to the next one with a site (an operand site in it, or an accumulator / term site
@@ -842,29 +864,37 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         const uint32_t my_signal = rank * EPI_WARPS + (uint32_t)(warp - 4);
         const uint32_t first_left = groups * (uint32_t)p.full_rounds;
         bool ok = true;
+        // This warp's share of what segment s starts from, into accumulator buffer `buf`: the sums the walker
+        // of the previous part left in C (after that walker's hand-over), or the addend.
+        auto preload = [&](const Segment &s, uint32_t buf) -> bool {
+            uint32_t tm, tn;
+            tile_coords(p, s.tile, tm, tn);
+            if (lane == 0) bulk_wait_read_all();       // the staging rows are free again
+            __syncwarp();
+            const uint32_t *sig = s.load ? p.signals + (size_t)(s.tile - first_left) * 16 + my_signal : nullptr;
+            const uint32_t t_dst = tmem_base + buf * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)(first * 32);
+            if (!load_partial(s.load ? p.C : p.addend, (uint32_t)p.M, (uint32_t)p.N, sig, (p.epoch << 3) | s.part, abort_flag,
+                              tm * TM + rank * BM + (uint32_t)(q * 32), tn * BN + (uint32_t)(first * 32), MY_PIECES,
+                              t_dst, my_out, lane, s.load || p.addend_vec_ok != 0))
+                return false;
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                if constexpr (kPair) mbar_arrive_cluster(lead_acc_loaded0 + buf * (uint32_t)sizeof(uint64_t));
+                else mbar_arrive(lead_acc_loaded0 + buf * (uint32_t)sizeof(uint64_t));
+            }
+            return true;
+        };
+        if (p.addend != nullptr && get_segment(p, gid, groups, 0, sg) && starts_from_memory(p, sg)) ok = preload(sg, 0u);
         for (uint32_t lt = 0; ok && get_segment(p, gid, groups, lt, sg); ++lt) {
             const uint32_t as = lt & 1u, ap = (lt >> 1) & 1u;
-            if (p.split_parts > 1) {
+            if (p.split_parts > 1 || p.addend != nullptr) {
                 // the other TMEM buffer is free (this warp has read its share of the segment before this
-                // one): if the next segment continues a tile, fetch its accumulators while this one runs
+                // one): if the next segment starts from memory, fetch its accumulators while this one runs
                 Segment nx;
-                if (get_segment(p, gid, groups, lt + 1, nx) && nx.load) {
-                    uint32_t tm, tn;
-                    tile_coords(p, nx.tile, tm, tn);
-                    if (lane == 0) bulk_wait_read_all();       // the staging rows are free again
-                    __syncwarp();
-                    const uint32_t *sig = p.signals + (size_t)(nx.tile - first_left) * 16 + my_signal;
-                    const uint32_t t_dst = tmem_base + ((lt + 1) & 1u) * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)(first * 32);
-                    ok = load_partial(p.C, (uint32_t)p.M, (uint32_t)p.N, sig, (p.epoch << 3) | nx.part, abort_flag,
-                                      tm * TM + rank * BM + (uint32_t)(q * 32), tn * BN + (uint32_t)(first * 32), MY_PIECES,
-                                      t_dst, my_out, lane);
+                if (get_segment(p, gid, groups, lt + 1, nx) && starts_from_memory(p, nx)) {
+                    ok = preload(nx, (lt + 1) & 1u);
                     if (!ok) break;
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if constexpr (kPair) mbar_arrive_cluster(lead_acc_loaded);
-                        else mbar_arrive(lead_acc_loaded);
-                    }
                 }
             }
             set_tile(sg.tile);

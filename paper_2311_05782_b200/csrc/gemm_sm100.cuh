@@ -25,6 +25,10 @@ struct GemmParams {
     const uint32_t *exp_a;
     const uint32_t *exp_b;
     int log2_k;
+    // Addend of D = A x B + C (null: none): M x N FP32 that every tile's accumulators start from. It may be
+    // the output itself (in place). addend_vec_ok: 16-byte aligned with a 16-byte row pitch.
+    const float *addend;
+    int addend_vec_ok;
     // Split schedule of the last round of tiles (split_parts <= 1: off). The tile walkers first share
     // out `full_rounds` whole tiles each; the `left_tiles` tiles that remain are cut along K into
     // `split_parts` parts run by different walkers, the accumulators travelling through C.

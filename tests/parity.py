@@ -54,26 +54,34 @@ def bits_f32(u):
     return np.array([u], dtype=np.uint32).view(np.float32)[0]
 
 
-def run_gpu_gemm(dtype, A, Bt, sites, mode):
+def run_gpu_gemm(dtype, A, Bt, sites, mode, addend=None, in_place=False):
     M, K = A.shape
     N = Bt.shape[0]
     n = 0 if sites is None else len(sites)
-    Cg, flags = mpg.gemm(dtype, to_dev(A, dtype), to_dev(Bt, dtype), sites, mode)
+    if addend is None:
+        Cg, flags = mpg.gemm(dtype, to_dev(A, dtype), to_dev(Bt, dtype), sites, mode)
+    else:
+        cin = torch.from_numpy(addend).cuda()
+        Cg, flags = mpg.gemm(dtype, to_dev(A, dtype), to_dev(Bt, dtype), sites, mode, addend=cin,
+                             C_out=cin if in_place else None)
     torch.cuda.synchronize()
     hdr, log, bm = mpg.split_flags(flags, M, N, n)
     return Cg.cpu().numpy(), hdr, log, bm
 
 
-def check_gemm_against_oracle(dtype, A, Bt, sites, mode, max_fragile=0):
-    """Full element-by-element comparison at sizes the oracle finishes quickly. Returns the number of fragile sites."""
+def check_gemm_against_oracle(dtype, A, Bt, sites, mode, max_fragile=0, addend=None, in_place=False):
+    """Full element-by-element comparison at sizes the oracle finishes quickly. Returns the number of fragile sites.
+    addend: the C_in of D = A x B + C_in (its magnitude joins the tolerance); in_place: D is written over it."""
     sites = np.zeros(0, dtype=orc.SITE) if sites is None else sites
     M, K = A.shape
     N = Bt.shape[0]
-    Cg, hdr_g, log_g, bm_g = run_gpu_gemm(dtype, A, Bt, sites, mode)
-    Co, hdr_o, log_o, bm_o = orc.gemm(dtype, A, Bt, sites, mode)
+    Cg, hdr_g, log_g, bm_g = run_gpu_gemm(dtype, A, Bt, sites, mode, addend, in_place)
+    Co, hdr_o, log_o, bm_o = orc.gemm(dtype, A, Bt, sites, mode, addend=addend)
     assert not (hdr_g[0] & mpg.STATUS_WAIT_LIMIT), "device wait limit hit"
     A2, B2 = faulted_operands(dtype, A, Bt, sites)
     tol = TOL * orc.absprod(dtype, A2, B2)
+    if addend is not None:
+        tol = tol + TOL * np.abs(addend).astype(np.float64)
 
     touched = np.zeros((M, N), dtype=bool)
     fragile = 0
