@@ -169,3 +169,27 @@ def test_addend_argument_errors():
     assert call(base + 64, base) == -1                  # partial overlap
     assert call(base, base) == 0 and call(base, base + 4 * 128 * 128) == 0
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_shapes_tables_and_modes_with_addend(seed, policies):
+    """Differential fuzz against the oracle: random shape, format, tiling, schedule, check mode, multi-bit site table
+    (repeats on one element, entries the device must skip), addend scale, in place or not."""
+    rng = np.random.default_rng(5000 + seed)
+    dtype = int(rng.integers(0, 3))
+    kt = synth.kstep(dtype)
+    unit = 4 if dtype == orc.TF32 else 8
+    M = int(rng.integers(1, 900)); N = int(rng.integers(1, 900)); K = unit * int(rng.integers(1, 60))
+    mode = int(rng.choice([orc.T_NONE, orc.T_BOUND, orc.T_BOUND | orc.CORRECT, orc.T_RMAX | orc.CORRECT, orc.T_RFLIP | orc.CORRECT]))
+    A, Bt = rand_operands(dtype, M, N, K, 6000 + seed)
+    cin = rand_addend(M, N, 7000 + seed, scale=float(rng.choice([0.0, 1.0, 100.0, 1.0e4])))   # (never near BoundCheck's threshold)
+    n = int(rng.integers(0, 40))
+    s = site_table(dtype, M, N, K, n, 8000 + seed)
+    width = np.where(s["kind"] <= orc.KIND_B, 19 if dtype == orc.TF32 else 16, 32)
+    nbits = rng.choice([1, 2, 4], n)
+    s["xor_mask"] = [(((1 << int(b)) - 1) << int(rng.integers(0, int(w) - int(b) + 1))) for b, w in zip(nbits, width)]
+    if n >= 4:
+        s[1] = s[0]; s["row"][2] = M + 5; s["kind"][3] = 7
+    assert mpg.mpgemmfi_set_tile_policy([mpg.TILES_AUTO, mpg.TILES_SINGLE, mpg.TILES_PAIR][seed % 3]) == 0
+    assert mpg.mpgemmfi_set_split_policy([mpg.SPLIT_AUTO, mpg.SPLIT_ON][seed % 2]) == 0
+    check_gemm_against_oracle(dtype, A, Bt, s, mode, max_fragile=2, addend=cin, in_place=bool(seed & 4))
