@@ -77,6 +77,8 @@ def lib():
         L.orc_campaign.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, vp]
         L.orc_sample.restype = C.c_int
         L.orc_sample.argtypes = [C.c_int] * 4 + [vp, vp, vp, C.c_int, vp, vp, C.c_int, vp, vp]
+        L.orc_sample_addend.restype = C.c_int
+        L.orc_sample_addend.argtypes = [C.c_int] * 4 + [vp, vp, vp, C.c_int, vp, vp, vp, C.c_int, vp, vp]
         L.orc_operand_exponents.restype = None
         L.orc_operand_exponents.argtypes = [C.c_int, C.c_int, C.c_int, vp, vp]
         L.orc_output_range_bound.restype = C.c_int
@@ -194,8 +196,10 @@ def campaign(dtype, A, Bt, C_clean, sites, detect_mode=0, kstep=None):
     return rec
 
 
-def sample(dtype, A, Bt, si, sj, sites=None):
-    """Clean (operand-faulted) C[i,j] and (|A||B|)_ij at sampled positions, any matrix size."""
+def sample(dtype, A, Bt, si, sj, sites=None, start=None):
+    """Clean (operand-faulted) C[i,j] and (|A||B|)_ij at sampled positions, any matrix size.
+    start: optional float32 value per sample that its running sum begins with (the addend c_ij of D = A x B + C);
+    its magnitude is added to the second result."""
     A = _storage(A, dtype)
     Bt = _storage(Bt, dtype)
     M, K = A.shape
@@ -205,7 +209,13 @@ def sample(dtype, A, Bt, si, sj, sites=None):
     s = _sites(sites)
     out = np.empty(len(si), dtype=np.float32)
     ap = np.empty(len(si), dtype=np.float64)
-    rc = lib().orc_sample(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(s), len(s), _ptr(si), _ptr(sj), len(si), _ptr(out), _ptr(ap))
+    if start is None:
+        rc = lib().orc_sample(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(s), len(s), _ptr(si), _ptr(sj), len(si), _ptr(out), _ptr(ap))
+    else:
+        st = np.ascontiguousarray(start, dtype=np.float32)
+        assert st.shape == (len(si),)
+        rc = lib().orc_sample_addend(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(s), len(s), _ptr(st), _ptr(si), _ptr(sj), len(si),
+                                     _ptr(out), _ptr(ap))
     assert rc == 0
     return out, ap
 

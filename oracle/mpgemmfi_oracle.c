@@ -574,17 +574,18 @@ int orc_campaign(int dtype, int M, int N, int K, const void *A, const void *Bt, 
  * Clean C[i,j] for n sampled (i,j) pairs straight from the storage matrices,
  * with the operand XORs of (optional) A/B sites applied, and (|A||B|)_ij in
  * double for tolerances. No matrix is widened as a whole.
+ * start (or NULL): start[t] is what sample t's running sum begins with, the addend c_ij of
+ * D = A x B + C (Section II-B); |start[t]| joins out_absprod[t].
  */
-int orc_sample(int dtype, int M, int N, int K, const void *A, const void *Bt,
-               const orc_site *sites, int n_faults,
-               const uint32_t *si, const uint32_t *sj, int n, float *out_c, double *out_absprod)
+static int sample_impl(int dtype, int K, const void *A, const void *Bt,
+                       const orc_site *sites, int n_faults, const float *start,
+                       const uint32_t *si, const uint32_t *sj, int n, float *out_c, double *out_absprod)
 {
-    (void)M; (void)N;
 #pragma omp parallel for schedule(dynamic, 16)
     for (int t = 0; t < n; ++t) {
         uint32_t i = si[t], j = sj[t];
-        float acc = 0.0f;
-        double ap = 0.0;
+        float acc = start ? start[t] : 0.0f;
+        double ap = start ? fabs((double)start[t]) : 0.0;
         for (int k = 0; k < K; ++k) {
             uint32_t sa = load_storage(dtype, A, (size_t)i * K + k);
             uint32_t sb = load_storage(dtype, Bt, (size_t)j * K + k);
@@ -602,6 +603,22 @@ int orc_sample(int dtype, int M, int N, int K, const void *A, const void *Bt,
         if (out_absprod) out_absprod[t] = ap;
     }
     return 0;
+}
+
+int orc_sample(int dtype, int M, int N, int K, const void *A, const void *Bt,
+               const orc_site *sites, int n_faults,
+               const uint32_t *si, const uint32_t *sj, int n, float *out_c, double *out_absprod)
+{
+    (void)M; (void)N;
+    return sample_impl(dtype, K, A, Bt, sites, n_faults, NULL, si, sj, n, out_c, out_absprod);
+}
+
+int orc_sample_addend(int dtype, int M, int N, int K, const void *A, const void *Bt,
+                      const orc_site *sites, int n_faults, const float *start,
+                      const uint32_t *si, const uint32_t *sj, int n, float *out_c, double *out_absprod)
+{
+    (void)M; (void)N;
+    return sample_impl(dtype, K, A, Bt, sites, n_faults, start, si, sj, n, out_c, out_absprod);
 }
 
 /* (|A||B|) for all elements, double precision; used only for tolerances at small sizes */

@@ -157,3 +157,43 @@ def test_large_configs_on_sampled_outputs(name):
         assert g["before_bits"] == int(Cc[int(s["row"]), int(s["col"])].view(np.uint32))
         assert g["after_bits"] == g["before_bits"] ^ s["xor_mask"]
         assert g["n_detected"] == orc.boundcheck_detect(int(g["after_bits"]))
+
+
+@pytest.mark.parametrize("name", ["c2", "c3a", "c4", "c5"])
+def test_full_size_addend_on_sampled_outputs(name):
+    """D = A x B + C_in at the benchmark's sizes and default launch configuration: sampled outputs against the oracle's
+    chains that start from the addend, no flags on a clean workload with a small addend, and the elements of an
+    accumulator / output site met by the addend-bearing sum."""
+    w = synth.make_workload(name, trials=16)
+    M, N, K = w.M, w.N, w.K
+    a, b = to_dev(w.A, w.dtype), to_dev(w.Bt, w.dtype)
+    g = torch.Generator(device="cuda"); g.manual_seed(99)
+    cin = torch.randn((M, N), dtype=torch.float32, device="cuda", generator=g)
+    kt = synth.kstep(w.dtype)
+    sites = np.zeros(2, dtype=orc.SITE)
+    sites["kind"] = [orc.KIND_ACC, orc.KIND_OUT]
+    sites["row"] = [M - 3, 130]; sites["col"] = [N - 2, 33]; sites["k"] = [kt, 0]; sites["xor_mask"] = [1 << 21, 1 << 31]
+    D, f = mpg.gemm(w.dtype, a, b, sites, w.detect_mode, addend=cin)
+    torch.cuda.synchronize()
+    hdr, log, bm = mpg.split_flags(f, M, N, 2)
+    assert hdr[0] == 0 and hdr[1] == 0 and hdr[3] == 2 and not bm.any()
+    rng = np.random.default_rng(6)
+    si = np.concatenate([rng.integers(0, M, 3000), [0, M - 1, 0, M - 1, 127, 128, 255, 256]]).astype(np.uint32)
+    sj = np.concatenate([rng.integers(0, N, 3000), [0, N - 1, N - 1, 0, N - 1, 0, 63, 32]]).astype(np.uint32)
+    ti, tj = torch.from_numpy(si.astype(np.int64)).cuda(), torch.from_numpy(sj.astype(np.int64)).cuda()
+    start = cin[ti, tj].cpu().numpy()
+    ref, ap = orc.sample(w.dtype, w.A, w.Bt, si, sj, start=start)
+    got = D[ti, tj].cpu().numpy()
+    hit = ((si == M - 3) & (sj == N - 2)) | ((si == 130) & (sj == 33))
+    assert close(got, ref, TOL * ap)[~hit].all()
+    # the accumulator site met addend + the first k-step's products; the output site the finished sum
+    i, j = M - 3, N - 2
+    c0 = np.array([float(cin[i, j].cpu())], dtype=np.float32)
+    r_acc, a_acc = orc.sample(w.dtype, np.ascontiguousarray(w.A[i:i + 1, :kt]), np.ascontiguousarray(w.Bt[j:j + 1, :kt]),
+                              np.zeros(1, np.uint32), np.zeros(1, np.uint32), start=c0)
+    assert close(bits_f32(log[0]["before_bits"]), r_acc[0], TOL * a_acc[0])
+    assert log[0]["after_bits"] == log[0]["before_bits"] ^ (1 << 21)
+    r_out, a_out = orc.sample(w.dtype, w.A, w.Bt, np.array([130], np.uint32), np.array([33], np.uint32),
+                              start=np.array([float(cin[130, 33].cpu())], dtype=np.float32))
+    assert close(bits_f32(log[1]["before_bits"]), r_out[0], TOL * a_out[0])
+    assert int(D[130, 33].cpu().numpy().view(np.uint32)) == int(log[1]["before_bits"]) ^ (1 << 31)

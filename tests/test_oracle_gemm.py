@@ -382,6 +382,12 @@ def test_addend_scalar_loop_and_sites():
     for i in range(M):
         for j in range(N):
             assert f32_bits(D[i, j]) == f32_bits(chain(i, j, K))
+    # sampled evaluation with a starting value per sample: the same chains, and |addend| joins the magnitude sum
+    si = np.array([0, 3, 2], dtype=np.uint32); sj = np.array([4, 0, 2], dtype=np.uint32)
+    sc, sap = orc.sample(dtype, A, Bt, si, sj, start=cin[si, sj])
+    assert [f32_bits(v) for v in sc] == [f32_bits(chain(int(i), int(j), K)) for i, j in zip(si, sj)]
+    ap = np.abs(af).astype(np.float64) @ np.abs(bf).astype(np.float64).T
+    assert np.allclose(sap, ap[si, sj] + np.abs(cin[si, sj]).astype(np.float64), rtol=1e-12)
     # ACC site at boundary 64 of element (1, 2): the word flipped is addend + 64 products
     sites = np.concatenate([site(orc.KIND_ACC, 1, 2, 64, 1 << 20), site(orc.KIND_OUT, 3, 4, 0, 1 << 31),
                             site(orc.KIND_TERM, 2, 0, 70, 1 << 22)])
