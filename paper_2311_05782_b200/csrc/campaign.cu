@@ -229,6 +229,17 @@ __global__ void __launch_bounds__(256) element_kernel(CampaignParams p)
 
 // A-site trials (row i fixed, walk the N columns) and, when with_b is set, B-site trials (column j
 // fixed, walk the M rows) in one launch: one CTA per trial, the A list first.
+// Eq. 1-2 on a finished sum c for an operand trial: remove the clean product x * y, add the faulty one xf * y,
+// every product and every sum rounded to FP32. The product of two FP16 values is exact in FP32 (22 significant
+// bits, magnitudes between 2^-48 and 2^32, so neither underflow nor overflow), and then a fused multiply-add
+// rounds once exactly where the separate sum would: the same bits (infinities, NaNs and signed zeros included)
+// for half the instructions. BF16 and TF32 products can leave FP32's range and keep the separate operations.
+__device__ __forceinline__ float operand_write_back(bool fp16, float c, float y, float x, float xf)
+{
+    if (fp16) return __fmaf_rn(xf, y, __fmaf_rn(-x, y, c));
+    return __fadd_rn(__fsub_rn(c, __fmul_rn(x, y)), __fmul_rn(xf, y));
+}
+
 __global__ void __launch_bounds__(VEC_THREADS) vector_kernel(CampaignParams p, int with_b)
 {
     __shared__ Stats warp_stats[VEC_THREADS / 32];
@@ -267,8 +278,7 @@ __global__ void __launch_bounds__(VEC_THREADS) vector_kernel(CampaignParams p, i
                 if (o < n_other) {
                     const float y = widen_operand(p.dtype, yw[u]);
                     const uint32_t lin = is_a ? s.row * (uint32_t)p.N + o : o * (uint32_t)p.N + s.col;
-                    const float rep = __fsub_rn(c[u], __fmul_rn(x, y));        // Eq. 1 on the finished sum
-                    const float cf = __fadd_rn(rep, __fmul_rn(xf, y));         // Eq. 2
+                    const float cf = operand_write_back(p.dtype == MPGEMMFI_FP16, c[u], y, x, xf);     // Eq. 1, Eq. 2
                     stats_account(st, p.detect_mode, f32_bits(cf), f32_bits(c[u]), lin);
                 }
             }
@@ -373,8 +383,7 @@ __device__ __forceinline__ void panel_rows(const uint32_t *As, const uint32_t *C
         if (two_byte) aw = __byte_perm(aw, 0u, a_sel);
         const float a = widen_operand(kDtype, aw);
         const float c = bits_f32(c_bits);
-        const float rep = __fsub_rn(c, __fmul_rn(a, b));          // Eq. 1 on the finished sum
-        const float cf = __fadd_rn(rep, __fmul_rn(a, bf));        // Eq. 2
+        const float cf = operand_write_back(kDtype == MPGEMMFI_FP16, c, a, b, bf);      // Eq. 1, Eq. 2 on the finished sum
         uint32_t fin = f32_bits(cf);
         if (do_bound && !(fabsf(cf) < 131072.0f)) {               // exponent field >= 0x90
             const uint32_t lin = lin_base + r * n_cols;
@@ -402,7 +411,7 @@ __device__ __forceinline__ void panel_rows(const uint32_t *As, const uint32_t *C
         for (int u = 0; u < 4; ++u) {
             const float a = widen_operand(kDtype, two_byte ? __byte_perm(aw[u], 0u, a_sel) : aw[u]);
             const float c = bits_f32(cb[u]);
-            const float cf = __fadd_rn(__fsub_rn(c, __fmul_rn(a, b)), __fmul_rn(a, bf));     // Eq. 1, Eq. 2
+            const float cf = operand_write_back(kDtype == MPGEMMFI_FP16, c, a, b, bf);       // Eq. 1, Eq. 2
             plain = plain && (fabsf(cf) < 131072.0f);
             ch |= f32_bits(cf) ^ cb[u];
             md = fmaxf(md, fabsf(__fsub_rn(cf, c)));        // cf finite and below the bound: never NaN (c is finite too)

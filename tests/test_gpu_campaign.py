@@ -199,3 +199,61 @@ def test_campaign_random_shapes_mixes_and_modes(seed):
     sites = np.concatenate(parts)
     sites["kind"][5] = 11                                   # an invalid entry
     check_campaign_against_oracle(dtype, A, Bt, sites, mode, max_fragile=3)
+
+
+def _widen_np(dtype, bits):
+    """Library conversions only: numpy's half type, or the storage word moved into a float32 word."""
+    bits = np.asarray(bits)
+    if dtype == orc.FP16:
+        return bits.astype(np.uint16).view(np.float16).astype(np.float32)
+    if dtype == orc.BF16:
+        return (bits.astype(np.uint32) << 16).view(np.float32)
+    return (bits.astype(np.uint32) & np.uint32(0xFFFFE000)).view(np.float32)
+
+
+@pytest.mark.parametrize("dtype,shape", [(orc.FP16, (8192, 64, 128)), (orc.BF16, (8192, 64, 128)), (orc.FP16, (700, 520, 72)),
+                                         (orc.TF32, (600, 200, 64))])
+@pytest.mark.parametrize("mode", [orc.T_NONE, orc.T_BOUND | orc.CORRECT])
+def test_operand_trials_are_eq1_eq2_on_the_clean_sum_bit_for_bit(dtype, shape, mode):
+    """An operand trial's statistics are those of Eq. 1-2 applied to the device's own clean C with every product and
+    every sum rounded to FP32, bit for bit: numpy float32 arithmetic (one rounding per operation) restates it.
+    Covers the row-panel kernel (long columns, first two shapes) and the one-CTA-per-trial kernel."""
+    M, N, K = shape
+    rng = np.random.default_rng(91)
+    A = synth.round_to_storage(np.maximum(rng.standard_normal((M, K)), 0).astype(np.float32), dtype)   # zeros among the values
+    Bt = synth.round_to_storage((rng.standard_normal((N, K)) * 0.1).astype(np.float32), dtype)
+    n = 160
+    s = np.zeros(n, dtype=orc.SITE)
+    s["kind"] = rng.integers(0, 2, n)
+    s["row"] = rng.integers(0, M, n); s["col"] = rng.integers(0, N, n); s["k"] = rng.integers(0, K, n)
+    width = 19 if dtype == orc.TF32 else 16
+    s["xor_mask"] = [1 << int(b) for b in rng.integers(0, width, n)]
+    Cg, rec = run_gpu_campaign(dtype, A, Bt, s, mode)
+    HASH_MUL = 0x9E3779B97F4A7C15
+    with np.errstate(all="ignore"):
+        for t in range(n):
+            is_a = int(s["kind"][t]) == orc.KIND_A
+            i, j, k = int(s["row"][t]), int(s["col"][t]), int(s["k"][t])
+            w_clean = int(A[i, k]) if is_a else int(Bt[j, k])
+            x = _widen_np(dtype, np.array([w_clean]))[0]
+            xf = _widen_np(dtype, np.array([orc.flip_operand(dtype, w_clean, int(s["xor_mask"][t]))]))[0]
+            y = _widen_np(dtype, Bt[:, k] if is_a else A[:, k])
+            c = Cg[i, :] if is_a else Cg[:, j]
+            lin = (i * N + np.arange(N)) if is_a else (np.arange(M) * N + j)
+            cf = (c - x * y).astype(np.float32) + (xf * y).astype(np.float32)       # Eq. 1, Eq. 2: four roundings
+            fin = cf.view(np.uint32).copy()
+            det = np.zeros(len(c), dtype=bool)
+            if (mode & 3) == orc.T_BOUND:
+                det = ~(np.abs(cf) < np.float32(131072.0))
+                if mode & orc.CORRECT:
+                    fin[det] &= np.uint32(~(7 << 27) & 0xFFFFFFFF)
+            g = rec[t]
+            assert g["n_affected"] == len(c) and g["n_detected"] == det.sum(), t
+            if np.isnan(cf).any():
+                continue                      # NaN payloads are not part of parity
+            dev = np.abs(fin.view(np.float32) - c)
+            assert g["max_abs_dev"].view(np.uint32) == np.float32(dev.max()).view(np.uint32), (t, g["max_abs_dev"], dev.max())
+            assert bool(g["status"] & 1) == bool((fin != c.view(np.uint32)).any())
+            if det.any():
+                assert g["first_detected"] == lin[det].min()
+                assert int(g["idx_hash"]) == sum((int(l) + 1) * HASH_MUL for l in lin[det]) & ((1 << 64) - 1)
