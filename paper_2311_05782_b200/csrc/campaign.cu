@@ -365,6 +365,14 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
     return v;
 }
 
+// 16-bit word of shared memory, zero-extended
+__device__ __forceinline__ uint32_t lds_u16(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
 template <int kDtype>
 __device__ __forceinline__ void panel_rows(const uint32_t *As, const uint32_t *Cs, const PanelShape &ps, uint32_t rows,
                                            uint32_t lin_base, uint32_t n_cols, uint32_t j, uint32_t k, float b, float bf,
@@ -372,15 +380,14 @@ __device__ __forceinline__ void panel_rows(const uint32_t *As, const uint32_t *C
                                            unsigned long long &hash, float &maxdev, uint32_t &changed)
 {
     constexpr bool two_byte = kDtype != MPGEMMFI_TF32;
-    // the trial's element of the first row: a 16-bit half of a word (byte selector for PRMT) or a word
-    uint32_t a_addr = (uint32_t)__cvta_generic_to_shared(As + (two_byte ? (k >> 1) : k));
+    // the trial's element of the first row: a 16-bit or a 32-bit word
+    uint32_t a_addr = (uint32_t)__cvta_generic_to_shared(As) + (two_byte ? 2u : 4u) * k;
     uint32_t c_addr = (uint32_t)__cvta_generic_to_shared(Cs + j);
-    const uint32_t a_sel = (k & 1u) ? 0x4432u : 0x4410u;          // bytes 2,3 or 0,1 into the low half, zeros above
+    auto lds_a = [](uint32_t addr) { return two_byte ? lds_u16(addr) : lds_u32(addr); };
     const uint32_t a_step = 4u * (uint32_t)ps.a_words, c_step = 4u * (uint32_t)ps.c_words;
 
     // one row, every case handled (flagged values, infinities, NaNs)
     auto exact_row = [&](uint32_t r, uint32_t aw, uint32_t c_bits) {
-        if (two_byte) aw = __byte_perm(aw, 0u, a_sel);
         const float a = widen_operand(kDtype, aw);
         const float c = bits_f32(c_bits);
         const float cf = operand_write_back(kDtype == MPGEMMFI_FP16, c, a, b, bf);      // Eq. 1, Eq. 2 on the finished sum
@@ -403,13 +410,13 @@ __device__ __forceinline__ void panel_rows(const uint32_t *As, const uint32_t *C
         // compare per row, folded into one branch per four rows); otherwise the four rows are done again, exactly.
         uint32_t aw[4], cb[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { aw[u] = lds_u32(a_addr + u * a_step); cb[u] = lds_u32(c_addr + u * c_step); }
+        for (int u = 0; u < 4; ++u) { aw[u] = lds_a(a_addr + u * a_step); cb[u] = lds_u32(c_addr + u * c_step); }
         bool plain = true;
         uint32_t ch = 0;
         float md = 0.0f;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const float a = widen_operand(kDtype, two_byte ? __byte_perm(aw[u], 0u, a_sel) : aw[u]);
+            const float a = widen_operand(kDtype, aw[u]);
             const float c = bits_f32(cb[u]);
             const float cf = operand_write_back(kDtype == MPGEMMFI_FP16, c, a, b, bf);       // Eq. 1, Eq. 2
             plain = plain && (fabsf(cf) < 131072.0f);
@@ -424,7 +431,7 @@ __device__ __forceinline__ void panel_rows(const uint32_t *As, const uint32_t *C
             for (int u = 0; u < 4; ++u) exact_row(r + u, aw[u], cb[u]);
         }
     }
-    for (; r < rows; ++r, a_addr += a_step, c_addr += c_step) exact_row(r, lds_u32(a_addr), lds_u32(c_addr));
+    for (; r < rows; ++r, a_addr += a_step, c_addr += c_step) exact_row(r, lds_a(a_addr), lds_u32(c_addr));
 }
 
 __global__ void __launch_bounds__(PANEL_THREADS) panel_kernel(CampaignParams p, PanelShape ps)
