@@ -404,18 +404,19 @@ __device__ __forceinline__ void panel_rows(const uint32_t *As, const uint32_t *C
         maxdev = d != d ? __uint_as_float(0x7F800000u) : fmaxf(maxdev, d);      // a NaN deviation counts as +inf
     };
 
+    constexpr int STEP = 8;
     uint32_t r = 0;
-    for (; r + 4 <= rows; r += 4, a_addr += 4 * a_step, c_addr += 4 * c_step) {
-        // Four rows at once on the assumption that nothing is flagged and nothing is infinite or NaN (one
-        // compare per row, folded into one branch per four rows); otherwise the four rows are done again, exactly.
-        uint32_t aw[4], cb[4];
+    for (; r + STEP <= rows; r += STEP, a_addr += STEP * a_step, c_addr += STEP * c_step) {
+        // STEP rows at once on the assumption that nothing is flagged and nothing is infinite or NaN (one
+        // compare per row, folded into one branch per step); otherwise the rows are done again, exactly.
+        uint32_t aw[STEP], cb[STEP];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { aw[u] = lds_a(a_addr + u * a_step); cb[u] = lds_u32(c_addr + u * c_step); }
+        for (int u = 0; u < STEP; ++u) { aw[u] = lds_a(a_addr + u * a_step); cb[u] = lds_u32(c_addr + u * c_step); }
         bool plain = true;
         uint32_t ch = 0;
         float md = 0.0f;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < STEP; ++u) {
             const float a = widen_operand(kDtype, aw[u]);
             const float c = bits_f32(cb[u]);
             const float cf = operand_write_back(kDtype == MPGEMMFI_FP16, c, a, b, bf);       // Eq. 1, Eq. 2
@@ -428,7 +429,7 @@ __device__ __forceinline__ void panel_rows(const uint32_t *As, const uint32_t *C
             maxdev = fmaxf(maxdev, md);
         } else {
 #pragma unroll
-            for (int u = 0; u < 4; ++u) exact_row(r + u, aw[u], cb[u]);
+            for (int u = 0; u < STEP; ++u) exact_row(r + u, aw[u], cb[u]);
         }
     }
     for (; r < rows; ++r, a_addr += a_step, c_addr += c_step) exact_row(r, lds_a(a_addr), lds_u32(c_addr));
