@@ -211,18 +211,20 @@ def _widen_np(dtype, bits):
     return (bits.astype(np.uint32) & np.uint32(0xFFFFE000)).view(np.float32)
 
 
-@pytest.mark.parametrize("dtype,shape", [(orc.FP16, (8192, 64, 128)), (orc.BF16, (8192, 64, 128)), (orc.FP16, (700, 520, 72)),
-                                         (orc.TF32, (600, 200, 64))])
+@pytest.mark.parametrize("dtype,shape,n", [(orc.FP16, (8192, 64, 128), 160), (orc.BF16, (8192, 64, 128), 160),
+                                           (orc.FP16, (700, 520, 72), 160), (orc.TF32, (600, 200, 64), 160),
+                                           (orc.FP16, (4608, 64, 576), 5000), (orc.TF32, (2048, 40, 64), 2500)])
 @pytest.mark.parametrize("mode", [orc.T_NONE, orc.T_BOUND | orc.CORRECT])
-def test_operand_trials_are_eq1_eq2_on_the_clean_sum_bit_for_bit(dtype, shape, mode):
+def test_operand_trials_are_eq1_eq2_on_the_clean_sum_bit_for_bit(dtype, shape, n, mode):
     """An operand trial's statistics are those of Eq. 1-2 applied to the device's own clean C with every product and
     every sum rounded to FP32, bit for bit: numpy float32 arithmetic (one rounding per operation) restates it.
-    Covers the row-panel kernel (long columns, first two shapes) and the one-CTA-per-trial kernel."""
+    Covers the row-panel kernel (long columns: the first two and the last two shapes, the last two with several groups of
+    1024 column trials, so that full and partial groups and their bank-wise dealing to warps all occur) and the
+    one-CTA-per-trial kernel."""
     M, N, K = shape
     rng = np.random.default_rng(91)
     A = synth.round_to_storage(np.maximum(rng.standard_normal((M, K)), 0).astype(np.float32), dtype)   # zeros among the values
     Bt = synth.round_to_storage((rng.standard_normal((N, K)) * 0.1).astype(np.float32), dtype)
-    n = 160
     s = np.zeros(n, dtype=orc.SITE)
     s["kind"] = rng.integers(0, 2, n)
     s["row"] = rng.integers(0, M, n); s["col"] = rng.integers(0, N, n); s["k"] = rng.integers(0, K, n)
