@@ -292,11 +292,29 @@ def main():
     total_flops = reduce_sum(flops * args.steps, world, dev)
     value = total_flops / (ms_inj_max * 1e-3) / 1e12
 
-    # ---- same kernel, injection and detection disabled
+    # ---- same kernel, injection and detection disabled: launches with and without injection alternate in one
+    # loop (each with its own event pair and L2 flush), so that both see the same clocks and temperatures
     off_steps = max(10, args.steps // 4)
-    ms_off, _ = timed(lambda i: gemm_step(i, False), off_steps, 3)
-    tflops_off = flops * off_steps / (ms_off * 1e-3) / 1e12
-    tflops_on_local = flops * args.steps / (ms_inj * 1e-3) / 1e12
+    ms_pair = [0.0, 0.0]
+    for i in range(3):
+        for inject in (True, False):
+            flush.zero_()
+            gemm_step(i, inject)
+    torch.cuda.synchronize(dev)
+    pair_events = []
+    for i in range(off_steps):
+        for inject in (True, False):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            gemm_step(i, inject)
+            e1.record(stream)
+            pair_events.append((0 if inject else 1, e0, e1))
+    torch.cuda.synchronize(dev)
+    for which, e0, e1 in pair_events:
+        ms_pair[which] += e0.elapsed_time(e1)
+    tflops_off = flops * off_steps / (ms_pair[1] * 1e-3) / 1e12
+    on_over_off_time = ms_pair[0] / ms_pair[1]
 
     # ---- campaign: one clean GEMM + this rank's trials per launch
     rec = torch.empty((n_my, 12), dtype=torch.int32, device=dev)
@@ -380,7 +398,8 @@ def main():
             "gpu_launches": args.steps,
             "roofline": roofline,
             "injection_off": {"tflops": tflops_off, "steps": off_steps,
-                              "injected_over_plain_time": tflops_off / tflops_on_local},
+                              "injected_over_plain_time": on_over_off_time,
+                              "how": "launches with and without injection alternate in one loop"},
             "campaign": {"trials_per_s": trials_per_s, "trials_per_launch": n_my, "launches": camp_steps,
                          "ms_per_launch": ms_camp_max / camp_steps},
             "cpu_baseline": baseline,
