@@ -377,6 +377,33 @@ def main():
                     "frac_of_sustained": achieved / (peaks["bf16_tflops_sustained"] * (0.5 if dtype == synth.DTYPE_TF32 else 1.0)),
                     "frac_of_nominal": achieved / (1125.0 if dtype == synth.DTYPE_TF32 else 2250.0),
                     "kernel": "gemm_kernel", "flops_per_launch": flops, "min_bytes_per_launch": min_bytes}
+        if dtype == synth.DTYPE_TF32 and rank == 0:
+            # there is no measured TF32 peak: time the library's TF32 GEMM on the same shape, in this run (context for
+            # the halved BF16 figure above; FP32 inputs, FP32 output, L2 flushed before every launch like the steps)
+            import torch.backends.cuda
+            old = torch.backends.cuda.matmul.allow_tf32
+            torch.backends.cuda.matmul.allow_tf32 = True
+            try:
+                xa = A.view(torch.float32)
+                xb = Bt.view(torch.float32).t()
+                for _ in range(3):
+                    flush.zero_()
+                    torch.matmul(xa, xb, out=C)
+                torch.cuda.synchronize(dev)
+                evs = []
+                for _ in range(10):
+                    flush.zero_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    torch.matmul(xa, xb, out=C)
+                    e1.record(stream)
+                    evs.append((e0, e1))
+                torch.cuda.synchronize(dev)
+                lib_ms = statistics.median(e0.elapsed_time(e1) for e0, e1 in evs)
+                roofline["library_tf32_tflops"] = flops / (lib_ms * 1e-3) / 1e12
+                roofline["frac_of_library_tf32"] = achieved / roofline["library_tf32_tflops"]
+            finally:
+                torch.backends.cuda.matmul.allow_tf32 = old
 
     if rank == 0:
         baseline = None
