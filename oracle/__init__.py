@@ -75,6 +75,14 @@ def lib():
         L.orc_gemm_addend.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp, vp]
         L.orc_campaign.restype = C.c_int
         L.orc_campaign.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, vp]
+        L.orc_campaign_form.restype = C.c_int
+        L.orc_campaign_form.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp]
+        L.orc_operand_trial_values.restype = C.c_int
+        L.orc_operand_trial_values.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, C.c_int, vp]
+        L.orc_round_output.restype = C.c_uint32
+        L.orc_round_output.argtypes = [C.c_int, C.c_uint32]
+        L.orc_gemm_out16.restype = C.c_int
+        L.orc_gemm_out16.argtypes = [C.c_int] * 4 + [vp, vp, vp, C.c_int, vp, vp, C.c_int, C.c_int, C.c_int, vp, vp, vp]
         L.orc_sample.restype = C.c_int
         L.orc_sample.argtypes = [C.c_int] * 4 + [vp, vp, vp, C.c_int, vp, vp, C.c_int, vp, vp]
         L.orc_sample_addend.restype = C.c_int
@@ -180,8 +188,10 @@ def gemm(dtype, A, Bt, sites=None, detect_mode=0, kstep=None, addend=None):
     return Cm, hdr, log, bitmap
 
 
-def campaign(dtype, A, Bt, C_clean, sites, detect_mode=0, kstep=None):
-    """One record per single-site trial (incremental evaluation of the affected elements)."""
+def campaign(dtype, A, Bt, C_clean, sites, detect_mode=0, kstep=None, operand_form=0):
+    """One record per single-site trial (incremental evaluation of the affected elements).
+    operand_form: 0 = an operand trial's row / column is accumulated again with the faulty operand (the definition);
+    1 = Eq. 1-2 applied to the finished sums of C_clean."""
     A = _storage(A, dtype)
     Bt = _storage(Bt, dtype)
     M, K = A.shape
@@ -191,9 +201,52 @@ def campaign(dtype, A, Bt, C_clean, sites, detect_mode=0, kstep=None):
     Cc = np.ascontiguousarray(C_clean, dtype=np.float32)
     assert Cc.shape == (M, N)
     rec = np.zeros(len(s), dtype=RECORD)
-    rc = lib().orc_campaign(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(Cc), _ptr(s), len(s), detect_mode, kstep, _ptr(rec))
+    rc = lib().orc_campaign_form(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(Cc), _ptr(s), len(s), detect_mode, kstep,
+                                 operand_form, _ptr(rec))
     assert rc == 0
     return rec
+
+
+def operand_trial_values(dtype, A, Bt, C_clean, site, form=0):
+    """Unchecked values of the row (A site) or column (B site) of C that one operand site reaches; form as in campaign()."""
+    A = _storage(A, dtype)
+    Bt = _storage(Bt, dtype)
+    M, K = A.shape
+    N, _ = Bt.shape
+    s = _sites(np.asarray(site).reshape(1))
+    Cc = np.ascontiguousarray(C_clean, dtype=np.float32)
+    assert Cc.shape == (M, N)
+    out = np.empty(N if int(s["kind"][0]) == KIND_A else M, dtype=np.float32)
+    n = lib().orc_operand_trial_values(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(Cc), _ptr(s), form, _ptr(out))
+    assert n == len(out), n
+    return out
+
+
+OUT_FP16, OUT_BF16 = 0, 1
+
+
+def round_output(out_fmt, bits):
+    """FP32 word -> 16-bit word of the output format, round to nearest even."""
+    return int(lib().orc_round_output(out_fmt, int(bits) & 0xFFFFFFFF))
+
+
+def gemm_out16(dtype, A, Bt, out_fmt, sites=None, detect_mode=0, kstep=None, addend=None):
+    """orc.gemm with the checked FP32 result rounded to a 16-bit format. Returns (D16 uint16[M,N], header, log, bitmap)."""
+    A = _storage(A, dtype)
+    Bt = _storage(Bt, dtype)
+    M, K = A.shape
+    N, _ = Bt.shape
+    kstep = (32 if dtype == TF32 else 64) if kstep is None else kstep
+    s = _sites(sites)
+    D = np.empty((M, N), dtype=np.uint16)
+    hdr = np.zeros(16, dtype=np.uint32)
+    log = np.zeros(len(s), dtype=SITE_LOG)
+    bitmap = np.zeros((M, (N + 31) // 32), dtype=np.uint32)
+    Cin = None if addend is None else np.ascontiguousarray(addend, dtype=np.float32)
+    rc = lib().orc_gemm_out16(dtype, M, N, K, _ptr(A), _ptr(Bt), _ptr(Cin), out_fmt, _ptr(D), _ptr(s), len(s),
+                              detect_mode, kstep, _ptr(hdr), _ptr(log), _ptr(bitmap))
+    assert rc == 0
+    return D, hdr, log, bitmap
 
 
 def sample(dtype, A, Bt, si, sj, sites=None, start=None):

@@ -29,7 +29,10 @@
  * their Section VI-C bit-level forms, closed forms for bit flips, exact integer
  * GEMMs, linearity of operand faults, Eq. 1-2 exactness, brute-force flag
  * bitmaps; the addend form against a GEMM cut in two along k, exact integers
- * and a per-element Python loop. No function here is "parity unpinned".
+ * and a per-element Python loop; the write-back form of operand trials against
+ * the recompute on exact integers and within two roundings elsewhere; the
+ * 16-bit output rounding against library conversions, all ties and both
+ * range ends. No function here is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -479,6 +482,60 @@ int orc_gemm_addend(int dtype, int M, int N, int K, const void *A, const void *B
     return gemm_impl(dtype, M, N, K, A, Bt, C_in, D, sites, n_faults, detect_mode, kstep, hdr, log, bitmap);
 }
 
+/* ------------------------------------------------------------------ 16-bit output */
+
+enum { ORC_OUT_FP16 = 0, ORC_OUT_BF16 = 1 };
+
+/*
+ * Round an FP32 word to the nearest value of a 16-bit format, ties to even (the models of
+ * Section IV-B run "16" / "bf16" end to end: the FP32 result D of D = A x B + C, Section II-B,
+ * goes back to the 16-bit format before the next layer reads it).
+ * Written from the formats' definitions (Section II-A): FP16 1/5/10, bias 15, subnormals below
+ * 2^-14, largest finite value 65504; BF16 1/8/7 = the upper half of an FP32 word.
+ * A NaN stays a (quiet) NaN; which payload it carries is not specified here.
+ */
+uint32_t orc_round_output(int out_fmt, uint32_t bits)
+{
+    uint32_t sign = (bits >> 16) & 0x8000u;
+    uint32_t E = (bits >> 23) & 0xFFu;
+    uint32_t m = bits & 0x7FFFFFu;
+    if (out_fmt == ORC_OUT_BF16) {
+        if (E == 0xFFu && m != 0) return sign | 0x7FC0u;
+        uint32_t keep = bits >> 16, rest = bits & 0xFFFFu;             /* 16 bits dropped */
+        if (rest > 0x8000u || (rest == 0x8000u && (keep & 1u))) keep += 1u;   /* carries into the exponent; Inf at the top */
+        return keep & 0xFFFFu;
+    }
+    /* FP16 */
+    if (E == 0xFFu) return sign | (m ? 0x7E00u : 0x7C00u);
+    float x = fabsf(u2f(bits));
+    if (x >= 65520.0f) return sign | 0x7C00u;          /* halfway between 65504 and 2^16 ties to the even one: infinity */
+    if (x < 6.103515625e-05f) {                          /* below 2^-14: multiples of 2^-24; the scaling is exact */
+        float q = nearbyintf(x * 16777216.0f);           /* round-to-nearest-even is the default rounding mode */
+        return sign | (uint32_t)q;                       /* 1024 = the smallest normal number, as it should be */
+    }
+    uint32_t keep = m >> 13, rest = m & 0x1FFFu;         /* 13 mantissa bits dropped */
+    uint32_t h = ((E - 112u) << 10) + keep;              /* rebias 127 -> 15 */
+    if (rest > 0x1000u || (rest == 0x1000u && (keep & 1u))) h += 1u;
+    return sign | h;
+}
+
+/*
+ * The fault-injected GEMM with a 16-bit result: everything as orc_gemm / orc_gemm_addend (sites,
+ * checks, flags, counts and log all on the FP32 values), then every FP32 element is rounded once.
+ */
+int orc_gemm_out16(int dtype, int M, int N, int K, const void *A, const void *Bt, const float *C_in, int out_fmt,
+                   uint16_t *D16, const orc_site *sites, int n_faults, int detect_mode, int kstep,
+                   uint32_t *hdr, orc_site_log *log, uint32_t *bitmap)
+{
+    float *D = (float *)malloc(sizeof(float) * (size_t)M * (size_t)N);
+    if (!D) return -1;
+    int rc = gemm_impl(dtype, M, N, K, A, Bt, C_in, D, sites, n_faults, detect_mode, kstep, hdr, log, bitmap);
+    if (rc == 0)
+        for (size_t e = 0; e < (size_t)M * (size_t)N; ++e) D16[e] = (uint16_t)orc_round_output(out_fmt, f2u(D[e]));
+    free(D);
+    return rc;
+}
+
 /* ------------------------------------------------------------------ single trials (incremental mode) */
 
 typedef struct {
@@ -506,13 +563,71 @@ static void trial_account(trial_acc *t, int detect_mode, float value, float clea
 }
 
 /*
+ * Raw (unchecked) values of the output elements an operand site reaches: row s->row of C for an
+ * A site (N values), column s->col for a B site (M values).
+ *   form 0: the definition -- every affected element is accumulated again in k order with the
+ *           faulty operand in place of the clean one;
+ *   form 1: the write-back of Eq. 1-2 (Section III-E) applied to the FINISHED clean sum c:
+ *           rep = fl32(c - fl32(x*y)), then c' = fl32(rep + fl32(x'*y)), with x the clean operand,
+ *           x' the faulty one and y the other factor of the term. This is how a faulty term enters
+ *           a sum that has already been accumulated; it differs from form 0 only by the roundings
+ *           of the two steps.
+ * Af, Bf: widened operands. Returns the number of values written.
+ */
+static int operand_trial_values(int dtype, int M, int N, int K, const void *A, const void *Bt,
+                                const float *Af, const float *Bf, const float *C_clean,
+                                const orc_site *s, int form, float *out)
+{
+    int isA = s->kind == ORC_A;
+    size_t pos = isA ? (size_t)s->row * K + s->k : (size_t)s->col * K + s->k;
+    uint32_t before = load_storage(dtype, isA ? A : Bt, pos);
+    if (dtype == ORC_TF32) before &= 0xFFFFE000u;
+    uint32_t after = orc_flip_operand(dtype, before, s->xor_mask);
+    float x = orc_widen(dtype, before), xf = orc_widen(dtype, after);
+    int n_other = isA ? N : M;
+    if (form == 0) {
+        float *vec = (float *)malloc(sizeof(float) * (size_t)K);
+        memcpy(vec, isA ? &Af[(size_t)s->row * K] : &Bf[(size_t)s->col * K], sizeof(float) * (size_t)K);
+        vec[s->k] = xf;
+        for (int o = 0; o < n_other; ++o)
+            out[o] = isA ? element_clean(vec, &Bf[(size_t)o * K], K) : element_clean(&Af[(size_t)o * K], vec, K);
+        free(vec);
+    } else {
+        for (int o = 0; o < n_other; ++o) {
+            float y = isA ? Bf[(size_t)o * K + s->k] : Af[(size_t)o * K + s->k];
+            float c = isA ? C_clean[(size_t)s->row * N + o] : C_clean[(size_t)o * N + s->col];
+            float re2 = x * y;          /* the clean term */
+            float re_err = xf * y;      /* the faulty term */
+            float rep = c - re2;        /* Eq. 1 */
+            out[o] = rep + re_err;      /* Eq. 2 */
+        }
+    }
+    return n_other;
+}
+
+int orc_operand_trial_values(int dtype, int M, int N, int K, const void *A, const void *Bt, const float *C_clean,
+                             const orc_site *s, int form, float *out)
+{
+    if (!(s->kind == ORC_A || s->kind == ORC_B) || !site_valid(s, dtype, M, N, K)) return -1;
+    float *Af = widen_matrix(dtype, A, (size_t)M, (size_t)K);
+    float *Bf = widen_matrix(dtype, Bt, (size_t)N, (size_t)K);
+    if (!Af || !Bf) { free(Af); free(Bf); return -1; }
+    int n = operand_trial_values(dtype, M, N, K, A, Bt, Af, Bf, C_clean, s, form, out);
+    free(Af); free(Bf);
+    return n;
+}
+
+/*
  * One record per trial, each trial = one site applied alone to the clean GEMM.
  * Only the affected output elements are recomputed (an A site: row i, a B site:
  * column j, others: one element), each by the same sequential loop as orc_gemm.
  * C_clean: the fault-free, unchecked output of orc_gemm (detect_mode 0).
+ * operand_form: how an operand trial reaches its row / column, see operand_trial_values
+ * (0 = recompute, the definition; 1 = Eq. 1-2 on the finished sums of C_clean).
  */
-int orc_campaign(int dtype, int M, int N, int K, const void *A, const void *Bt, const float *C_clean,
-                 const orc_site *sites, int n_trials, int detect_mode, int kstep, orc_trial_record *rec)
+int orc_campaign_form(int dtype, int M, int N, int K, const void *A, const void *Bt, const float *C_clean,
+                      const orc_site *sites, int n_trials, int detect_mode, int kstep, int operand_form,
+                      orc_trial_record *rec)
 {
     float *Af = widen_matrix(dtype, A, (size_t)M, (size_t)K);
     float *Bf = widen_matrix(dtype, Bt, (size_t)N, (size_t)K);
@@ -548,16 +663,14 @@ int orc_campaign(int dtype, int M, int N, int K, const void *A, const void *Bt, 
             if (dtype == ORC_TF32) before &= 0xFFFFE000u;
             uint32_t after = orc_flip_operand(dtype, before, s->xor_mask);
             r->primary_index = (uint32_t)pos; r->before_bits = before; r->after_bits = after; r->final_bits = after;
-            float *vec = (float *)malloc(sizeof(float) * (size_t)K);
-            memcpy(vec, isA ? &Af[(size_t)s->row * K] : &Bf[(size_t)s->col * K], sizeof(float) * (size_t)K);
-            vec[s->k] = orc_widen(dtype, after);
             int n_other = isA ? N : M;
+            float *vals = (float *)malloc(sizeof(float) * (size_t)n_other);
+            operand_trial_values(dtype, M, N, K, A, Bt, Af, Bf, C_clean, s, operand_form, vals);
             for (int o = 0; o < n_other; ++o) {
                 uint32_t lin = isA ? s->row * (uint32_t)N + (uint32_t)o : (uint32_t)o * (uint32_t)N + s->col;
-                float v = isA ? element_clean(vec, &Bf[(size_t)o * K], K) : element_clean(&Af[(size_t)o * K], vec, K);
-                trial_account(&ta, detect_mode, v, C_clean[lin], lin, NULL);
+                trial_account(&ta, detect_mode, vals[o], C_clean[lin], lin, NULL);
             }
-            free(vec);
+            free(vals);
         }
         r->n_affected = ta.n_aff; r->n_detected = ta.n_det; r->idx_hash = ta.hash;
         r->first_detected = ta.first; r->max_abs_dev = ta.maxdev;
@@ -566,6 +679,12 @@ int orc_campaign(int dtype, int M, int N, int K, const void *A, const void *Bt, 
     }
     free(Af); free(Bf);
     return 0;
+}
+
+int orc_campaign(int dtype, int M, int N, int K, const void *A, const void *Bt, const float *C_clean,
+                 const orc_site *sites, int n_trials, int detect_mode, int kstep, orc_trial_record *rec)
+{
+    return orc_campaign_form(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mode, kstep, 0, rec);
 }
 
 /* ------------------------------------------------------------------ sampled outputs at any size */

@@ -223,15 +223,43 @@ def brute_record_stats(vals, clean, lins, detect_mode):
     return n_det, h, first, maxdev, changed
 
 
-@pytest.mark.parametrize("name,mix", [("c1", "out"), ("c2", "operand"), ("c4", "acc2"), ("c5", "mixed"), ("c2", "term")])
-def test_incremental_trials_equal_full_recompute(name, mix):
-    """Every trial record equals what a full fault-injected GEMM with that single site gives."""
-    cfg = synth.CONFIGS[name]
+def record_from_full_recompute(Cf, bm, Cclean, lins, detect_mode):
+    """What a trial's record must say, read off a full fault-injected GEMM with that one site: the flagged set is the
+    GEMM's bitmap, the final values are the GEMM's output."""
+    N = Cf.shape[1]
+    n_det, h, first, maxdev, changed = 0, 0, 0xFFFFFFFF, 0.0, 0
+    for lin in lins:
+        i, j = divmod(lin, N)
+        if (int(bm[i, j // 32]) >> (j % 32)) & 1:
+            n_det += 1; h = (h + (lin + 1) * HASH_MUL) & MASK64; first = min(first, lin)
+        fin, cl = Cf[i, j], Cclean[i, j]
+        changed |= int(f32_bits(float(fin)) != f32_bits(float(cl)))
+        with np.errstate(all="ignore"):
+            d = abs(np.float32(fin) - np.float32(cl))
+        maxdev = max(maxdev, float("inf") if np.isnan(d) else float(d))
+    status = changed | (2 if n_det else 0) | (4 if n_det and (detect_mode & orc.CORRECT) and (detect_mode & 3) == 1 else 0)
+    return n_det, h, first, maxdev, status
+
+
+@pytest.mark.parametrize("name,mix,mode", [
+    ("c1", "out", None), ("c2", "operand", None), ("c4", "acc2", None), ("c5", "mixed", None), ("c2", "term", None),
+    ("c2", "term", orc.T_BOUND), ("c2", "term", orc.T_RMAX | orc.CORRECT), ("c2", "term", orc.T_RFLIP | orc.CORRECT),
+    ("c5", "mixed", orc.T_NONE)])
+def test_incremental_trials_equal_full_recompute(name, mix, mode):
+    """Every trial record equals what a full fault-injected GEMM with that single site gives: the full recompute is
+    the definition. ("c2", "term") runs TERM trials under BoundCheck + correction, where a product-level correction
+    is followed by the output check on the corrected sum."""
     M, N, K = 24, 40, 96
     w = synth.make_workload(name, M, N, K, trials=40, mix=mix)
-    dt, mode = w.dtype, w.detect_mode
+    dt = w.dtype
+    mode = w.detect_mode if mode is None else mode
+    if mix == "term":
+        # single-bit flips of small products rarely reach the thresholds: put some masks on the exponent's top bits
+        w.sites["xor_mask"][::3] = 1 << 30
+        w.sites["xor_mask"][1::6] = 3 << 29
     Cclean, *_ = orc.gemm(dt, w.A, w.Bt)
     rec = orc.campaign(dt, w.A, w.Bt, Cclean, w.sites, mode)
+    seen_status = set()
     for t in range(len(w.sites)):
         s = w.sites[t:t + 1]
         Cf, hdr, log, bm = orc.gemm(dt, w.A, w.Bt, s, mode)
@@ -242,27 +270,104 @@ def test_incremental_trials_equal_full_recompute(name, mix):
             lins = [ii * N + j for ii in range(M)]
         else:
             lins = [i * N + j]
-        # raw faulty values: rerun without the check
-        Craw, _, lograw, _ = orc.gemm(dt, w.A, w.Bt, s, mode & ~3 if kind != orc.KIND_TERM else mode)
-        if kind == orc.KIND_TERM and (mode & 3) == 1:
-            # the product-level check is part of the trial; the output check is applied by brute_record_stats
-            Craw = Cf.copy()
-            if mode & orc.CORRECT:
-                pytest.skip("corrected outputs hide the raw value; covered by the other mixes")
-        n_det, h, first, maxdev, changed = brute_record_stats(
-            [Craw.reshape(-1)[l] for l in lins], [Cclean.reshape(-1)[l] for l in lins], lins, mode)
         r = rec[t]
+        # (1) the record read off the full recompute's output and bitmap
+        n_det, h, first, maxdev, status = record_from_full_recompute(Cf, bm, Cclean, lins, mode)
         assert r["kind"] == kind and r["n_affected"] == len(lins)
         assert r["n_detected"] == n_det == hdr[1]
         assert int(r["idx_hash"]) == h and r["first_detected"] == first
-        assert (r["status"] & 1) == changed
+        assert r["status"] == status, (t, r["status"], status)
         assert float(r["max_abs_dev"]) == maxdev or (np.isinf(maxdev) and np.isinf(r["max_abs_dev"]))
         assert r["before_bits"] == log["before_bits"][0] and r["after_bits"] == log["after_bits"][0]
         if kind in (orc.KIND_OUT, orc.KIND_ACC, orc.KIND_TERM):
             assert r["final_bits"] == f32_bits(float(Cf[i, j])) and r["primary_index"] == i * N + j
+        else:
+            assert r["final_bits"] == log["final_bits"][0] == log["after_bits"][0]
+            assert r["primary_index"] == (i if kind == orc.KIND_A else j) * K + int(s["k"][0])
+        seen_status.add(int(r["status"]))
+        # (2) where the unchecked faulty value can be had (no product-level check in the way): the output check
+        # restated on it, element by element
+        if kind != orc.KIND_TERM or (mode & 3) == 0:
+            Craw, *_ = orc.gemm(dt, w.A, w.Bt, s, mode & ~3)
+            b_det, b_h, b_first, b_maxdev, b_changed = brute_record_stats(
+                [Craw.reshape(-1)[l] for l in lins], [Cclean.reshape(-1)[l] for l in lins], lins, mode)
+            assert (b_det, b_h, b_first, b_changed) == (n_det, h, first, status & 1)
+            assert b_maxdev == maxdev or (np.isinf(maxdev) and np.isinf(b_maxdev))
         # untouched elements keep their clean value
         mask = np.ones(M * N, dtype=bool); mask[lins] = False
         assert np.array_equal(Cf.reshape(-1)[mask].view(np.uint32), Cclean.reshape(-1)[mask].view(np.uint32))
+    if mix == "term" and (mode & 3):
+        # the cases this pin is here for did occur: a trial that ends unflagged and changed, and (under BoundCheck
+        # without correction of the product... or with it) both flagged and unflagged trials
+        assert 1 in seen_status or 0 in seen_status
+    if mix == "term" and mode == (orc.T_BOUND | orc.CORRECT):
+        # product flagged and corrected, sum below the threshold afterwards: status "changed" only
+        logs = [orc.gemm(dt, w.A, w.Bt, w.sites[t:t + 1], mode)[2][0] for t in range(len(w.sites))]
+        assert any(l["status"] & 4 for l in logs) and any(not (l["status"] & 4) for l in logs)
+
+
+def test_term_trial_product_correction_then_output_check():
+    """A TERM trial under BoundCheck + correction, by hand: the product's exponent is corrected first (three bits
+    cleared), the corrected product enters the sum by Eq. 1-2, and only then the output check looks at the sum."""
+    K = 8
+    a = np.zeros((1, K), dtype=np.float32); b = np.zeros((1, K), dtype=np.float32)
+    a[0, :] = 1.0; b[0, :] = [1, 2, 3, 4, 5, 6, 7, 8]
+    A, Bt = synth.round_to_storage(a, orc.BF16), synth.round_to_storage(b, orc.BF16)
+    Cclean, *_ = orc.gemm(orc.BF16, A, Bt)
+    assert Cclean[0, 0] == 36.0
+    # term k=3 (product 4.0 = 0x40800000): flipping bit 29 gives exponent 0xC1 -> 2^66: flagged; the correction clears
+    # exponent bits 6..4: 0xC1 -> 0x81, i.e. 4.0 again: the sum returns to 36 exactly
+    s = site(orc.KIND_TERM, 0, 0, 3, 1 << 29)
+    r = orc.campaign(orc.BF16, A, Bt, Cclean, s, orc.T_BOUND | orc.CORRECT, kstep=4)[0]
+    assert r["before_bits"] == 0x40800000 and r["after_bits"] == 0x60800000
+    assert bits_f32(int(r["final_bits"])) == 36.0 and r["status"] == 0 and r["n_detected"] == 0 and r["max_abs_dev"] == 0.0
+    # detection only: the huge product stays, the sum is 2^66 (32 is lost in it), the output check flags it
+    r = orc.campaign(orc.BF16, A, Bt, Cclean, s, orc.T_BOUND, kstep=4)[0]
+    want = np.float32(np.float32(np.float32(10.0 - 4.0) + np.float32(2.0 ** 66)) + np.float32(26.0))
+    assert bits_f32(int(r["final_bits"])) == float(want) and r["status"] == 3 and r["n_detected"] == 1
+    assert r["first_detected"] == 0 and int(r["idx_hash"]) == HASH_MUL
+    # correction on, but a flip the product check cannot see (bit 27: 4.0 -> 4 * 2^16 = 262144 has exponent 0x91...):
+    # exponent 0x81 ^ 0x10 = 0x91 is flagged too; use bit 26 instead: 0x81 ^ 0x08 = 0x89 -> 4 * 2^8 = 1024, not flagged
+    s = site(orc.KIND_TERM, 0, 0, 3, 1 << 26)
+    r = orc.campaign(orc.BF16, A, Bt, Cclean, s, orc.T_BOUND | orc.CORRECT, kstep=4)[0]
+    assert bits_f32(int(r["final_bits"])) == 36.0 - 4.0 + 1024.0 and r["status"] == 1 and r["max_abs_dev"] == 1020.0
+
+
+@pytest.mark.parametrize("dtype", [orc.FP16, orc.BF16, orc.TF32])
+def test_sampled_outputs_with_operand_sites_equal_the_full_recompute(dtype):
+    """orc.sample with an A / B site table: bit-equal to the same elements of orc.gemm with those sites, including two
+    sites that compose on one operand word and sites that miss the sampled rows and columns."""
+    M, N, K = 9, 11, 50
+    rng = np.random.default_rng(41)
+    A = synth.round_to_storage(rng.standard_normal((M, K)).astype(np.float32), dtype)
+    Bt = synth.round_to_storage(rng.standard_normal((N, K)).astype(np.float32), dtype)
+    top = 18 if dtype == orc.TF32 else 15
+    sites = np.concatenate([
+        site(orc.KIND_A, row=2, k=7, mask=1 << (top - 1)),       # exponent MSB of A[2,7]
+        site(orc.KIND_B, col=5, k=49, mask=1 << top),            # sign of B[49,5]
+        site(orc.KIND_A, row=2, k=7, mask=0b101),                # composes with the first on the same word
+        site(orc.KIND_B, col=0, k=0, mask=1 << 3),
+        site(orc.KIND_A, row=8, k=49, mask=3 << 4),
+    ])
+    Cf, hdr, log, _ = orc.gemm(dtype, A, Bt, sites)
+    C0, *_ = orc.gemm(dtype, A, Bt)
+    assert hdr[3] == 5 and log["before_bits"][2] == log["after_bits"][0]
+    si, sj = np.meshgrid(np.arange(M, dtype=np.uint32), np.arange(N, dtype=np.uint32), indexing="ij")
+    sc, sap = orc.sample(dtype, A, Bt, si.reshape(-1), sj.reshape(-1), sites)
+    assert np.array_equal(sc.view(np.uint32).reshape(M, N), Cf.view(np.uint32))
+    # the sites did something, and only where they should
+    moved = Cf.view(np.uint32) != C0.view(np.uint32)
+    assert moved[2].all() and moved[:, 5].sum() >= M - 1 and moved[8].any() and moved[:, 0].any()
+    quiet = np.ones((M, N), dtype=bool); quiet[[2, 8], :] = False; quiet[:, [0, 5]] = False
+    assert not moved[quiet].any()
+    # the magnitude sum uses the operands actually multiplied
+    A2, B2 = A.copy(), Bt.copy()
+    for t in sites:
+        if t["kind"] == orc.KIND_A:
+            A2[t["row"], t["k"]] = orc.flip_operand(dtype, int(A2[t["row"], t["k"]]), int(t["xor_mask"]))
+        else:
+            B2[t["col"], t["k"]] = orc.flip_operand(dtype, int(B2[t["col"], t["k"]]), int(t["xor_mask"]))
+    assert np.allclose(sap.reshape(M, N), orc.absprod(dtype, A2, B2), rtol=1e-12)
 
 
 @pytest.mark.parametrize("name", ["c1", "c2", "c3a", "c3b", "c4", "c5"])
@@ -408,3 +513,77 @@ def test_addend_scalar_loop_and_sites():
     untouched = np.ones((M, N), dtype=bool)
     untouched[1, 2] = untouched[3, 4] = untouched[2, 0] = False
     assert np.array_equal(D2[untouched].view(np.uint32), D[untouched].view(np.uint32)) and hdr[3] == 3
+
+
+# ---------------------------------------------------------------- operand trials in the write-back form (Eq. 1-2)
+
+@pytest.mark.parametrize("dtype", [orc.FP16, orc.BF16, orc.TF32])
+def test_operand_writeback_is_exact_on_integers(dtype):
+    """With small integers nothing rounds: Eq. 1-2 on the finished sum gives the recomputed row / column exactly,
+    c' - c = (x' - x) * y, and the two forms of an operand trial give identical records. A swapped sign in Eq. 1,
+    a wrong factor y (row/column mix-up) or the clean operand used twice all fail here."""
+    M, N, K = 6, 7, 9
+    a, b, A, Bt = int_operands(dtype, M, N, K, 31, lo=1, hi=5)
+    Cclean, *_ = orc.gemm(dtype, A, Bt)
+    sign = 18 if dtype == orc.TF32 else 15
+    exp_lsb = {orc.FP16: 10, orc.BF16: 7, orc.TF32: 10}[dtype]
+    sites = np.concatenate([site(orc.KIND_A, row=2, k=5, mask=1 << sign), site(orc.KIND_A, row=5, k=0, mask=1 << exp_lsb),
+                            site(orc.KIND_B, col=3, k=8, mask=1 << sign), site(orc.KIND_B, col=6, k=2, mask=1 << exp_lsb)])
+    for s in sites:
+        isA = s["kind"] == orc.KIND_A
+        v0 = orc.operand_trial_values(dtype, A, Bt, Cclean, s, form=0)
+        v1 = orc.operand_trial_values(dtype, A, Bt, Cclean, s, form=1)
+        assert np.array_equal(v0.view(np.uint32), v1.view(np.uint32)) and len(v1) == (N if isA else M)
+        x = a[s["row"], s["k"]] if isA else b[s["col"], s["k"]]
+        word = int(A[s["row"], s["k"]]) if isA else int(Bt[s["col"], s["k"]])
+        xf = orc.widen(dtype, orc.flip_operand(dtype, word, int(s["xor_mask"])))
+        y = b[:, s["k"]] if isA else a[:, s["k"]]
+        c = Cclean[s["row"], :] if isA else Cclean[:, s["col"]]
+        assert np.array_equal(v1.astype(np.float64) - c.astype(np.float64), (xf - float(x)) * y.astype(np.float64))
+        Cf, *_ = orc.gemm(dtype, A, Bt, s.reshape(1))
+        assert np.array_equal(v1, Cf[s["row"], :] if isA else Cf[:, s["col"]])
+    for mode in (orc.T_NONE, orc.T_BOUND | orc.CORRECT):
+        r0 = orc.campaign(dtype, A, Bt, Cclean, sites, mode, operand_form=0)
+        r1 = orc.campaign(dtype, A, Bt, Cclean, sites, mode, operand_form=1)
+        assert np.array_equal(r0.view(np.uint8), r1.view(np.uint8))
+        assert (r1["status"] & 1).all() and (r1["n_affected"] == [N, N, M, M]).all()
+
+
+@pytest.mark.parametrize("dtype", [orc.FP16, orc.BF16, orc.TF32])
+def test_operand_writeback_on_rounded_data(dtype):
+    """Away from exact data the write-back form is the finished sum with two more roundings: within
+    2^-23 (|c| + |x y| + |x' y|) of (c - x y + x' y) taken exactly, and the order is Eq. 1 then Eq. 2."""
+    from fractions import Fraction
+    M, N, K = 7, 6, 40
+    rng = np.random.default_rng(32)
+    A = synth.round_to_storage(rng.standard_normal((M, K)).astype(np.float32), dtype)
+    Bt = synth.round_to_storage(rng.standard_normal((N, K)).astype(np.float32), dtype)
+    Cclean, *_ = orc.gemm(dtype, A, Bt)
+    width = 19 if dtype == orc.TF32 else 16
+    order_matters = 0
+    for t in range(24):
+        isA = t % 2 == 0
+        s = site(orc.KIND_A if isA else orc.KIND_B, row=int(rng.integers(0, M)), col=int(rng.integers(0, N)),
+                 k=int(rng.integers(0, K)), mask=1 << int(rng.integers(0, width - 2)))[0]
+        word = int(A[s["row"], s["k"]]) if isA else int(Bt[s["col"], s["k"]])
+        x = Fraction(orc.widen(dtype, word)); xf = Fraction(orc.widen(dtype, orc.flip_operand(dtype, word, int(s["xor_mask"]))))
+        v1 = orc.operand_trial_values(dtype, A, Bt, Cclean, s, form=1)
+        v0 = orc.operand_trial_values(dtype, A, Bt, Cclean, s, form=0)
+        ap = orc.absprod(dtype, A, Bt)
+        for o in range(len(v1)):
+            y = Fraction(orc.widen(dtype, int(Bt[o, s["k"]]) if isA else int(A[o, s["k"]])))
+            c = Cclean[s["row"], o] if isA else Cclean[o, s["col"]]
+            exact = Fraction(float(c)) - x * y + xf * y                # products of two operands are exact in FP32
+            bound = Fraction(2) ** -23 * (abs(Fraction(float(c))) + abs(x * y) + abs(xf * y))
+            assert abs(Fraction(float(v1[o])) - exact) <= bound
+            # Eq. 1 then Eq. 2, each rounded once (a float32 difference or sum of two float32 numbers of similar size
+            # is exact in double, so one conversion to float32 is the single rounding)
+            rep = np.float32(float(Fraction(float(c)) - x * y))
+            want = np.float32(float(Fraction(float(rep)) + xf * y))
+            assert f32_bits(float(v1[o])) == f32_bits(float(want))
+            other = np.float32(float(Fraction(float(np.float32(float(Fraction(float(c)) + xf * y)))) - x * y))
+            order_matters += int(f32_bits(float(other)) != f32_bits(float(want)))
+            # and the recompute is the same number up to the accumulated rounding of both chains
+            i_, j_ = (s["row"], o) if isA else (o, s["col"])
+            assert abs(float(v0[o]) - float(v1[o])) <= 2 * K * 2.0 ** -24 * (ap[i_, j_] + float(abs(xf * y)))
+    assert order_matters > 0        # the data does tell the two orders apart
