@@ -165,7 +165,7 @@ typedef struct {
 
 /*
  * One record per campaign trial (48 bytes). A trial is one site applied alone to
- * the clean GEMM ("a single fault is injected in each trial", Section IV-A).
+ * the clean GEMM (one fault per trial, Section IV-A).
  *   status        bit0 changed (some affected element's final bits differ from the
  *                 clean ones: the complement of the paper's "zero difference",
  *                 Section V-B), bit1 detected, bit2 corrected, bit8 invalid site

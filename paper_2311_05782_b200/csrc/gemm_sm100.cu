@@ -1225,12 +1225,6 @@ cudaError_t gemm_launch_slot(uint32_t *epoch, uint32_t **signals, uint32_t **rea
     return cudaSuccess;
 }
 
-int gemm_stage_count(int bn, bool pair)
-{
-    if (pair) return Cfg<256, true>::STAGES;
-    return bn == 256 ? Cfg<256, false>::STAGES : (bn == 128 ? Cfg<128, false>::STAGES : Cfg<64, false>::STAGES);
-}
-
 cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c,
                         const GemmParams &p, int grid, cudaStream_t stream)
 {

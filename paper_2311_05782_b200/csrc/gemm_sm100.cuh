@@ -51,9 +51,6 @@ constexpr int LAUNCH_SLOTS = 16;
 constexpr int LAUNCH_SLOT_WORDS = SPLIT_SIGNAL_WORDS + 16;
 cudaError_t gemm_launch_slot(uint32_t *epoch, uint32_t **signals, uint32_t **ready);
 
-// shared-memory pipeline depth used for an output tile that is bn columns wide
-int gemm_stage_count(int bn, bool pair);
-
 // Single mode (pair = false): bn in {64, 128, 256} is the width of the 128-row output tile; tm_b
 // must have been encoded with a box of (128 bytes x bn rows); `grid` CTAs; p.tiles_m counts
 // 128-row tiles.

@@ -217,7 +217,8 @@ def _widen_np(dtype, bits):
 @pytest.mark.parametrize("mode", [orc.T_NONE, orc.T_BOUND | orc.CORRECT])
 def test_operand_trials_are_eq1_eq2_on_the_clean_sum_bit_for_bit(dtype, shape, n, mode):
     """An operand trial's statistics are those of Eq. 1-2 applied to the device's own clean C with every product and
-    every sum rounded to FP32, bit for bit: numpy float32 arithmetic (one rounding per operation) restates it.
+    every sum rounded to FP32, bit for bit: first against the oracle's write-back form (all record fields), then
+    against numpy float32 arithmetic (one rounding per operation) restated here.
     Covers the row-panel kernel (long columns: the first two and the last two shapes, the last two with several groups of
     1024 column trials, so that full and partial groups and their bank-wise dealing to warps all occur) and the
     one-CTA-per-trial kernel."""
@@ -231,6 +232,16 @@ def test_operand_trials_are_eq1_eq2_on_the_clean_sum_bit_for_bit(dtype, shape, n
     width = 19 if dtype == orc.TF32 else 16
     s["xor_mask"] = [1 << int(b) for b in rng.integers(0, width, n)]
     Cg, rec = run_gpu_campaign(dtype, A, Bt, s, mode)
+    # the oracle's form of the same thing: Eq. 1-2 on the finished sums of the clean C the device produced
+    rw = orc.campaign(dtype, A, Bt, Cg, s, mode, operand_form=1)
+    # a faulty operand that is Inf or NaN puts NaNs among the values (Inf * 0); what the correction makes of a NaN
+    # depends on its payload, which is left open
+    special = ~np.isfinite(np.array([orc.widen(dtype, int(x)) for x in rw["after_bits"]]))
+    for f in rec.dtype.names:
+        same = rec[f] == rw[f]
+        if f in ("max_abs_dev", "status"):
+            same |= special
+        assert same.all(), (f, np.nonzero(~same)[0][:5], rec[~same][:2], rw[~same][:2])
     HASH_MUL = 0x9E3779B97F4A7C15
     with np.errstate(all="ignore"):
         for t in range(n):

@@ -1,9 +1,10 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py times (default tile policy).
 
-c1 and c2 are compared in full against the oracle (the oracle's 4096^3 GEMM takes seconds on the host cores).
-The larger configs are compared on sampled outputs that the oracle computes one by one, plus properties
-that hold at any size (flag count = popcount of the bitmap, a flag exactly where the stored value calls for
-one, untouched rows/columns bit-identical to the fault-free run).
+Every config is compared in full against the oracle: every element of C, the whole flag bitmap, the header
+counts and the site log of a GEMM with 16 or more sites of the config's mix, then the campaign's records (the
+oracle's GEMM takes seconds at these sizes on the host cores, about half a minute for the 8192^3 one). The
+sampled-output test that follows adds properties that hold at any size (flag count = popcount of the bitmap,
+untouched rows / columns bit-identical to the fault-free run).
 """
 import numpy as np
 import pytest
@@ -12,7 +13,8 @@ import torch
 import oracle as orc
 import paper_2311_05782_b200 as mpg
 import synth
-from parity import TOL, bits_f32, close, run_gpu_campaign, run_gpu_gemm, to_dev
+from parity import (TOL, absprod_fast, bits_f32, check_campaign_against_oracle, check_gemm_against_oracle,
+                    check_operand_trial, close, run_gpu_campaign, run_gpu_gemm, to_dev)
 
 pytestmark = pytest.mark.gpu
 
@@ -55,14 +57,13 @@ def test_c2_full_size_gemm_and_campaign():
     ro = orc.campaign(w.dtype, w.A, w.Bt, Cclean, w.sites, w.detect_mode)
     for f in ("kind", "primary_index", "before_bits", "after_bits", "final_bits", "n_affected"):
         assert np.array_equal(rec[f], ro[f]), f
-    fragile = (rec["n_detected"] != ro["n_detected"]) | (rec["idx_hash"] != ro["idx_hash"])
-    assert fragile.sum() <= 1, f"{fragile.sum()} trials disagree on their detected sets"
-    good = ~fragile
-    assert np.array_equal(rec["first_detected"][good], ro["first_detected"][good])
-    assert np.array_equal(rec["status"][good] & 6, ro["status"][good] & 6)
     assert (rec["n_detected"] > 0).sum() > 20        # exponent-MSB flips of an operand light up a whole row/column
-    dev_ok = close(rec["max_abs_dev"], ro["max_abs_dev"], 1e-3 * np.abs(ro["max_abs_dev"]) + 1e-3)
-    assert dev_ok[good].all()
+    # every trial: bit for bit against Eq. 1-2 on the device's clean C; against the recompute the detected sets, the
+    # status bits and the largest deviation, element by element wherever the two records are not identical (and on
+    # every 64th trial regardless)
+    rw = orc.campaign(w.dtype, w.A, w.Bt, Cc, w.sites, w.detect_mode, operand_form=1)
+    for t, st in enumerate(w.sites):
+        check_operand_trial(w.dtype, w.A, w.Bt, st, w.detect_mode, Cc, Cclean, rec[t], ro[t], rw[t], deep=t % 64 == 0)
 
 
 def test_c1_full_size_all_trials_in_one_gemm_and_as_campaign():
@@ -70,6 +71,26 @@ def test_c1_full_size_all_trials_in_one_gemm_and_as_campaign():
     w = synth.make_workload("c1")
     check_gemm_against_oracle(w.dtype, w.A, w.Bt, w.sites, w.detect_mode, max_fragile=1)
     check_campaign_against_oracle(w.dtype, w.A, w.Bt, w.sites, w.detect_mode, max_fragile=1)
+
+
+@pytest.mark.parametrize("name,n_sites,n_trials", [("c3a", 24, 4096), ("c3b", 24, 4096), ("c4", 16, 2048), ("c5", 48, 2048)])
+def test_large_configs_whole(name, n_sites, n_trials):
+    """The whole output of a faulty GEMM at the benchmark's size and default launch policy (so with the tile order and,
+    where it applies, the cut last round that bench.py times): every element within tolerance of the oracle's, flag
+    bitmap, header and site log word for word; then the campaign's records for the config's trial table (c5: the
+    first 2048 of its 100000 trials -- a column trial costs the oracle half a billion multiply-adds)."""
+    w = synth.make_workload(name, trials=max(n_trials, n_sites))
+    sites = w.sites[:n_sites].copy()
+    # sites at tile corners and seams as well as where the generator put them
+    M, N = w.M, w.N
+    corners = [(0, 0), (M - 1, N - 1), (127, N - 1), (128, 0), (255, min(255, N - 1)), (256, min(256, N - 1)), (M - 129, N // 2)]
+    movable = [t for t in range(n_sites) if int(sites["kind"][t]) in (orc.KIND_OUT, orc.KIND_ACC)][:len(corners)]
+    for t, (i, j) in zip(movable, corners):
+        sites["row"][t] = i; sites["col"][t] = j
+    check_gemm_against_oracle(w.dtype, w.A, w.Bt, sites, w.detect_mode, max_fragile=1, fast_tol=True)
+    Cclean, *_ = orc.gemm(w.dtype, w.A, w.Bt)
+    check_campaign_against_oracle(w.dtype, w.A, w.Bt, w.sites[:n_trials], w.detect_mode, max_fragile=2, Cclean=Cclean,
+                                  ap=absprod_fast(w.dtype, w.A, w.Bt), deep_every=0 if name != "c5" else 500)
 
 
 @pytest.mark.parametrize("name", ["c3a", "c3b", "c4", "c5"])
