@@ -12,7 +12,10 @@
  * A GEMM launch that has a flags buffer, or whose last round of tiles is cut (see
  * mpgemmfi_set_split_policy), carries a tag drawn from a counter when the entry point is
  * called, and uses one of 16 slots of a 160 KB static device array for the words its CTAs
- * hand to each other: launches on several streams may overlap, but a launch recorded once
+ * hand to each other. Launches on several streams may overlap. A slot comes round again
+ * every 16 such launches; the seventeenth is made to wait, on the device and in stream
+ * order (an event per slot, no host synchronisation), until the launch that last held
+ * its slot has finished, so any number of launches may be queued. A launch recorded once
  * and replayed (a CUDA graph) would reuse its tag and is not supported.
  *
  * Operation (paper Section II-B, IV-C): D = A x B with A (M x K) and B (K x N) in a
@@ -361,6 +364,30 @@ enum {
     MPGEMMFI_SPLIT_ON = 2
 };
 int mpgemmfi_set_split_policy(int policy);
+
+/*
+ * Robustness knob (no counterpart in the paper): how long any single device-side wait of the GEMM
+ * kernel (on a shared-memory barrier, on another CTA's hand-over of a cut tile, on the cleared
+ * header) may last before the launch gives up. A launch that gives up frees its tensor memory,
+ * returns normally and reports MPGEMMFI_STATUS_WAIT_LIMIT in the flags header; its C is invalid;
+ * the device stays usable. ms in 1..60000, default 4000. Process-wide, read when a launch is
+ * queued. Returns MPGEMMFI_OK or MPGEMMFI_ERR_ARG.
+ */
+int mpgemmfi_set_wait_limit_ms(int ms);
+
+/*
+ * Test hook (no counterpart in the paper): while on, the CTAs that continue a cut tile (see
+ * mpgemmfi_set_split_policy) wait for a hand-over tag that nobody writes, so that their bounded
+ * wait runs out and the give-up path above can be exercised without any fault. Launches queued
+ * while it is on produce invalid results by design. Never switch it on outside a test.
+ */
+int mpgemmfi_debug_break_handover(int on);
+
+/*
+ * Host logic of the launch slots (no device needed): returns the slot (0..15) that the launch with
+ * counter value `counter` uses and stores its tag (29 bits, never 0) in *tag (if non-NULL).
+ */
+int mpgemmfi_debug_launch_slot(uint32_t counter, uint32_t *tag);
 
 /* k elements between two accumulator boundaries: 64 (FP16, BF16), 32 (TF32); 0 for a bad dtype. */
 int mpgemmfi_kstep(int dtype);

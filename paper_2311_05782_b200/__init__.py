@@ -19,4 +19,5 @@ from .binding import (  # noqa: F401
     mpgemmfi_validate_sites, mpgemmfi_strerror, mpgemmfi_last_cuda_error, mpgemmfi_version,
     gemm, campaign, split_flags, mpgemmfi_campaign_summary, campaign_summary,
     mpgemmfi_operand_exponents, mpgemmfi_gemm_ranged, mpgemmfi_gemm_addend,
+    mpgemmfi_set_wait_limit_ms, mpgemmfi_debug_break_handover, mpgemmfi_debug_launch_slot,
 )

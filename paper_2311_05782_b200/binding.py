@@ -45,7 +45,7 @@ _SYMBOLS = [
     "mpgemmfi_flags_bitmap_offset", "mpgemmfi_campaign_workspace_bytes", "mpgemmfi_validate_sites",
     "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version", "mpgemmfi_campaign_static",
     "mpgemmfi_set_tile_policy", "mpgemmfi_set_split_policy", "mpgemmfi_campaign_summary", "mpgemmfi_operand_exponents", "mpgemmfi_gemm_ranged",
-    "mpgemmfi_gemm_addend",
+    "mpgemmfi_gemm_addend", "mpgemmfi_set_wait_limit_ms", "mpgemmfi_debug_break_handover", "mpgemmfi_debug_launch_slot",
 ]
 
 
@@ -94,6 +94,12 @@ def load_library():
     L.mpgemmfi_set_tile_policy.argtypes = [i]
     L.mpgemmfi_set_split_policy.restype = i
     L.mpgemmfi_set_split_policy.argtypes = [i]
+    L.mpgemmfi_set_wait_limit_ms.restype = i
+    L.mpgemmfi_set_wait_limit_ms.argtypes = [i]
+    L.mpgemmfi_debug_break_handover.restype = i
+    L.mpgemmfi_debug_break_handover.argtypes = [i]
+    L.mpgemmfi_debug_launch_slot.restype = i
+    L.mpgemmfi_debug_launch_slot.argtypes = [C.c_uint32, C.POINTER(C.c_uint32)]
     L.mpgemmfi_kstep.restype = i
     L.mpgemmfi_kstep.argtypes = [i]
     L.mpgemmfi_flags_bytes.restype = sz
@@ -174,6 +180,23 @@ def mpgemmfi_set_tile_policy(policy):
 def mpgemmfi_set_split_policy(policy):
     """SPLIT_AUTO (0), SPLIT_OFF (1) or SPLIT_ON (2); process-wide."""
     return load_library().mpgemmfi_set_split_policy(policy)
+
+
+def mpgemmfi_set_wait_limit_ms(ms):
+    """How long a device-side wait of the GEMM kernel may last before the launch gives up (1..60000 ms, default 4000)."""
+    return load_library().mpgemmfi_set_wait_limit_ms(ms)
+
+
+def mpgemmfi_debug_break_handover(on):
+    """Test hook: make the continuation of a cut tile wait for a hand-over that never comes."""
+    return load_library().mpgemmfi_debug_break_handover(int(bool(on)))
+
+
+def mpgemmfi_debug_launch_slot(counter):
+    """(slot, tag) of the launch with the given counter value."""
+    tag = C.c_uint32(0)
+    slot = load_library().mpgemmfi_debug_launch_slot(int(counter) & 0xFFFFFFFF, C.byref(tag))
+    return slot, tag.value
 
 
 def mpgemmfi_kstep(dtype):

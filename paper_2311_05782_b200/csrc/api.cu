@@ -103,6 +103,8 @@ int encode_output_map(CUtensorMap *map, float *C, int M, int N)
 
 int g_tile_policy = MPGEMMFI_TILES_AUTO;
 int g_split_policy = MPGEMMFI_SPLIT_AUTO;
+int g_wait_limit_ms = 4000;
+int g_break_handover = 0;
 
 // Split schedule for `tiles` tiles on `walkers` tile walkers: fills the three schedule fields of p.
 // Off unless there is at least one full round, the left-over tiles number at most half the walkers,
@@ -201,14 +203,18 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
     while ((1 << p.log2_k) < K) ++p.log2_k;
     const int walkers = pair ? max_pairs : di.num_sms;
     p.epoch = 0; p.signals = nullptr; p.ready = nullptr;
+    p.wait_limit_ns = (uint64_t)g_wait_limit_ms * 1000000ull;
+    p.tag_skew = g_break_handover ? 4u : 0u;        // test hook: an expected part number that nobody writes
     choose_split(p, walkers);
+    int slot = -1;
     if (p.split_parts > 1 || flags) {
         // (the header and the site log of `flags` are cleared by the kernel itself)
-        const cudaError_t es = mpg::gemm_launch_slot(&p.epoch, &p.signals, &p.ready);
+        const cudaError_t es = mpg::gemm_slot_acquire(stream, &slot, &p.epoch, &p.signals, &p.ready);
         if (es != cudaSuccess) return cuda_fail(es);
     }
     const int grid = (p.num_tiles < walkers ? p.num_tiles : walkers) * (pair ? 2 : 1);
-    const cudaError_t e = mpg::launch_gemm(bn, pair, tm_a, tm_b, tm_c, p, grid, stream);
+    cudaError_t e = mpg::launch_gemm(bn, pair, tm_a, tm_b, tm_c, p, grid, stream);
+    if (e == cudaSuccess && slot >= 0) e = mpg::gemm_slot_release(slot, stream);
     return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
 }
 
@@ -380,6 +386,25 @@ int mpgemmfi_set_split_policy(int policy)
         return MPGEMMFI_ERR_ARG;
     g_split_policy = policy;
     return MPGEMMFI_OK;
+}
+
+int mpgemmfi_set_wait_limit_ms(int ms)
+{
+    if (ms < 1 || ms > 60000) return MPGEMMFI_ERR_ARG;
+    g_wait_limit_ms = ms;
+    return MPGEMMFI_OK;
+}
+
+int mpgemmfi_debug_break_handover(int on)
+{
+    g_break_handover = on ? 1 : 0;
+    return MPGEMMFI_OK;
+}
+
+int mpgemmfi_debug_launch_slot(uint32_t counter, uint32_t *epoch)
+{
+    if (epoch) *epoch = mpg::gemm_epoch_of(counter);
+    return mpg::gemm_slot_of(counter);
 }
 
 int mpgemmfi_kstep(int dtype)

@@ -30,7 +30,7 @@
 // accumulator site still meets the running sum. Parts in between sit after the walker's g-th full
 // tile. A part's hand-over is one flag word per epilogue warp in a per-launch slot of a static
 // device array; the waits on it are bounded like every other wait here.
-#include <atomic>
+#include <mutex>
 #include <cstdint>
 #include <type_traits>
 #include <cuda.h>
@@ -407,7 +407,7 @@ __device__ __forceinline__ uint32_t signal_load_acquire(const uint32_t *ptr)
 
 // bounded wait for *ptr == want; same give-up rules as mbar_wait
 __device__ __forceinline__ bool signal_wait(const uint32_t *ptr, uint32_t want, volatile uint32_t *abort_flag,
-                                            uint64_t limit_ns = 4000000000ull)
+                                            uint64_t limit_ns)
 {
     if (signal_load_acquire(ptr) == want) return true;
     uint64_t t0 = 0;
@@ -434,12 +434,12 @@ __device__ __forceinline__ bool signal_wait(const uint32_t *ptr, uint32_t want, 
 // threads of one half-warp pick up their own rows. (One 128-byte row per thread instead: 11 us per
 // tile, during which the main loop next to it stood still.) Returns false when the wait gave up.
 __device__ __forceinline__ bool load_partial(const float *C, uint32_t M, uint32_t N, const uint32_t *sig, uint32_t want,
-                                             volatile uint32_t *abort_flag, uint32_t row0, uint32_t col0, int pieces,
-                                             uint32_t t_dst, uint8_t *park, int lane, bool vec = true)
+                                             volatile uint32_t *abort_flag, uint64_t limit_ns, uint32_t row0, uint32_t col0,
+                                             int pieces, uint32_t t_dst, uint8_t *park, int lane, bool vec = true)
 {
     if (sig) {
         bool got = true;
-        if (lane == 0) got = signal_wait(sig, want, abort_flag);
+        if (lane == 0) got = signal_wait(sig, want, abort_flag, limit_ns);
         got = __shfl_sync(0xFFFFFFFFu, got, 0);
         if (!got) return false;
         __threadfence();
@@ -592,6 +592,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     uint8_t *stage_out = smem + STAGES * C::STAGE_BYTES;     // output staging of the epilogue warps
     Control *ctl = reinterpret_cast<Control *>(stage_out + OUT_STAGING_BYTES);
     volatile uint32_t *abort_flag = &ctl->abort_flag;
+    const uint64_t wait_ns = p.wait_limit_ns;       // how long any one wait below may last before the CTA gives up
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = kPair ? cluster_cta_rank() : 0u;          // 0 = leader of the pair
@@ -635,7 +636,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     }
     build_site_list<TM, BN>(p, ctl, gid, groups, first_site);
     // a CTA with sites writes log entries as it goes: not before CTA 0 has cleared the log
-    if (threadIdx.x == 0 && blockIdx.x != 0 && p.flags && ctl->site_count != 0) signal_wait(p.ready, p.epoch, abort_flag);
+    if (threadIdx.x == 0 && blockIdx.x != 0 && p.flags && ctl->site_count != 0) signal_wait(p.ready, p.epoch, abort_flag, wait_ns);
     tc_fence_before_sync();
     if constexpr (kPair) cluster_sync_all(); else __syncthreads();
     tc_fence_after_sync();
@@ -675,7 +676,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 const bool own_barrier = !kPair || leader || kt == next_op;
                 if (kPair && kt == next_op) next_op = scan_next_operand(tc, kt + 1, lane);
                 if (lane == 0) {
-                    ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag);
+                    ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, wait_ns);
                     if (ok) {
                         uint8_t *sa = smem + stage * C::STAGE_BYTES;
                         if (own_barrier) {
@@ -718,7 +719,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 uint32_t kt = scan_next_operand(tc, sg.kt0, lane);
                 while (kt < sg.kt1) {          // NONE is larger than any k-tile
                     const uint32_t g = steps_before + (kt - sg.kt0), stage = g % STAGES;
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->full[stage]), (own_phase >> stage) & 1u, abort_flag));
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->full[stage]), (own_phase >> stage) & 1u, abort_flag, wait_ns));
                     if (!ok) break;
                     own_phase ^= 1u << stage;
                     if (lane == 0) {
@@ -742,12 +743,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             set_tile(sg.tile);
             uint32_t next_op = NONE, next_b = NONE;
             if (has_sites) { next_op = scan_next_operand(tc, sg.kt0, lane); next_b = scan_next_boundary(tc, sg.kt0 + 1, lane); }
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_empty[as]), ap ^ 1u, abort_flag));
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_empty[as]), ap ^ 1u, abort_flag, wait_ns));
             if (!ok) break;
             const bool preloaded = starts_from_memory(p, sg);
             if (preloaded) {
                 // continued tile or addend: the epilogue warps put the starting accumulators into TMEM first
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_loaded[as]), (loaded_phase >> as) & 1u, abort_flag));
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_loaded[as]), (loaded_phase >> as) & 1u, abort_flag, wait_ns));
                 if (!ok) break;
                 loaded_phase ^= 1u << as;
             }
@@ -767,7 +768,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     const uint64_t desc0 = umma_smem_desc_sw128(smem_u32(smem));
                     uint32_t accumulate = kt == fresh_kt ? 0u : 1u;
                     for (; kt < stop; ++kt) {
-                        if (!mbar_wait(full0 + stage * 8u, phase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(full0 + stage * 8u, phase, abort_flag, wait_ns)) { ok = false; break; }
                         tc_fence_after_sync();
                         // the address field counts 16-byte units: stage s starts s * STAGE_BYTES / 16 further on
                         const uint64_t a_desc = desc0 + (uint64_t)(stage * (uint32_t)(C::STAGE_BYTES >> 4));
@@ -792,7 +793,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
               }
               // one k-tile with a site, by the whole warp
               {
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag));
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag, wait_ns));
                 if (!ok) break;
                 tc_fence_after_sync();
                 uint8_t *sa = smem + stage * C::STAGE_BYTES;
@@ -824,7 +825,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                         else umma_commit(smem_u32(&ctl->pause_full));
                     }
                     __syncwarp();
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->pause_done), pause_phase, abort_flag));
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->pause_done), pause_phase, abort_flag, wait_ns));
                     if (!ok) break;
                     pause_phase ^= 1u;
                     tc_fence_after_sync();
@@ -873,8 +874,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             __syncwarp();
             const uint32_t *sig = s.load ? p.signals + (size_t)(s.tile - first_left) * 16 + my_signal : nullptr;
             const uint32_t t_dst = tmem_base + buf * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)(first * 32);
-            if (!load_partial(s.load ? p.C : p.addend, (uint32_t)p.M, (uint32_t)p.N, sig, (p.epoch << 3) | s.part, abort_flag,
-                              tm * TM + rank * BM + (uint32_t)(q * 32), tn * BN + (uint32_t)(first * 32), MY_PIECES,
+            // (p.tag_skew is zero outside the tests, see GemmParams)
+            if (!load_partial(s.load ? p.C : p.addend, (uint32_t)p.M, (uint32_t)p.N, sig, ((p.epoch << 3) | s.part) ^ p.tag_skew,
+                              abort_flag, wait_ns, tm * TM + rank * BM + (uint32_t)(q * 32), tn * BN + (uint32_t)(first * 32), MY_PIECES,
                               t_dst, my_out, lane, s.load || p.addend_vec_ok != 0))
                 return false;
             tc_fence_before_sync();
@@ -903,7 +905,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             if (has_sites) {
                 uint32_t b = scan_next_boundary(tc, sg.kt0 + 1, lane);
                 while (b <= sg.kt1) {          // boundaries of this segment's k-tiles (NONE is larger than any)
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->pause_full), pause_phase, abort_flag));
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->pause_full), pause_phase, abort_flag, wait_ns));
                     if (!ok) break;
                     pause_phase ^= 1u;
                     tc_fence_after_sync();
@@ -919,7 +921,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 if (!ok) break;
                 tile_has_out = !sg.save && scan_has_out(tc, lane);
             }
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_full[as]), ap, abort_flag));
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->acc_full[as]), ap, abort_flag, wait_ns));
             if (!ok) break;
             tc_fence_after_sync();
 
@@ -1118,7 +1120,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         }
         if (lane == 0) bulk_wait_read_all();       // shared memory stays until the last store has read it
         n_det = __reduce_add_sync(0xFFFFFFFFu, n_det);
-        if (lane == 0 && n_det && p.flags && (blockIdx.x == 0 || signal_wait(p.ready, p.epoch, abort_flag))) {
+        if (lane == 0 && n_det && p.flags && (blockIdx.x == 0 || signal_wait(p.ready, p.epoch, abort_flag, wait_ns))) {
             atomicAdd(&p.flags[1], n_det);
             if (want_corr) atomicAdd(&p.flags[2], n_det);
         }
@@ -1204,25 +1206,60 @@ namespace {
 __device__ uint32_t g_launch_slots[LAUNCH_SLOTS][LAUNCH_SLOT_WORDS];
 }
 
-cudaError_t gemm_launch_slot(uint32_t *epoch, uint32_t **signals, uint32_t **ready)
+namespace {
+struct SlotState {
+    uint32_t *base = nullptr;            // device address of g_launch_slots
+    cudaEvent_t done[LAUNCH_SLOTS] = {};  // recorded behind the last launch that used the slot
+    bool used[LAUNCH_SLOTS] = {};
+};
+SlotState g_slot_state[64];
+std::mutex g_slot_mutex;
+uint32_t g_launch_counter = 0;
+}
+
+cudaError_t gemm_slot_acquire(cudaStream_t stream, int *slot, uint32_t *epoch, uint32_t **signals, uint32_t **ready)
 {
-    static uint32_t *base[64] = {};
-    static std::atomic<uint32_t> counter{0};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!base[dev]) {
+    std::lock_guard<std::mutex> lock(g_slot_mutex);
+    SlotState &st = g_slot_state[dev];
+    if (!st.base) {
         void *ptr = nullptr;
         e = cudaGetSymbolAddress(&ptr, g_launch_slots);
         if (e != cudaSuccess) return e;
-        base[dev] = static_cast<uint32_t *>(ptr);
+        for (int i = 0; i < LAUNCH_SLOTS; ++i) {
+            e = cudaEventCreateWithFlags(&st.done[i], cudaEventDisableTiming);
+            if (e != cudaSuccess) return e;
+        }
+        st.base = static_cast<uint32_t *>(ptr);
     }
-    const uint32_t n = counter.fetch_add(1u) + 1u;
-    *epoch = n & 0x1FFFFFFFu ? n & 0x1FFFFFFFu : 1u;     // 29 bits (3 more carry the part number), never 0
-    *signals = base[dev] + (size_t)(n % LAUNCH_SLOTS) * LAUNCH_SLOT_WORDS;
+    const uint32_t n = ++g_launch_counter;
+    const int sl = gemm_slot_of(n);
+    if (st.used[sl]) {
+        // the launch that had this slot LAUNCH_SLOTS launches ago may still be running on another stream
+        e = cudaStreamWaitEvent(stream, st.done[sl], 0);
+        if (e != cudaSuccess) return e;
+    }
+    *slot = sl;
+    *epoch = gemm_epoch_of(n);
+    *signals = st.base + (size_t)sl * LAUNCH_SLOT_WORDS;
     *ready = *signals + SPLIT_SIGNAL_WORDS;
     return cudaSuccess;
+}
+
+cudaError_t gemm_slot_release(int slot, cudaStream_t stream)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || slot < 0 || slot >= LAUNCH_SLOTS) return cudaErrorInvalidValue;
+    std::lock_guard<std::mutex> lock(g_slot_mutex);
+    SlotState &st = g_slot_state[dev];
+    e = cudaEventRecord(st.done[slot], stream);
+    if (e == cudaSuccess) st.used[slot] = true;
+    return e;
 }
 
 cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c,

@@ -38,6 +38,12 @@ struct GemmParams {
     // With a flags buffer: CTA 0 clears the header and the site log when it starts, then stores `epoch`
     // here (release); any other CTA reads it (acquire, bounded wait) before it touches header or log.
     uint32_t *ready;
+    // Every device-side wait (on a barrier, a hand-over word, *ready) gives up after this many nanoseconds; the
+    // launch then ends with MPGEMMFI_STATUS_WAIT_LIMIT in the flags header instead of hanging.
+    uint64_t wait_limit_ns;
+    // XORed into the tag that the consumer of a cut tile waits for. Zero in every real launch; the tests set it so
+    // that a hand-over never arrives and the give-up path runs.
+    uint32_t tag_skew;
 };
 
 // hand-over words one launch can use: 16 per left-over tile, fewer left-over tiles than walkers
@@ -45,11 +51,20 @@ constexpr int SPLIT_MAX_WALKERS = 160;
 constexpr int SPLIT_SIGNAL_WORDS = SPLIT_MAX_WALKERS * 16;
 
 // Gives a launch its tag, its hand-over words and its ready word: a slot of a static device array,
-// slots handed out in turn (a slot comes round again after LAUNCH_SLOTS launches; the tag keeps a
-// launch from reading what an earlier one left there).
+// slots handed out in turn. A slot comes round again after LAUNCH_SLOTS launches; the tag keeps a
+// launch from reading what an earlier one left there, and an event per slot keeps a launch from
+// starting on a slot whose previous launch (on whatever stream) is still running:
+// gemm_slot_acquire makes `stream` wait for that launch, gemm_slot_release (after the kernel has been
+// queued on `stream`) records the slot's event there. The first acquire on a device creates the
+// events. Both are cheap and never block the host.
 constexpr int LAUNCH_SLOTS = 16;
 constexpr int LAUNCH_SLOT_WORDS = SPLIT_SIGNAL_WORDS + 16;
-cudaError_t gemm_launch_slot(uint32_t *epoch, uint32_t **signals, uint32_t **ready);
+cudaError_t gemm_slot_acquire(cudaStream_t stream, int *slot, uint32_t *epoch, uint32_t **signals, uint32_t **ready);
+cudaError_t gemm_slot_release(int slot, cudaStream_t stream);
+// slot index a launch counter value maps to (host logic, testable without a device)
+inline int gemm_slot_of(uint32_t counter) { return (int)(counter % (uint32_t)LAUNCH_SLOTS); }
+// 29-bit tag of a launch counter value, never 0 (three more bits carry a part number)
+inline uint32_t gemm_epoch_of(uint32_t counter) { return (counter & 0x1FFFFFFFu) ? (counter & 0x1FFFFFFFu) : 1u; }
 
 // Single mode (pair = false): bn in {64, 128, 256} is the width of the 128-row output tile; tm_b
 // must have been encoded with a box of (128 bytes x bn rows); `grid` CTAs; p.tiles_m counts

@@ -60,7 +60,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait. Gives up after `limit_ns` or as soon as another thread of the CTA
 // has given up (*abort_flag != 0); on giving up it raises *abort_flag itself.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          uint64_t limit_ns = 4000000000ull)
+                                          uint64_t limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t t0 = 0;

@@ -167,3 +167,76 @@ def test_random_shapes_under_split_schedule(seed, policies):
     mpg.mpgemmfi_set_tile_policy([mpg.TILES_PAIR, mpg.TILES_SINGLE][seed % 2])
     mpg.mpgemmfi_set_split_policy(mpg.SPLIT_ON)
     check_gemm_against_oracle(dtype, A, Bt, s, mode, max_fragile=2)
+
+
+def test_more_launches_in_flight_than_slots(policies):
+    """24 split-schedule GEMMs with flags buffers queued on 4 streams before any has finished: more than the 16
+    hand-over slots. A launch that gets a slot for the second time waits (in stream order, on the device) for the
+    launch that held it before, so every result equals the one of the same GEMM run alone."""
+    dtype = orc.BF16
+    M, N, K = 2304, 2304, 2048
+    mpg.mpgemmfi_set_tile_policy(mpg.TILES_PAIR)
+    mpg.mpgemmfi_set_split_policy(mpg.SPLIT_ON)
+    A, Bt = rand_operands(dtype, M, N, K, 60)
+    sites = site_table(dtype, M, N, K, 32, 61)
+    a, b = to_dev(A, dtype), to_dev(Bt, dtype)
+    sd = torch.from_numpy(sites.view(np.int32).reshape(-1, 8)).cuda()
+    Cg, flags = mpg.gemm(dtype, a, b, sites, orc.T_BOUND | orc.CORRECT)
+    torch.cuda.synchronize()
+    want_c, want_f = Cg.cpu().numpy().view(np.uint32), flags.cpu().numpy()
+    assert want_f.view(np.uint32)[5] >= 2                 # the last round is cut: the hand-over words are in use
+    n_launch = 24
+    streams = [torch.cuda.Stream() for _ in range(4)]
+    outs = [(torch.empty((M, N), dtype=torch.float32, device="cuda"),
+             torch.empty(mpg.mpgemmfi_flags_bytes(M, N, 32) // 4, dtype=torch.int32, device="cuda")) for _ in range(n_launch)]
+    torch.cuda.synchronize()
+    for i, (c, f) in enumerate(outs):
+        rc = mpg.mpgemmfi_gemm(dtype, M, N, K, a.data_ptr(), b.data_ptr(), c.data_ptr(), sd.data_ptr(), 32,
+                               orc.T_BOUND | orc.CORRECT, f.data_ptr(), streams[i % 4].cuda_stream)
+        assert rc == 0
+    torch.cuda.synchronize()
+    for i, (c, f) in enumerate(outs):
+        fg = f.cpu().numpy()
+        assert not (int(fg[0]) & mpg.STATUS_WAIT_LIMIT), i
+        assert np.array_equal(fg, want_f), i
+        assert np.array_equal(c.cpu().numpy().view(np.uint32), want_c), i
+
+
+def test_a_wait_that_runs_out_ends_the_launch_with_a_status(policies):
+    """The give-up path of the bounded waits, made to run without any fault: with the test hook on, the CTAs that
+    continue a cut tile wait for a hand-over tag that nobody writes; with the limit set to a few milliseconds the wait
+    runs out, every warp of the CTA (pair) leaves its loop, tensor memory is released, the kernel returns, and the
+    header says WAIT_LIMIT. The device stays usable: the same GEMM queued next, with the hook off, gives bit for bit
+    what it gave before."""
+    dtype = orc.BF16
+    M, N, K = 2560, 2560, 1024                            # 100 tiles of 256 x 256 on 74 pairs: 26 left over, cut in two
+    mpg.mpgemmfi_set_tile_policy(mpg.TILES_PAIR)
+    mpg.mpgemmfi_set_split_policy(mpg.SPLIT_ON)
+    A, Bt = rand_operands(dtype, M, N, K, 70)
+    sites = site_table(dtype, M, N, K, 16, 71)
+    a, b = to_dev(A, dtype), to_dev(Bt, dtype)
+    C0, f0 = mpg.gemm(dtype, a, b, sites, orc.T_BOUND)
+    torch.cuda.synchronize()
+    want_c, want_f = C0.cpu().numpy().view(np.uint32), f0.cpu().numpy().view(np.uint32)
+    assert want_f[5] >= 2 and not (want_f[0] & mpg.STATUS_WAIT_LIMIT)
+    try:
+        assert mpg.mpgemmfi_set_wait_limit_ms(3) == 0
+        assert mpg.mpgemmfi_debug_break_handover(1) == 0
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        C1, f1 = mpg.gemm(dtype, a, b, sites, orc.T_BOUND)
+        t1.record()
+        torch.cuda.synchronize()
+    finally:
+        mpg.mpgemmfi_debug_break_handover(0)
+        mpg.mpgemmfi_set_wait_limit_ms(4000)
+    got = f1.cpu().numpy().view(np.uint32)
+    assert got[0] & mpg.STATUS_WAIT_LIMIT, "the launch did not report that a wait ran out"
+    assert t0.elapsed_time(t1) < 3000.0                  # it gave up after milliseconds (plus the drain), not seconds
+    # the whole tiles of that launch did not depend on the hand-over and are as before
+    assert np.array_equal(C1.cpu().numpy().view(np.uint32)[:256, :256], want_c[:256, :256])
+    # the next ordinary launch: everything as in the first one
+    C2, f2 = mpg.gemm(dtype, a, b, sites, orc.T_BOUND)
+    torch.cuda.synchronize()
+    assert np.array_equal(f2.cpu().numpy().view(np.uint32), want_f)
+    assert np.array_equal(C2.cpu().numpy().view(np.uint32), want_c)

@@ -39,6 +39,8 @@ def test_host_helpers():
     # tuning knobs: argument checks need no device
     assert mpg.mpgemmfi_set_tile_policy(7) == -1 and mpg.mpgemmfi_set_tile_policy(mpg.TILES_AUTO) == 0
     assert mpg.mpgemmfi_set_split_policy(-1) == -1 and mpg.mpgemmfi_set_split_policy(mpg.SPLIT_AUTO) == 0
+    assert mpg.mpgemmfi_set_wait_limit_ms(0) == -1 and mpg.mpgemmfi_set_wait_limit_ms(60001) == -1
+    assert mpg.mpgemmfi_set_wait_limit_ms(4000) == 0
     # struct sizes the ABI promises
     assert mpg.SITE_DTYPE.itemsize == 32 and mpg.SITE_LOG_DTYPE.itemsize == 16 and mpg.RECORD_DTYPE.itemsize == 48
 
@@ -55,3 +57,19 @@ def test_validate_sites_rules():
     s["row"][3] = 8
     assert mpg.mpgemmfi_validate_sites(s, mpg.TF32, 8, 8, 100) == (-4, 3)
     assert mpg.mpgemmfi_validate_sites(s, 5, 8, 8, 100)[0] == -2
+
+
+def test_launch_slots_and_tags():
+    """Slots are handed out in turn, 16 of them; a launch's tag is its counter value in 29 bits and never 0 (0 is what
+    a never-used hand-over word holds), also where the counter wraps."""
+    seen = [mpg.mpgemmfi_debug_launch_slot(n) for n in range(1, 40)]
+    assert [s for s, _ in seen] == [n % 16 for n in range(1, 40)]
+    assert [t for _, t in seen] == list(range(1, 40))
+    for n in (0x20000000, 0x40000000, 0xE0000000, 0):
+        slot, tag = mpg.mpgemmfi_debug_launch_slot(n)
+        assert tag == 1 and slot == 0
+    slot, tag = mpg.mpgemmfi_debug_launch_slot(0x3FFFFFFF)
+    assert tag == 0x1FFFFFFF and slot == 15
+    # two launches that share a slot never share a tag unless 2^29 launches lie between them
+    assert mpg.mpgemmfi_debug_launch_slot(5)[1] != mpg.mpgemmfi_debug_launch_slot(21)[1]
+    assert mpg.mpgemmfi_debug_launch_slot(5)[0] == mpg.mpgemmfi_debug_launch_slot(21)[0]
