@@ -52,7 +52,10 @@ constexpr int NUM_THREADS = 384;     // 4 control warps + 8 epilogue warps
 constexpr int EPI_WARPS = 8;
 constexpr int SITE_CACHE = 64;
 constexpr int MAX_STAGES = 8;
-constexpr int OUT_STAGING_BYTES = EPI_WARPS * 16 * 128;   // a 16-row x 32-column FP32 block per epilogue warp
+constexpr int OUT_BUF_BYTES = 16 * 128;                    // staging of one epilogue warp: 16 rows x 128 bytes
+constexpr int OUT_STAGING_BYTES = EPI_WARPS * OUT_BUF_BYTES;
+constexpr int SMEM_BUDGET = 227 * 1024;                    // dynamic shared memory one CTA may have
+constexpr int CONTROL_RESERVE = 12 * 1024;                 // control block + 1 KB of alignment slack
 
 template <int BN, bool kPair>
 struct Cfg {
@@ -60,7 +63,10 @@ struct Cfg {
     static constexpr int A_BYTES = BM * 128;
     static constexpr int B_BYTES = B_ROWS * 128;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (200 * 1024 / STAGE_BYTES) < MAX_STAGES ? (200 * 1024 / STAGE_BYTES) : MAX_STAGES;
+    // the operand ring gets what the output staging and the control block leave
+    static constexpr int STAGES_FIT = (SMEM_BUDGET - CONTROL_RESERVE - OUT_STAGING_BYTES) / STAGE_BYTES;
+    static constexpr int STAGES = STAGES_FIT < MAX_STAGES ? STAGES_FIT : MAX_STAGES;
+    static_assert(STAGES >= 3, "operand ring too short");
     static constexpr int TMEM_COLS = 2 * BN;   // two accumulators; 128, 256 or 512 columns
     static_assert(BN == 64 || BN == 128 || BN == 256, "BN must be 64, 128 or 256");
     static_assert(!kPair || BN == 256, "pair tiles are 256 x 256");
@@ -858,7 +864,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         const int epi_mode = want_range ? EPI_RANGE : (want_bound ? (want_corr ? EPI_BOUND_CORRECT : EPI_BOUND) : EPI_PLAIN);
         uint32_t pause_phase = 0, n_det = 0;
         uint32_t *bitmap = p.flags ? p.flags + MPGEMMFI_HEADER_WORDS + 4 * (size_t)p.n_faults : nullptr;
-        uint8_t *my_out = stage_out + (warp - 4) * (16 * 128);
+        uint8_t *my_out = stage_out + (warp - 4) * OUT_BUF_BYTES;
+        // where this thread parks 16-byte chunk j of its row for a TMA store: park_addr ^ (j << 4) (128-byte swizzle:
+        // chunk j of row r sits at chunk position j ^ (r & 7))
+        const uint32_t park_addr = smem_u32(my_out) + ((uint32_t)lane & 15u) * 128u + (((uint32_t)lane & 7u) << 4);
         constexpr int MY_PIECES = BN / 64;          // 32-column pieces per warp (half the tile's columns)
         const int first = h * MY_PIECES;
         // hand-over words of this warp for left-over tile j: signals[j * 16 + my_signal]
@@ -966,23 +975,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                         if (c0 + jj < (uint32_t)p.N) crow[c0 + jj] = bits_f32(v[jj]);
                 }
             };
-            // The same for a finished tile when C allows 16-byte accesses: the rows are parked in the layout
-            // of the 128-byte swizzle and one thread hands them to the TMA engine (16 rows x 128 bytes a
-            // store). The warp does not wait for the store, only -- before it parks the next rows -- for
-            // its staging to have been read: the SM's write port (about 32 bytes a cycle) then drains one
-            // warp's rows while the other warps check and park theirs, instead of all eight warps
-            // checking together and then queueing behind the port together.
+            // The same for a finished tile when C allows 16-byte accesses: the rows are parked in the layout of the
+            // 128-byte swizzle and one thread hands them to the TMA engine (16 rows x 128 bytes a store, the two
+            // half-warps in turn). The warp does not wait for the store, only -- before it parks the next rows -- for
+            // its staging to have been read: the SM's write port (about 32 bytes a cycle) then drains one warp's rows
+            // while the other warps check and park theirs, instead of all eight warps checking together and then
+            // queueing behind the port together.
             auto store_piece_tma = [&](uint32_t (&v)[32], uint32_t c0) {
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     if (lane == 0) bulk_wait_read_all();
                     __syncwarp();
                     if ((lane >> 4) == half) {
-                        uint8_t *srow = my_out + (lane & 15) * 128;
 #pragma unroll
                         for (int jj = 0; jj < 8; ++jj)
-                            *reinterpret_cast<uint4 *>(srow + ((jj ^ (lane & 7)) << 4)) =
-                                make_uint4(v[4 * jj], v[4 * jj + 1], v[4 * jj + 2], v[4 * jj + 3]);
+                            st_shared_v4(park_addr ^ (uint32_t)(jj << 4), v[4 * jj], v[4 * jj + 1], v[4 * jj + 2], v[4 * jj + 3]);
                         fence_proxy_async_smem();
                     }
                     __syncwarp();
@@ -1031,10 +1038,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 constexpr bool do_range = kMode == EPI_RANGE;
                 const bool do_corr = kMode == EPI_BOUND_CORRECT || (kMode == EPI_RANGE && want_corr);
                 const uint32_t row_e = (do_range && row_ok) ? __ldg(p.exp_a + row) : 0u;
-                uint32_t flagw[MY_PIECES];
 
                 // One 32-column piece of this thread's row: output sites, check, flags, store.
-                auto finish_piece = [&](uint32_t (&v)[32], int i) {
+                auto finish_piece = [&](uint32_t (&v)[32], int i) -> uint32_t {
                     const uint32_t c0 = tc.n0 + (uint32_t)((first + i) * 32);
                     // output-level range check: this lane fetches the exponent maximum of column c0 + lane early
                     uint32_t col_e = 0;
@@ -1057,9 +1063,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     if constexpr (do_bound) {
                         // A flagged element has exponent bit 7 (word bit 30) set. The OR of the 32 words costs a
                         // third of the per-element test and settles the usual case (every |value| < 2) at once.
-                        uint32_t any = 0;
+                        uint32_t o8[8];
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) any |= v[j];
+                        for (int j = 0; j < 8; ++j) o8[j] = (v[4 * j] | v[4 * j + 1]) | (v[4 * j + 2] | v[4 * j + 3]);
+                        const uint32_t any = ((o8[0] | o8[1]) | (o8[2] | o8[3])) | ((o8[4] | o8[5]) | (o8[6] | o8[7]));
                         if (any & 0x40000000u) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
@@ -1074,41 +1081,41 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                         if (c0 + 32 > (uint32_t)p.N) fw &= c0 < (uint32_t)p.N ? (1u << ((uint32_t)p.N - c0)) - 1u : 0u;
                     }
                     if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 1);
-                    flagw[i] = fw;
                     if (p.c_vec_ok) store_piece_tma(v, c0);
                     else store_piece(v, c0);
+                    return fw;
                 };
 
-                // software pipeline: the TMEM read of the next piece is in flight while this one is finished
+                // Software pipeline: the TMEM read of the next piece is in flight while this one is finished. Two
+                // pieces per trip of a loop that is NOT unrolled: the epilogue's code stays a quarter of what four
+                // inlined copies take, which is what the instruction cache can hold next to the other warps' loops.
                 uint32_t va[32], vb[32];
                 tmem_ld_32x32(t_first, va);
-#pragma unroll
+                uint32_t *frow = nullptr;
+                const uint32_t w0 = tc.n0 / 32 + (uint32_t)first;
+                if (bitmap && row_ok) frow = bitmap + (size_t)row * p.wpr + w0;
+#pragma unroll 1
                 for (int i = 0; i < MY_PIECES; i += 2) {
                     tmem_wait_ld();
                     if (i + 1 < MY_PIECES) tmem_ld_32x32(t_first + (uint32_t)((i + 1) * 32), vb);
                     else release_acc();
-                    finish_piece(va, i);
+                    const uint32_t fa = finish_piece(va, i);
+                    uint32_t fb = 0;
                     if (i + 1 < MY_PIECES) {
                         tmem_wait_ld();
                         if (i + 2 < MY_PIECES) tmem_ld_32x32(t_first + (uint32_t)((i + 2) * 32), va);
                         else release_acc();
-                        finish_piece(vb, i + 1);
+                        fb = finish_piece(vb, i + 1);
                     }
-                }
-                if (bitmap && row_ok) {
-                    const uint32_t w0 = tc.n0 / 32 + (uint32_t)first;
-                    uint32_t *frow = bitmap + (size_t)row * p.wpr + w0;
-                    if (MY_PIECES == 4 && (p.wpr & 3) == 0) {       // this thread's 4 words are 16-byte aligned
-                        if (w0 < (uint32_t)p.wpr)
-                            *reinterpret_cast<uint4 *>(frow) = make_uint4(flagw[0], flagw[MY_PIECES > 1 ? 1 : 0],
-                                                                           flagw[MY_PIECES > 2 ? 2 : 0], flagw[MY_PIECES > 3 ? 3 : 0]);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < MY_PIECES; ++i)
-                            if (w0 + i < (uint32_t)p.wpr) frow[i] = flagw[i];
+                    if (frow) {
+                        if (MY_PIECES > 1 && (p.wpr & 1) == 0) {          // this thread's two words are 8-byte aligned
+                            if (w0 + i < (uint32_t)p.wpr) *reinterpret_cast<uint2 *>(frow + i) = make_uint2(fa, fb);
+                        } else {
+                            if (w0 + i < (uint32_t)p.wpr) frow[i] = fa;
+                            if (i + 1 < MY_PIECES && w0 + i + 1 < (uint32_t)p.wpr) frow[i + 1] = fb;
+                        }
+                        n_det += __popc(fa) + __popc(fb);
                     }
-#pragma unroll
-                    for (int i = 0; i < MY_PIECES; ++i) n_det += __popc(flagw[i]);
                 }
             };
             switch (epi_mode) {
@@ -1147,6 +1154,7 @@ cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const C
 {
     using C = Cfg<BN, kPair>;
     const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024;
+    static_assert(C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024 <= SMEM_BUDGET, "shared memory over budget");
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -1182,6 +1190,7 @@ int gemm_max_resident_pairs(int dtype)
     if (cache[dev][tf] == 0) {
         using C = Cfg<256, true>;
         const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024;
+    static_assert(C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024 <= SMEM_BUDGET, "shared memory over budget");
         auto kern = tf ? gemm_kernel<256, true, true> : gemm_kernel<256, false, true>;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
         cudaLaunchConfig_t cfg = {};
