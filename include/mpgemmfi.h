@@ -226,6 +226,32 @@ int mpgemmfi_gemm_addend(int dtype, int M, int N, int K, const void *A, const vo
                          uint32_t *flags_out, mpgemmfi_stream stream);
 
 /*
+ * The same with a 16-bit result. The paper states the tensor-core operation as D = A x B + C with the
+ * products accumulated in FP32 (Section II-B) and runs its models in "16" / "bf16" precision from end
+ * to end (Section IV-B): the FP32 result of a layer's GEMM goes back to the 16-bit format before the
+ * next layer reads it. Here everything up to and including the output check happens on the FP32 values
+ * exactly as in mpgemmfi_gemm / mpgemmfi_gemm_addend (sites, flags, counts and the site log are those
+ * of the FP32 result); then each element is rounded once, to nearest with ties to even, to
+ * `out_format`: values beyond the format's range become infinities (FP16: |v| >= 65520), NaN stays
+ * NaN (payload unspecified).
+ *   C_in        NULL for D = A x B, or the FP32 addend (device, M x N, 4-byte aligned); it must not
+ *               overlap D16 (ERR_ARG).
+ *   out_format  MPGEMMFI_OUT_FP16 or MPGEMMFI_OUT_BF16 (ERR_DTYPE otherwise), independent of `dtype`.
+ *   D16         device pointer, M x N row-major 2-byte words, written in full (16-byte alignment and
+ *               N a multiple of 8 let it be written by bulk stores).
+ * The last round of tiles is never cut for this entry point (see mpgemmfi_set_split_policy).
+ * Everything else, and the errors, as for mpgemmfi_gemm.
+ */
+enum {
+    MPGEMMFI_OUT_FP32 = 0,  /* what the other entry points write; not accepted here */
+    MPGEMMFI_OUT_FP16 = 1,
+    MPGEMMFI_OUT_BF16 = 2
+};
+int mpgemmfi_gemm_out16(int dtype, int M, int N, int K, const void *A, const void *Bt, const float *C_in,
+                        int out_format, void *D16, const mpgemmfi_site *fault_sites, int n_faults,
+                        int detect_mode, uint32_t *flags_out, mpgemmfi_stream stream);
+
+/*
  * Largest FP32 exponent field of each row of a rows x K operand matrix (A, or Bt): out[r] in
  * 0..255; 0 for an all-zero row, 255 if the row holds Inf or NaN. X and out are device pointers
  * (X 16-byte aligned, K * element size a multiple of 16 bytes). Input of mpgemmfi_gemm_ranged.

@@ -17,6 +17,7 @@ SITE_A, SITE_B, SITE_ACC, SITE_OUT, SITE_TERM = 0, 1, 2, 3, 4
 DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP = 0, 1, 2, 3
 CORRECT = 16
 TERM_HMMA_STEP = 32
+OUT_FP32, OUT_FP16, OUT_BF16 = 0, 1, 2
 OUTPUT_RANGE = 64
 STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT = 1, 2
 MAX_FAULTS = 4096
@@ -46,6 +47,7 @@ _SYMBOLS = [
     "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version", "mpgemmfi_campaign_static",
     "mpgemmfi_set_tile_policy", "mpgemmfi_set_split_policy", "mpgemmfi_campaign_summary", "mpgemmfi_operand_exponents", "mpgemmfi_gemm_ranged",
     "mpgemmfi_gemm_addend", "mpgemmfi_set_wait_limit_ms", "mpgemmfi_debug_break_handover", "mpgemmfi_debug_launch_slot",
+    "mpgemmfi_gemm_out16",
 ]
 
 
@@ -80,6 +82,8 @@ def load_library():
     L.mpgemmfi_gemm.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp]
     L.mpgemmfi_gemm_addend.restype = i
     L.mpgemmfi_gemm_addend.argtypes = [i, i, i, i, vp, vp, vp, vp, vp, i, i, vp, vp]
+    L.mpgemmfi_gemm_out16.restype = i
+    L.mpgemmfi_gemm_out16.argtypes = [i, i, i, i, vp, vp, vp, i, vp, vp, i, i, vp, vp]
     L.mpgemmfi_campaign.restype = i
     L.mpgemmfi_campaign.argtypes = [i, i, i, i, vp, vp, vp, vp, i, i, vp, vp, sz, vp]
     L.mpgemmfi_campaign_static.restype = i
@@ -130,6 +134,12 @@ def mpgemmfi_gemm_addend(dtype, M, N, K, A, Bt, C_in, D, fault_sites, n_faults, 
     """Raw call of D = A x B + C_in (device addresses; C_in may be D itself)."""
     return load_library().mpgemmfi_gemm_addend(dtype, M, N, K, A, Bt, C_in, D, fault_sites, n_faults, detect_mode,
                                                flags_out, stream)
+
+
+def mpgemmfi_gemm_out16(dtype, M, N, K, A, Bt, C_in, out_format, D16, fault_sites, n_faults, detect_mode, flags_out, stream):
+    """Raw call of the GEMM with a 16-bit result (OUT_FP16 / OUT_BF16); C_in is None or the FP32 addend."""
+    return load_library().mpgemmfi_gemm_out16(dtype, M, N, K, A, Bt, C_in, out_format, D16, fault_sites, n_faults,
+                                              detect_mode, flags_out, stream)
 
 
 def mpgemmfi_campaign(dtype, M, N, K, A, Bt, C_clean, sites, n_trials, detect_mode, records, workspace,
@@ -268,10 +278,12 @@ def _sites_tensor(sites, device):
     return (sites, sites.shape[0]) if sites.shape[0] else (None, 0)
 
 
-def gemm(dtype, A, Bt, sites=None, detect_mode=DETECT_NONE, C_out=None, flags_out=None, stream=None, addend=None):
+def gemm(dtype, A, Bt, sites=None, detect_mode=DETECT_NONE, C_out=None, flags_out=None, stream=None, addend=None,
+         out_format=OUT_FP32):
     """Fault-injected GEMM on CUDA tensors. Returns (C, flags) where flags is the raw uint32 buffer
     (as an int32 tensor) laid out as documented in include/mpgemmfi.h; see split_flags().
-    addend: optional M x N float32 CUDA tensor, the C_in of D = A x B + C_in (it may be C_out itself)."""
+    addend: optional M x N float32 CUDA tensor, the C_in of D = A x B + C_in (it may be C_out itself).
+    out_format: OUT_FP16 / OUT_BF16 give an M x N float16 / bfloat16 result (mpgemmfi_gemm_out16)."""
     torch = _torch()
     _check_operand(A, dtype, "A")
     _check_operand(Bt, dtype, "Bt")
@@ -280,11 +292,23 @@ def gemm(dtype, A, Bt, sites=None, detect_mode=DETECT_NONE, C_out=None, flags_ou
     if K != K2:
         raise ValueError("A and Bt disagree on K")
     st, n_faults = _sites_tensor(sites, A.device)
+    out_dtype = {OUT_FP32: torch.float32, OUT_FP16: torch.float16, OUT_BF16: torch.bfloat16}[out_format]
     if C_out is None:
-        C_out = torch.empty((M, N), dtype=torch.float32, device=A.device)
+        C_out = torch.empty((M, N), dtype=out_dtype, device=A.device)
     if flags_out is None:
         flags_out = torch.empty(mpgemmfi_flags_bytes(M, N, n_faults) // 4, dtype=torch.int32, device=A.device)
     stream_h = (torch.cuda.current_stream(A.device) if stream is None else stream).cuda_stream
+    if out_format != OUT_FP32:
+        if detect_mode & OUTPUT_RANGE:
+            raise ValueError("the output-level range check writes FP32 only")
+        if C_out.dtype != out_dtype or tuple(C_out.shape) != (M, N) or not C_out.is_contiguous():
+            raise ValueError("C_out must be a contiguous M x N tensor of the output format")
+        rc = mpgemmfi_gemm_out16(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), None if addend is None else addend.data_ptr(),
+                                 out_format, C_out.data_ptr(), st.data_ptr() if st is not None else None, n_faults,
+                                 detect_mode, flags_out.data_ptr(), stream_h)
+        if rc != 0:
+            raise MpgemmfiError(rc, "mpgemmfi_gemm_out16")
+        return C_out, flags_out
     if detect_mode & OUTPUT_RANGE:
         if addend is not None:
             raise ValueError("the output-level range check takes no addend")

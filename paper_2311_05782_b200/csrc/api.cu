@@ -101,6 +101,23 @@ int encode_output_map(CUtensorMap *map, float *C, int M, int N)
     return MPGEMMFI_OK;
 }
 
+// the same for a 16-bit output (FP16 or BF16 words): box = 32 columns (64 bytes) x 32 rows, 64-byte swizzle: one
+// whole 32 x 32 piece of an epilogue warp per store
+int encode_output_map16(CUtensorMap *map, void *D, int out_fmt, int M, int N)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return cuda_fail(cudaErrorUnknown);
+    const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)N * 2u};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapDataType dt = out_fmt == MPGEMMFI_OUT_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const CUresult r = fn(map, dt, 2, D, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return MPGEMMFI_ERR_CUDA; }
+    return MPGEMMFI_OK;
+}
+
 int g_tile_policy = MPGEMMFI_TILES_AUTO;
 int g_split_policy = MPGEMMFI_SPLIT_AUTO;
 int g_wait_limit_ms = 4000;
@@ -112,7 +129,8 @@ int g_break_handover = 0;
 void choose_split(mpg::GemmParams &p, int walkers)
 {
     p.split_parts = 0; p.full_rounds = 0; p.left_tiles = 0;
-    if (g_split_policy == MPGEMMFI_SPLIT_OFF || !p.c_vec_ok) return;
+    // (a cut tile's unfinished FP32 sums wait in C: not with a 16-bit C)
+    if (g_split_policy == MPGEMMFI_SPLIT_OFF || !p.c_vec_ok || p.out_fmt != MPGEMMFI_OUT_FP32) return;
     const int rounds = p.num_tiles / walkers, left = p.num_tiles % walkers;
     if (rounds < 1 || left == 0 || left * 16 > mpg::SPLIT_SIGNAL_WORDS) return;
     int parts = walkers / left;
@@ -163,9 +181,10 @@ int check_common(int dtype, int M, int N, int K, const void *A, const void *Bt, 
     return MPGEMMFI_OK;
 }
 
-int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, float *C, const mpgemmfi_site *sites,
+int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, void *C, const mpgemmfi_site *sites,
              int n_faults, int detect_mode, uint32_t *flags, cudaStream_t stream, const DeviceInfo &di,
-             const uint32_t *exp_a = nullptr, const uint32_t *exp_bt = nullptr, const float *addend = nullptr)
+             const uint32_t *exp_a = nullptr, const uint32_t *exp_bt = nullptr, const float *addend = nullptr,
+             int out_fmt = MPGEMMFI_OUT_FP32)
 {
     int max_pairs = 0;
     const bool pair = choose_pair(dtype, M, N, &max_pairs);
@@ -188,14 +207,17 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, floa
     const int ks = mpg::kstep_of(dtype);
     p.num_kt = (K + ks - 1) / ks;
     p.wpr = (N + 31) / 32;
-    p.c_vec_ok = (N % 4 == 0) && (((uintptr_t)C & 15) == 0);
+    p.out_fmt = out_fmt;
+    const int out_es = out_fmt == MPGEMMFI_OUT_FP32 ? 4 : 2;
+    p.c_vec_ok = (((size_t)N * out_es) % 16 == 0) && (((uintptr_t)C & 15) == 0);
     CUtensorMap tm_c;
     memset(&tm_c, 0, sizeof(tm_c));
     if (p.c_vec_ok) {
-        rc = encode_output_map(&tm_c, C, M, N);
+        rc = out_fmt == MPGEMMFI_OUT_FP32 ? encode_output_map(&tm_c, static_cast<float *>(C), M, N)
+                                          : encode_output_map16(&tm_c, C, out_fmt, M, N);
         if (rc) return rc;
     }
-    p.A = A; p.Bt = Bt; p.C = C; p.sites = sites; p.flags = flags;
+    p.A = A; p.Bt = Bt; p.C = static_cast<float *>(C); p.sites = sites; p.flags = flags;
     p.exp_a = exp_a; p.exp_b = exp_bt;
     p.addend = addend;
     p.addend_vec_ok = (N % 4 == 0) && (((uintptr_t)addend & 15) == 0);
@@ -288,6 +310,34 @@ int mpgemmfi_gemm_addend(int dtype, int M, int N, int K, const void *A, const vo
     if (di.major != 10) return MPGEMMFI_ERR_ARCH;
     return run_gemm(dtype, M, N, K, A, Bt, D, fault_sites, n_faults, detect_mode, flags_out,
                     static_cast<cudaStream_t>(stream), di, nullptr, nullptr, C_in);
+}
+
+int mpgemmfi_gemm_out16(int dtype, int M, int N, int K, const void *A, const void *Bt, const float *C_in, int out_format,
+                        void *D16, const mpgemmfi_site *fault_sites, int n_faults, int detect_mode, uint32_t *flags_out,
+                        mpgemmfi_stream stream)
+{
+    if (out_format != MPGEMMFI_OUT_FP16 && out_format != MPGEMMFI_OUT_BF16) return MPGEMMFI_ERR_DTYPE;
+    if (dtype != MPGEMMFI_FP16 && dtype != MPGEMMFI_BF16 && dtype != MPGEMMFI_TF32) return MPGEMMFI_ERR_DTYPE;
+    if (M <= 0 || N <= 0 || K <= 0 || !A || !Bt || !D16) return MPGEMMFI_ERR_ARG;
+    if ((unsigned long long)M * (unsigned long long)N >= 0xFFFFFFFFull) return MPGEMMFI_ERR_ARG;
+    if (((uintptr_t)A & 15) || ((uintptr_t)Bt & 15) || ((uintptr_t)D16 & 1) || ((uintptr_t)C_in & 3) ||
+        ((size_t)K * mpg::esize_of(dtype)) % 16)
+        return MPGEMMFI_ERR_ALIGN;
+    if (C_in) {
+        // the addend is read tile by tile while other tiles' results are written: the two must not share memory
+        const uintptr_t c0 = (uintptr_t)C_in, d0 = (uintptr_t)D16;
+        if (c0 < d0 + (size_t)M * N * 2 && d0 < c0 + (size_t)M * N * 4) return MPGEMMFI_ERR_ARG;
+    }
+    if (n_faults < 0 || n_faults > MPGEMMFI_MAX_FAULTS || (n_faults > 0 && !fault_sites)) return MPGEMMFI_ERR_ARG;
+    if (detect_mode & ~(MPGEMMFI_DETECT_TECHNIQUE_MASK | MPGEMMFI_CORRECT)) return MPGEMMFI_ERR_ARG;
+    if (!flags_out && (n_faults > 0 || (detect_mode & MPGEMMFI_DETECT_TECHNIQUE_MASK))) return MPGEMMFI_ERR_ARG;
+    if (((uintptr_t)fault_sites & 15) || ((uintptr_t)flags_out & 15)) return MPGEMMFI_ERR_ALIGN;
+    DeviceInfo di;
+    const int rc = device_info(di);
+    if (rc) return rc;
+    if (di.major != 10) return MPGEMMFI_ERR_ARCH;
+    return run_gemm(dtype, M, N, K, A, Bt, D16, fault_sites, n_faults, detect_mode, flags_out,
+                    static_cast<cudaStream_t>(stream), di, nullptr, nullptr, C_in, out_format);
 }
 
 int mpgemmfi_operand_exponents(int dtype, int rows, int K, const void *X, uint32_t *out, mpgemmfi_stream stream)

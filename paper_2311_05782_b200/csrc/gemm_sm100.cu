@@ -34,6 +34,8 @@
 #include <cstdint>
 #include <type_traits>
 #include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include "checks.cuh"
@@ -580,6 +582,18 @@ __device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid,
     }
 }
 
+// two FP32 words -> one word holding their roundings (to nearest, ties to even) to the 16-bit output format,
+// the first in the low half
+__device__ __forceinline__ uint32_t pack_out16(int out_fmt, uint32_t lo_bits, uint32_t hi_bits)
+{
+    if (out_fmt == MPGEMMFI_OUT_FP16) {
+        const __half2 h = __floats2half2_rn(bits_f32(lo_bits), bits_f32(hi_bits));
+        return *reinterpret_cast<const uint32_t *>(&h);
+    }
+    const __nv_bfloat162 b = __floats2bfloat162_rn(bits_f32(lo_bits), bits_f32(hi_bits));
+    return *reinterpret_cast<const uint32_t *>(&b);
+}
+
 // kPair = false: grid of single CTAs, tiles 128 x BN.
 // kPair = true : grid of CTA pairs (cluster dimension 2), tiles 256 x BN, BN = 256.
 template <int BN, bool kTF32, bool kPair>
@@ -868,6 +882,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         // where this thread parks 16-byte chunk j of its row for a TMA store: park_addr ^ (j << 4) (128-byte swizzle:
         // chunk j of row r sits at chunk position j ^ (r & 7))
         const uint32_t park_addr = smem_u32(my_out) + ((uint32_t)lane & 15u) * 128u + (((uint32_t)lane & 7u) << 4);
+        // the same for a 16-bit output: rows of 64 bytes, 64-byte swizzle (chunk c of row r at position c ^ ((r >> 1) & 3))
+        const uint32_t park16_addr = smem_u32(my_out) + (uint32_t)lane * 64u + ((((uint32_t)lane >> 1) & 3u) << 4);
         constexpr int MY_PIECES = BN / 64;          // 32-column pieces per warp (half the tile's columns)
         const int first = h * MY_PIECES;
         // hand-over words of this warp for left-over tile j: signals[j * 16 + my_signal]
@@ -1000,6 +1016,31 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     }
                 }
             };
+            // 16-bit output: the checked FP32 values are rounded once (to nearest even) and the whole 32 x 32 piece, now
+            // 64 bytes a row, fits the staging: all 32 threads park their rows at once and the piece leaves as ONE store.
+            auto store_piece16 = [&](uint32_t (&v)[32], uint32_t c0) {
+                uint32_t h[16];
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) h[jj] = pack_out16(p.out_fmt, v[2 * jj], v[2 * jj + 1]);
+                if (p.c_vec_ok) {
+                    if (lane == 0) bulk_wait_read_all();
+                    __syncwarp();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        st_shared_v4(park16_addr ^ (uint32_t)(c << 4), h[4 * c], h[4 * c + 1], h[4 * c + 2], h[4 * c + 3]);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && row0 < (uint32_t)p.M && c0 < (uint32_t)p.N) {
+                        tma_store_2d(&tm_c, smem_u32(my_out), (int)c0, (int)row0);
+                        bulk_commit_group();
+                    }
+                } else if (row_ok) {
+                    unsigned short *drow = reinterpret_cast<unsigned short *>(p.C) + (size_t)row * p.N;
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj)
+                        if (c0 + jj < (uint32_t)p.N) drow[c0 + jj] = (unsigned short)(h[jj >> 1] >> (16 * (jj & 1)));
+                }
+            };
             // accumulator columns of this warp fully read: one arrival towards handing the TMEM
             // buffer back to the MMA warp
             auto release_acc = [&]() {
@@ -1081,7 +1122,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                         if (c0 + 32 > (uint32_t)p.N) fw &= c0 < (uint32_t)p.N ? (1u << ((uint32_t)p.N - c0)) - 1u : 0u;
                     }
                     if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 1);
-                    if (p.c_vec_ok) store_piece_tma(v, c0);
+                    if (p.out_fmt != MPGEMMFI_OUT_FP32) store_piece16(v, c0);
+                    else if (p.c_vec_ok) store_piece_tma(v, c0);
                     else store_piece(v, c0);
                     return fw;
                 };

@@ -16,6 +16,7 @@ struct GemmParams {
     int group_m;    // tile rows per band of the tile order (>= 1)
     int wpr;        // bitmap words per row = ceil(N / 32)
     int c_vec_ok;   // C is 16-byte aligned with a 16-byte row pitch: the epilogue may use 16-byte stores
+    int out_fmt;    // MPGEMMFI_OUT_FP32, or a 16-bit format: C then points to M x N 2-byte words
     const void *A;
     const void *Bt;
     float *C;
@@ -72,8 +73,9 @@ inline uint32_t gemm_epoch_of(uint32_t counter) { return (counter & 0x1FFFFFFFu)
 // Pair mode (pair = true): 256 x 256 tiles walked by CTA pairs; tm_b box is (128 bytes x 128 rows);
 // `grid` is even (two CTAs per pair); p.tiles_m counts 256-row tiles.
 // tm_a always has a box of (128 bytes x 128 rows). Both maps use the 128-byte swizzle.
-// tm_c covers C (FP32, box 32 columns x 16 rows, 128-byte swizzle) and is used for the stores of finished
-// tiles when p.c_vec_ok is set; otherwise its contents do not matter.
+// tm_c covers C and is used for the stores of finished tiles when p.c_vec_ok is set (otherwise its contents do
+// not matter): FP32 output: box 32 columns x 16 rows, 128-byte swizzle; 16-bit output: box 32 columns x 32 rows,
+// 64-byte swizzle.
 cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c,
                         const GemmParams &p, int grid, cudaStream_t stream);
 
