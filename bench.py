@@ -53,8 +53,9 @@ WORKLOAD_TEXT = {
           "detection+correction",
 }
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMM kernel, from the ncu capture summarised
-# under profiles/; None once the kernel has changed since the counters were taken
-KERNEL_TRAFFIC_BYTES = {"c2": 152.6e6}
+# under profiles/ (the capture names the kernel source it was taken on); None for a config without a capture of the
+# present kernel
+KERNEL_TRAFFIC_BYTES = {}
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 
 
@@ -151,6 +152,82 @@ def cpu_baseline(w, budget_s=12.0):
                       f"trial table, the config's check, {t:.2f} s"}
 
 
+def quick_config(name, mpg, synth, torch, dev, flush, peaks, steps=40, out16=False):
+    """One config in brief, for the `all_configs` key: us per injected GEMM (L2 flushed, per-step events), its rate and
+    roofline fraction, the time ratio against the same kernel without injection and check (alternating launches), and
+    the campaign's trials/s. out16: the GEMM writes an FP16 result (mpgemmfi_gemm_out16) instead of FP32."""
+    w = synth.make_workload(name)
+    M, N, K, dtype, mode = w.M, w.N, w.K, w.dtype, w.detect_mode
+    view = np.int32 if dtype == synth.DTYPE_TF32 else np.int16
+    A = torch.from_numpy(w.A.view(view)).to(dev)
+    Bt = torch.from_numpy(w.Bt.view(view)).to(dev)
+    sites = torch.from_numpy(w.sites.view(np.int32).reshape(-1, 8)).to(dev)
+    C = torch.empty((M, N), dtype=torch.float16 if out16 else torch.float32, device=dev)
+    flags = torch.empty(mpg.mpgemmfi_flags_bytes(M, N, 1) // 4, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    sh = stream.cuda_stream
+    n = len(w.sites)
+
+    def step(i, inject):
+        sp, nf, md, fl = (sites.data_ptr() + 32 * (i % n), 1, mode, flags.data_ptr()) if inject else (None, 0, 0, None)
+        if out16:
+            rc = mpg.mpgemmfi_gemm_out16(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), None, mpg.OUT_FP16, C.data_ptr(), sp, nf,
+                                         md, fl, sh)
+        else:
+            rc = mpg.mpgemmfi_gemm(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), C.data_ptr(), sp, nf, md, fl, sh)
+        if rc != 0:
+            raise mpg.MpgemmfiError(rc, "mpgemmfi_gemm")
+
+    for i in range(3):
+        for inject in (True, False):
+            flush.zero_(); step(i, inject)
+    torch.cuda.synchronize(dev)
+    ev = []
+    for i in range(steps):
+        for inject in (True, False):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream); step(i, inject); e1.record(stream)
+            ev.append((inject, e0, e1))
+    torch.cuda.synchronize(dev)
+    t_on = statistics.median(e0.elapsed_time(e1) for inj, e0, e1 in ev if inj) * 1e-3
+    t_off = statistics.median(e0.elapsed_time(e1) for inj, e0, e1 in ev if not inj) * 1e-3
+    if int(flags[0].item()) & mpg.STATUS_WAIT_LIMIT:
+        raise SystemExit(f"device wait limit hit on {name}")
+    flops = 2.0 * M * N * K
+    out = {"us_per_gemm": t_on * 1e6, "tflops": flops / t_on / 1e12, "injected_over_plain_time": t_on / t_off,
+           "dtype": DTYPE_NAMES[dtype], "output": "fp16" if out16 else "fp32", "steps": steps}
+    es = A.element_size()
+    min_bytes = (M * K + N * K) * es + M * N * C.element_size() + M * ((N + 31) // 32) * 4
+    if name == "c1":
+        out.update({"bound": "latency", "frac": None})          # one wave of four tiles: launch and pipeline fill
+    elif name == "c5":
+        gbs = min_bytes / t_on / 1e9
+        out.update({"bound": "hbm", "achieved_gbs": gbs, "frac": gbs / peaks["hbm_gbs"]})
+    else:
+        peak = peaks["bf16_tflops"] * (0.5 if dtype == synth.DTYPE_TF32 else 1.0)
+        out.update({"bound": "tensor", "frac": out["tflops"] / peak})
+    if not out16:
+        rec = torch.empty((n, 12), dtype=torch.int32, device=dev)
+        Cc = C
+        ws = torch.empty(mpg.mpgemmfi_campaign_workspace_bytes(dtype, M, N, K, n), dtype=torch.uint8, device=dev)
+        ts = []
+        for i in range(5):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            rc = mpg.mpgemmfi_campaign(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), Cc.data_ptr(), sites.data_ptr(), n, mode,
+                                       rec.data_ptr(), ws.data_ptr(), ws.numel(), sh)
+            e1.record(stream)
+            if rc != 0:
+                raise mpg.MpgemmfiError(rc, "mpgemmfi_campaign")
+            ts.append((e0, e1))
+        torch.cuda.synchronize(dev)
+        t_c = statistics.median(e0.elapsed_time(e1) for e0, e1 in ts[2:]) * 1e-3
+        out.update({"campaign_trials": n, "campaign_ms": t_c * 1e3, "campaign_trials_per_s": n / t_c})
+    return out
+
+
 def run_reference(args):
     """The CPU oracle as the reference arm: each step is a bounded row-panel sample of the workload."""
     import oracle as orc
@@ -190,6 +267,7 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiling runs)")
     ap.add_argument("--config", default=WORKLOAD, help="workload to time (c1, c2, c3a, c3b, c4, c5); default c2")
+    ap.add_argument("--no-all-configs", action="store_true", help="skip the brief pass over the other workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
@@ -202,7 +280,7 @@ def main():
 
     import paper_2311_05782_b200 as mpg
     import synth
-    from paper_2311_05782_b200.sharding import shard_range, reduce_max, reduce_sum
+    from paper_2311_05782_b200.sharding import campaign_sharded, shard_range, reduce_max, reduce_sum
 
     world = env_int("WORLD_SIZE", 1)
     rank = env_int("RANK", 0)
@@ -333,6 +411,27 @@ def main():
     trials_total = reduce_sum(float(n_my * camp_steps), world, dev)
     trials_per_s = trials_total / (ms_camp_max * 1e-3)
 
+    # ---- N > 1: the whole table through the library's sharded campaign (every rank its share, then ONE all_gather of
+    # the 48-byte records): time of the gather included, on the device, max over ranks
+    sharded = None
+    if world > 1:
+        def local_campaign(dt_, A_, Bt_, share, mode_):
+            campaign_step(0)
+            return C, rec
+
+        for _ in range(2):
+            campaign_sharded(dtype, A, Bt, w.sites, mode, run_local=local_campaign)
+        torch.cuda.synchronize(dev)
+        dist.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        _, allrec = campaign_sharded(dtype, A, Bt, w.sites, mode, run_local=local_campaign)
+        e1.record(stream)
+        torch.cuda.synchronize(dev)
+        ms_sh = reduce_max(e0.elapsed_time(e1), world, dev)
+        sharded = {"trials": len(w.sites), "ms": ms_sh, "trials_per_s": len(w.sites) / (ms_sh * 1e-3),
+                   "gathered_record_bytes": int(allrec.numel() * 4), "collective": "one all_gather (nccl)"}
+
     # ---- end to end: pinned host buffers, copies inside the timed region
     hA = torch.from_numpy(w.A.view(view)).pin_memory()
     hB = torch.from_numpy(w.Bt.view(view)).pin_memory()
@@ -405,6 +504,16 @@ def main():
             finally:
                 torch.backends.cuda.matmul.allow_tf32 = old
 
+    all_configs = None
+    if world == 1 and not args.no_all_configs:
+        # the other workloads in brief (same timing rules, fewer steps), so that one run shows all of them
+        del hA, hB, hC, hF
+        all_configs = {}
+        for name, o16 in (("c1", False), ("c2", False), ("c3a", False), ("c3a", True), ("c3b", False), ("c4", False), ("c5", False)):
+            key = name + ("_fp16_output" if o16 else "")
+            all_configs[key] = quick_config(name, mpg, synth, torch, dev, flush, peaks, steps=12 if name == "c4" else 40, out16=o16)
+            torch.cuda.empty_cache()
+
     if rank == 0:
         baseline = None
         if world == 1 and not args.no_cpu_baseline:
@@ -428,8 +537,9 @@ def main():
                               "injected_over_plain_time": on_over_off_time,
                               "how": "launches with and without injection alternate in one loop"},
             "campaign": {"trials_per_s": trials_per_s, "trials_per_launch": n_my, "launches": camp_steps,
-                         "ms_per_launch": ms_camp_max / camp_steps},
+                         "ms_per_launch": ms_camp_max / camp_steps, "sharded": sharded},
             "cpu_baseline": baseline,
+            "all_configs": all_configs,
         }
         print(json.dumps(line))
     if world > 1:

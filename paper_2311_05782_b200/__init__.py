@@ -22,3 +22,4 @@ from .binding import (  # noqa: F401
     mpgemmfi_set_wait_limit_ms, mpgemmfi_debug_break_handover, mpgemmfi_debug_launch_slot,
     mpgemmfi_gemm_out16, OUT_FP32, OUT_FP16, OUT_BF16,
 )
+from .sharding import campaign_sharded, shard_range  # noqa: F401,E402

@@ -36,12 +36,52 @@ def reduce_sum(value: float, world: int, device="cpu") -> float:
     return _reduce(value, world, device, "SUM")
 
 
-def gather_records(local_records, world: int):
-    """Concatenate per-rank trial records (numpy structured arrays) in rank order on every rank."""
-    if world <= 1:
-        return local_records
-    import numpy as np
+RECORD_BYTES = 48
+
+
+def gather_records(local, counts, group=None):
+    """All ranks' trial records in rank order, on every rank: ONE all_gather of fixed-size byte blocks.
+
+    local: this rank's records as a uint8 tensor [n_local * 48] (or any tensor of that many bytes) on the device the
+    process group communicates on (CUDA for nccl, CPU for gloo); counts: trials per rank (known to every rank from
+    shard_range, so no size exchange is needed). Every rank contributes a block padded to the largest share; the
+    padding is cut out after the gather. Returns a uint8 tensor [sum(counts) * 48]."""
+    import torch
     import torch.distributed as dist
-    parts = [None] * world
-    dist.all_gather_object(parts, local_records)
-    return np.concatenate(parts)
+    world = len(counts)
+    flat = local.reshape(-1).view(torch.uint8)
+    if world <= 1:
+        return flat
+    block = max(counts) * RECORD_BYTES
+    send = torch.zeros(block, dtype=torch.uint8, device=flat.device)
+    send[:flat.numel()] = flat
+    recv = torch.empty(world * block, dtype=torch.uint8, device=flat.device)
+    dist.all_gather_into_tensor(recv, send, group=group)
+    if all(c == counts[0] for c in counts):
+        return recv
+    return torch.cat([recv[r * block:r * block + counts[r] * RECORD_BYTES] for r in range(world)])
+
+
+def campaign_sharded(dtype, A, Bt, sites, detect_mode, group=None, run_local=None):
+    """A campaign whose trial table is shared out over the ranks of a process group (one process per GPU).
+
+    Every rank holds the whole operands and the whole table (a numpy structured array of 32-byte sites), runs the clean
+    GEMM and ITS contiguous share of the trials through mpgemmfi_campaign, and receives every rank's records through
+    one all_gather. There is no other exchange: trials are independent. Returns (C_clean, records) with records an
+    int32 tensor [n_trials, 12] in table order, identical on every rank.
+
+    run_local(dtype, A, Bt, sites_share, detect_mode) -> (C_clean, records int32 [n, 12]) stands in for the library
+    call in tests that have no GPU; the default is the library's campaign()."""
+    import torch
+    import torch.distributed as dist
+    if run_local is None:
+        from .binding import campaign as run_local
+    world = dist.get_world_size(group) if dist.is_available() and dist.is_initialized() else 1
+    rank = dist.get_rank(group) if world > 1 else 0
+    n = 0 if sites is None else len(sites)
+    spans = [shard_range(n, r, world) for r in range(world)]
+    lo, hi = spans[rank]
+    C_clean, rec = run_local(dtype, A, Bt, sites[lo:hi] if n else None, detect_mode)
+    rec = rec.reshape(-1, 12)[:hi - lo].contiguous()
+    allrec = gather_records(rec, [b - a for a, b in spans], group)
+    return C_clean, allrec.view(torch.int32).reshape(n, 12)
