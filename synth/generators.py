@@ -122,9 +122,12 @@ def config_seed(name: str) -> int:
     return BASE_SEED + 1000 * cfg["index"] + cfg.get("seed_shift", 0)
 
 
-def make_operands(name: str, M=None, N=None, K=None, seed=None):
-    """Return (A_bits[M,K], Bt_bits[N,K]) for a config, optionally at reduced sizes."""
+def make_operands(name: str, M=None, N=None, K=None, seed=None, dtype=None):
+    """Return (A_bits[M,K], Bt_bits[N,K]) for a config, optionally at reduced sizes and, with `dtype`, with the same
+    draws rounded to another storage format."""
     cfg = CONFIGS[name]
+    if dtype is not None:
+        cfg = dict(cfg, dtype=dtype)
     M = cfg["M"] if M is None else M
     N = cfg["N"] if N is None else N
     K = cfg["K"] if K is None else K

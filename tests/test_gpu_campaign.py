@@ -270,3 +270,35 @@ def test_operand_trials_are_eq1_eq2_on_the_clean_sum_bit_for_bit(dtype, shape, n
             if det.any():
                 assert g["first_detected"] == lin[det].min()
                 assert int(g["idx_hash"]) == sum((int(l) + 1) * HASH_MUL for l in lin[det]) & ((1 << 64) - 1)
+
+
+@pytest.mark.parametrize("workload,fmt,nbits,mode", [("relu_k576", orc.FP16, 1, 0), ("relu_k576", orc.BF16, 4, orc.T_BOUND | orc.CORRECT),
+                                                     ("gelu_k4096", orc.TF32, 2, orc.T_RMAX | orc.CORRECT),
+                                                     ("gelu_k4096", orc.FP16, 4, orc.T_RFLIP | orc.CORRECT)])
+def test_deviation_study_cell_against_the_oracle(workload, fmt, nbits, mode):
+    """A cell of the deviation study (term trials at HMMA granularity, reduced on the device) against the oracle's
+    campaign and summary on the same operands and trial table: the whole summary, word for word."""
+    from paper_2311_05782_b200 import deviation_study as ds
+    trials = 600
+    summ, cell = ds.run_cell(mpg, synth, torch, workload, fmt, nbits, mode, trials)
+    cfg, M, N, K = ds.WORKLOADS[workload]
+    A, Bt = synth.make_operands(cfg, M, N, K, dtype=fmt)
+    sites = synth.make_sites("term", fmt, M, N, K, trials, synth.config_seed(cfg) + 100 * nbits + 1, nbits=nbits)
+    # the oracle needs only the rows of A and Bt that the trials touch: one 1 x 1 problem per trial
+    rec = np.zeros(trials, dtype=orc.RECORD)
+    for t, s in enumerate(sites):
+        i, j = int(s["row"]), int(s["col"])
+        one = s.copy().reshape(1); one["row"] = 0; one["col"] = 0
+        Cs, *_ = orc.gemm(fmt, A[i:i + 1], Bt[j:j + 1])
+        rec[t] = orc.campaign(fmt, A[i:i + 1], Bt[j:j + 1], Cs, one, mode, kstep=8 if fmt == orc.TF32 else 16)[0]
+    want = orc.summary(rec)
+    raw = np.zeros(trials, dtype=orc.RECORD)
+    got = np.concatenate([[summ["n_trials"], summ["n_invalid"], summ["n_zero_diff"], summ["n_detected"], summ["n_corrected"],
+                           summ["n_nonfinite"]], summ["kind_trials"], summ["kind_zero_diff"], summ["dev_exponent_hist"]]).astype(np.uint32)
+    # a NaN that a fault creates keeps an unspecified payload through the later additions; what a correction makes of it
+    # is then not unique: such trials can sit in different bins on the two sides, all others must agree
+    nan_made = sum(1 for r in rec if np.isnan(np.uint32(r["final_bits"]).view(np.float32)) or np.isinf(r["max_abs_dev"]))
+    diff = np.abs(got.astype(np.int64) - want.astype(np.int64))
+    assert diff[:5].sum() == 0 and diff[6:16].sum() == 0, (got[:16], want[:16])
+    assert diff[16:].sum() <= 2 * nan_made and diff[5] <= nan_made
+    assert cell["trials"] == trials and abs(cell["zero_diff_pct"] - 100.0 * want[2] / trials) < 1e-9
