@@ -22,6 +22,7 @@ KIND_A, KIND_B, KIND_ACC, KIND_OUT, KIND_TERM = 0, 1, 2, 3, 4
 T_NONE, T_BOUND, T_RMAX, T_RFLIP = 0, 1, 2, 3
 CORRECT = 16
 OUTPUT_RANGE = 64
+TERM_IN_FORMAT = 128
 
 SITE = np.dtype([("kind", "<u4"), ("row", "<u4"), ("col", "<u4"), ("k", "<u4"),
                  ("xor_mask", "<u4"), ("trial", "<u4"), ("pad0", "<u4"), ("pad1", "<u4")])
@@ -79,6 +80,8 @@ def lib():
         L.orc_campaign_form.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp]
         L.orc_operand_trial_values.restype = C.c_int
         L.orc_operand_trial_values.argtypes = [C.c_int] * 4 + [vp, vp, vp, vp, C.c_int, vp]
+        L.orc_round_to_operand.restype = C.c_uint32
+        L.orc_round_to_operand.argtypes = [C.c_int, C.c_uint32]
         L.orc_round_output.restype = C.c_uint32
         L.orc_round_output.argtypes = [C.c_int, C.c_uint32]
         L.orc_gemm_out16.restype = C.c_int
@@ -223,6 +226,11 @@ def operand_trial_values(dtype, A, Bt, C_clean, site, form=0):
 
 
 OUT_FP16, OUT_BF16 = 0, 1
+
+
+def round_to_operand(dtype, bits):
+    """FP32 word -> storage word of the operand format (round to nearest even)."""
+    return int(lib().orc_round_to_operand(dtype, int(bits) & 0xFFFFFFFF))
 
 
 def round_output(out_fmt, bits):

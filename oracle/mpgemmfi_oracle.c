@@ -179,6 +179,26 @@ static uint32_t product_check(int detect_mode, uint32_t p_err, uint32_t a_bits, 
 
 /* ------------------------------------------------------------------ one output element */
 
+uint32_t orc_round_output(int out_fmt, uint32_t bits);      /* defined with the 16-bit output further down */
+
+/*
+ * An FP32 word rounded to the operand format `dtype`, to nearest with ties to even, as that format's storage word
+ * (16 bits for FP16 and BF16; for TF32 the FP32 word with its low 13 bits zero). Used by the alternative reading of
+ * the paper's fault in which the product lives in the operand format when its bits are flipped.
+ */
+uint32_t orc_round_to_operand(int dtype, uint32_t bits)
+{
+    if (dtype == ORC_FP16) return orc_round_output(0, bits);
+    if (dtype == ORC_BF16) return orc_round_output(1, bits);
+    uint32_t E = (bits >> 23) & 0xFFu;
+    if (E == 0xFFu) return (bits & 0xFFFFE000u) | ((bits & 0x7FFFFFu) ? 0x00400000u : 0u);   /* Inf stays, NaN stays NaN */
+    uint32_t keep = bits >> 13, rest = bits & 0x1FFFu;
+    if (rest > 0x1000u || (rest == 0x1000u && (keep & 1u))) keep += 1u;     /* may carry into the exponent, up to Inf */
+    return keep << 13;
+}
+
+#define ORC_TERM_IN_FORMAT 128
+
 static inline uint32_t term_boundary(uint32_t k, int kstep, int K)
 {
     uint32_t kb = (k / (uint32_t)kstep + 1u) * (uint32_t)kstep;
@@ -192,7 +212,7 @@ static inline uint32_t term_boundary(uint32_t k, int kstep, int K)
  * idx[n_idx]: indices into sites[] of this element's ACC/TERM sites, ascending.
  * acc0: what the running sum starts from (+0, or the addend c_ij of D = A x B + C, Section II-B).
  */
-static float element_with_sites(const float *a, const float *b, int K, int kstep, int detect_mode,
+static float element_with_sites(int dtype, const float *a, const float *b, int K, int kstep, int detect_mode,
                                 const orc_site *sites, const int *idx, int n_idx, orc_site_log *log, float acc0)
 {
     float acc = acc0;
@@ -213,8 +233,19 @@ static float element_with_sites(const float *a, const float *b, int K, int kstep
                 float re2 = a[s->k] * b[s->k];
                 uint32_t before = f2u(re2);
                 uint32_t after = before ^ s->xor_mask;
+                uint32_t p_err = after;
+                if (detect_mode & ORC_TERM_IN_FORMAT) {
+                    /* alternative reading: the multiplication's result is held in the operand format (the paper's own
+                     * example of a flipped zero is a 16-bit pattern, Section V-B). re_2 is the product rounded to that
+                     * format, the mask addresses that format's storage bits like an operand site's, and Eq. 1-2 are
+                     * applied with this re_2 and its flipped version widened back to FP32. */
+                    before = orc_round_to_operand(dtype, f2u(re2));
+                    after = orc_flip_operand(dtype, before, s->xor_mask);
+                    re2 = orc_widen(dtype, before);
+                    p_err = orc_widen_bits(dtype, after);
+                }
                 int det;
-                uint32_t fin = product_check(detect_mode, after, f2u(a[s->k]), f2u(b[s->k]), &det);
+                uint32_t fin = product_check(detect_mode, p_err, f2u(a[s->k]), f2u(b[s->k]), &det);
                 float rep = acc - re2;          /* Eq. 1 */
                 acc = rep + u2f(fin);           /* Eq. 2 */
                 if (log) { log[idx[t]].before_bits = before; log[idx[t]].after_bits = after;
@@ -415,7 +446,7 @@ static int gemm_impl(int dtype, int M, int N, int K, const void *A, const void *
                 site_valid(e, dtype, M, N, K)) { idx[n_idx++] = q; done[q] = 1; }
         }
         C[(size_t)s->row * N + s->col] =
-            element_with_sites(&Af[(size_t)s->row * K], &Bf[(size_t)s->col * K], K, kstep, detect_mode,
+            element_with_sites(dtype, &Af[(size_t)s->row * K], &Bf[(size_t)s->col * K], K, kstep, detect_mode,
                                sites, idx, n_idx, log,
                                addend ? addend[(size_t)s->row * N + s->col] : 0.0f);
     }
@@ -484,7 +515,7 @@ int orc_gemm_addend(int dtype, int M, int N, int K, const void *A, const void *B
 
 /* ------------------------------------------------------------------ 16-bit output */
 
-enum { ORC_OUT_FP16 = 0, ORC_OUT_BF16 = 1 };
+enum { ORC_OUT_FP16 = 0, ORC_OUT_BF16 = 1 };      /* (orc_round_to_operand above relies on these two values) */
 
 /*
  * Round an FP32 word to the nearest value of a 16-bit format, ties to even (the models of
@@ -652,7 +683,7 @@ int orc_campaign_form(int dtype, int M, int N, int K, const void *A, const void 
             uint32_t lin = s->row * (uint32_t)N + s->col;
             orc_site_log lg; int idx0 = 0;
             orc_site one = *s;
-            float v = element_with_sites(&Af[(size_t)s->row * K], &Bf[(size_t)s->col * K], K, kstep,
+            float v = element_with_sites(dtype, &Af[(size_t)s->row * K], &Bf[(size_t)s->col * K], K, kstep,
                                          detect_mode, &one, &idx0, 1, &lg, 0.0f);
             r->primary_index = lin; r->before_bits = lg.before_bits; r->after_bits = lg.after_bits;
             trial_account(&ta, detect_mode, v, C_clean[lin], lin, &r->final_bits);

@@ -151,6 +151,8 @@ def make_sites(mix: str, dtype: int, M: int, N: int, K: int, n: int, seed: int,
          "acc"     one accumulator element after a uniformly chosen k boundary
          "acc2"    as "acc" with two adjacent bits
          "term"    one product term (i, j, k), bit(s) uniform in the 32-bit product
+         "term_op" the same with the bit(s) uniform in a word of the operand format (16 bits; 19 for TF32), for the
+                   reading in which the product is held in that format
          "mixed"   kind uniform over {operand, acc, out}
     """
     rng = _rng(seed)
@@ -176,7 +178,7 @@ def make_sites(mix: str, dtype: int, M: int, N: int, K: int, n: int, seed: int,
         kind = np.where(u_ab == 0, KIND_A, KIND_B)
     elif mix == "acc":
         kind = np.full(n, KIND_ACC)
-    elif mix == "term":
+    elif mix in ("term", "term_op"):
         kind = np.full(n, KIND_TERM)
     elif mix == "mixed":
         kind = np.where(u_kind == 0, np.where(u_ab == 0, KIND_A, KIND_B),
@@ -185,7 +187,7 @@ def make_sites(mix: str, dtype: int, M: int, N: int, K: int, n: int, seed: int,
         raise ValueError(mix)
 
     is_op = (kind == KIND_A) | (kind == KIND_B)
-    width = np.where(is_op, obits, 32)
+    width = np.where(is_op | (mix == "term_op"), obits, 32)
     start = np.floor(u_bit * (width - nbits + 1)).astype(np.uint32)
     s["kind"] = kind
     s["row"] = np.where(kind == KIND_B, 0, row)

@@ -244,7 +244,8 @@ def record_from_full_recompute(Cf, bm, Cclean, lins, detect_mode):
 @pytest.mark.parametrize("name,mix,mode", [
     ("c1", "out", None), ("c2", "operand", None), ("c4", "acc2", None), ("c5", "mixed", None), ("c2", "term", None),
     ("c2", "term", orc.T_BOUND), ("c2", "term", orc.T_RMAX | orc.CORRECT), ("c2", "term", orc.T_RFLIP | orc.CORRECT),
-    ("c5", "mixed", orc.T_NONE)])
+    ("c5", "mixed", orc.T_NONE), ("c2", "term_op", orc.TERM_IN_FORMAT), ("c1", "term_op", orc.T_BOUND | orc.CORRECT | orc.TERM_IN_FORMAT),
+    ("c4", "term_op", orc.T_RMAX | orc.CORRECT | orc.TERM_IN_FORMAT)])
 def test_incremental_trials_equal_full_recompute(name, mix, mode):
     """Every trial record equals what a full fault-injected GEMM with that single site gives: the full recompute is
     the definition. ("c2", "term") runs TERM trials under BoundCheck + correction, where a product-level correction
@@ -257,6 +258,9 @@ def test_incremental_trials_equal_full_recompute(name, mix, mode):
         # single-bit flips of small products rarely reach the thresholds: put some masks on the exponent's top bits
         w.sites["xor_mask"][::3] = 1 << 30
         w.sites["xor_mask"][1::6] = 3 << 29
+    if mix == "term_op":
+        top = 18 if dt == orc.TF32 else 15
+        w.sites["xor_mask"][::3] = 1 << (top - 1)
     Cclean, *_ = orc.gemm(dt, w.A, w.Bt)
     rec = orc.campaign(dt, w.A, w.Bt, Cclean, w.sites, mode)
     seen_status = set()
@@ -587,3 +591,84 @@ def test_operand_writeback_on_rounded_data(dtype):
             i_, j_ = (s["row"], o) if isA else (o, s["col"])
             assert abs(float(v0[o]) - float(v1[o])) <= 2 * K * 2.0 ** -24 * (ap[i_, j_] + float(abs(xf * y)))
     assert order_matters > 0        # the data does tell the two orders apart
+
+
+# ---------------------------------------------------------------- the product held in the operand format (alternative reading)
+
+def test_round_to_operand_format():
+    """TF32: ties to even on the 13 dropped bits, carries into the exponent, against the generators' rounding; FP16 and
+    BF16 are the 16-bit output rounding (pinned in test_oracle_output16.py)."""
+    for w, want in [(0x3F801000, 0x3F800000), (0x3F803000, 0x3F804000), (0x3F801001, 0x3F802000), (0x3F800FFF, 0x3F800000),
+                    (0x3FFFF000, 0x40000000), (0x7F7FF000, 0x7F800000), (0x7F800000, 0x7F800000), (0x80001000, 0x80000000),
+                    (0x00003000, 0x00004000)]:
+        assert orc.round_to_operand(orc.TF32, w) == want, hex(w)
+    assert orc.round_to_operand(orc.TF32, 0x7F800001) & 0x007FE000                     # NaN stays NaN
+    rng = np.random.default_rng(81)
+    w = rng.integers(0, 1 << 32, 100000, dtype=np.uint64).astype(np.uint32)
+    w = w[((w >> 23) & 0xFF) != 0xFF]
+    got = np.array([orc.round_to_operand(orc.TF32, int(x)) for x in w], dtype=np.uint32)
+    assert np.array_equal(got, synth.round_to_storage(w.view(np.float32), orc.TF32))
+    assert orc.round_to_operand(orc.FP16, f32_bits(1.0 + 2.0 ** -11)) == 0x3C00 and orc.round_to_operand(orc.BF16, 0x3F818000) == 0x3F82
+
+
+def test_term_in_operand_format_paper_example_and_closed_forms():
+    """Section V-B's example: a product that is zero, held in FP16, with its first mantissa bit flipped, is
+    0.00003052 (the value the paper prints) and changes the sum; the same flip of a BF16 zero is far too small to
+    survive the accumulation. Then closed forms on exact data."""
+    K = 8
+    a = np.array([[1, 2, 0, 3, 1, 1, 2, 1]], dtype=np.float32); b = np.array([[2, 1, 5, 1, 1, 3, 1, 2]], dtype=np.float32)
+    import os
+    rows = [l.split() for l in open(os.path.join(os.path.dirname(__file__), "golden", "fp16_subnormal_example.txt"))
+            if l.strip() and l[0] != "#"]
+    fp16_row = [r for r in rows if r[0] == "FP16"][0]
+    assert int(fp16_row[1], 2) == 1 << 9                   # the pattern the paper prints: first mantissa bit only
+    golden = float(fp16_row[2])                            # 0.00003052 as printed
+    for dtype, first_mantissa_bit, survives in ((orc.FP16, 9, True), (orc.BF16, 6, False)):
+        A, Bt = synth.round_to_storage(a, dtype), synth.round_to_storage(b, dtype)
+        C0, *_ = orc.gemm(dtype, A, Bt)
+        assert C0[0, 0] == 15.0
+        s = site(orc.KIND_TERM, 0, 0, 2, 1 << first_mantissa_bit)                       # term 2 is 0 * 5 = 0
+        r = orc.campaign(dtype, A, Bt, C0, s, orc.TERM_IN_FORMAT, kstep=4)[0]
+        assert r["before_bits"] == 0 and r["after_bits"] == 1 << first_mantissa_bit
+        flipped = orc.widen(dtype, 1 << first_mantissa_bit)
+        if dtype == orc.FP16:
+            assert abs(flipped - golden) < 5e-9 and flipped == 2.0 ** -15               # 0000001000000000 = 0.00003052
+        else:
+            assert flipped == 2.0 ** -127
+        if survives:
+            assert bits_f32(int(r["final_bits"])) == float(np.float32(np.float32(7.0 - 0.0 + 2.0 ** -15) + np.float32(8.0)))
+            assert r["status"] & 1 and r["max_abs_dev"] > 0
+        else:
+            assert bits_f32(int(r["final_bits"])) == 15.0 and r["status"] == 0 and r["max_abs_dev"] == 0.0
+        # under the FP32-product reading the same mask is a low mantissa bit of an FP32 zero: nothing survives
+        r32 = orc.campaign(dtype, A, Bt, C0, s, 0, kstep=4)[0]
+        assert r32["status"] == 0
+    # closed forms, exact data: sign flip of the narrow product subtracts it twice; exponent LSB doubles or halves it
+    for dtype in (orc.FP16, orc.BF16, orc.TF32):
+        A, Bt = synth.round_to_storage(a, dtype), synth.round_to_storage(b, dtype)
+        C0, *_ = orc.gemm(dtype, A, Bt)
+        sign = 18 if dtype == orc.TF32 else 15
+        exp_lsb = {orc.FP16: 10, orc.BF16: 7, orc.TF32: 10}[dtype]
+        r = orc.campaign(dtype, A, Bt, C0, site(orc.KIND_TERM, 0, 0, 3, 1 << sign), orc.TERM_IN_FORMAT, kstep=4)[0]
+        assert bits_f32(int(r["final_bits"])) == 15.0 - 2 * 3.0
+        r = orc.campaign(dtype, A, Bt, C0, site(orc.KIND_TERM, 0, 0, 3, 1 << exp_lsb), orc.TERM_IN_FORMAT, kstep=4)[0]
+        p_new = orc.widen(dtype, orc.flip_operand(dtype, orc.round_to_operand(dtype, f32_bits(3.0)), 1 << exp_lsb))
+        assert p_new in (1.5, 6.0) and bits_f32(int(r["final_bits"])) == 15.0 - 3.0 + p_new
+        # the product-level check sees the widened faulty product: top exponent bit of the format's word
+        top = sign - 1
+        # term 4 is 1 * 1 = 1.0: with the top exponent bit of the format's word set it is infinite in every format;
+        # RangeCheck-max detects it (exponent 255 above the bound 127 + 127 - 126 = 128) and puts the bound in: 2.0
+        mode = orc.T_RMAX | orc.CORRECT | orc.TERM_IN_FORMAT
+        r = orc.campaign(dtype, A, Bt, C0, site(orc.KIND_TERM, 0, 0, 4, 1 << top), mode, kstep=4)[0]
+        Cf, _, log, _ = orc.gemm(dtype, A, Bt, site(orc.KIND_TERM, 0, 0, 4, 1 << top), mode, kstep=4)
+        assert r["final_bits"] == f32_bits(float(Cf[0, 0])) and log["status"][0] & 4
+        assert np.isinf(orc.widen(dtype, int(log["after_bits"][0]))) and log["final_bits"][0] == f32_bits(2.0)
+        assert float(Cf[0, 0]) == 15.0 - 1.0 + 2.0
+    # mask 0 away from exact data: the narrow product is subtracted and added back, at most two roundings of the sum
+    rng = np.random.default_rng(82)
+    A = synth.round_to_storage(rng.standard_normal((1, 40)).astype(np.float32), orc.BF16)
+    Bt = synth.round_to_storage(rng.standard_normal((1, 40)).astype(np.float32), orc.BF16)
+    C0, *_ = orc.gemm(orc.BF16, A, Bt)
+    r = orc.campaign(orc.BF16, A, Bt, C0, site(orc.KIND_TERM, 0, 0, 17, 0), orc.TERM_IN_FORMAT, kstep=8)[0]
+    ap = orc.absprod(orc.BF16, A, Bt)[0, 0]
+    assert abs(bits_f32(int(r["final_bits"])) - float(C0[0, 0])) <= 2 * 2.0 ** -23 * ap
