@@ -111,6 +111,18 @@ enum {
      */
     MPGEMMFI_TERM_HMMA_STEP = 32,
     /*
+     * Campaigns only: an alternative reading of where the paper's fault lands. Section IV-C flips bits "within the
+     * result of a multiplication" without saying in which format that result is held; Section V-B's example of a
+     * flipped zero is a 16-bit FP16 pattern, and the paper's format-dependent findings (Table II) need the product
+     * to live in the operand format. With this flag a TERM trial rounds the product to the operand format (to
+     * nearest even), applies xor_mask to that format's storage bits exactly as for an operand site (bits 0..15;
+     * TF32: bits 0..18 addressing bits 13..31 of the word), widens the result back to FP32, and applies Eq. 1-2
+     * with the rounded product as the term taken out and the flipped one as the term put in. The record's
+     * before_bits / after_bits are then words of the operand format. Without the flag (the default, and what
+     * mpgemmfi_gemm does) the flipped word is the FP32 product.
+     */
+    MPGEMMFI_TERM_IN_FORMAT = 128,
+    /*
      * mpgemmfi_gemm_ranged only, together with RANGE_MAX or RANGE_FLIP: also range-check every
      * OUTPUT element. This extends the product bound of Section VI-A to a dot product and is not in
      * the paper: with EA_i / EB_j the largest FP32 exponent fields in row i of A / row j of Bt,

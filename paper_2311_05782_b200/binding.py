@@ -19,6 +19,7 @@ CORRECT = 16
 TERM_HMMA_STEP = 32
 OUT_FP32, OUT_FP16, OUT_BF16 = 0, 1, 2
 OUTPUT_RANGE = 64
+TERM_IN_FORMAT = 128
 STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT = 1, 2
 MAX_FAULTS = 4096
 STATIC_MAX_TRIALS = 65536

@@ -359,7 +359,7 @@ int mpgemmfi_campaign(int dtype, int M, int N, int K, const void *A, const void 
     int rc = check_common(dtype, M, N, K, A, Bt, C_clean);
     if (rc) return rc;
     if (n_trials < 0 || (n_trials > 0 && (!sites || !records))) return MPGEMMFI_ERR_ARG;
-    if (detect_mode & ~(MPGEMMFI_DETECT_TECHNIQUE_MASK | MPGEMMFI_CORRECT | MPGEMMFI_TERM_HMMA_STEP)) return MPGEMMFI_ERR_ARG;
+    if (detect_mode & ~(MPGEMMFI_DETECT_TECHNIQUE_MASK | MPGEMMFI_CORRECT | MPGEMMFI_TERM_HMMA_STEP | MPGEMMFI_TERM_IN_FORMAT)) return MPGEMMFI_ERR_ARG;
     if (((uintptr_t)sites & 15) || ((uintptr_t)records & 7)) return MPGEMMFI_ERR_ALIGN;
     if (!workspace || ((uintptr_t)workspace & 255) ||
         workspace_bytes < mpgemmfi_campaign_workspace_bytes(dtype, M, N, K, n_trials))
@@ -387,7 +387,7 @@ int mpgemmfi_campaign_static(int dtype, int M, int N, int K, const void *A, cons
     int rc = check_common(dtype, M, N, K, A, Bt, C_clean);
     if (rc) return rc;
     if (n_trials < 0 || (n_trials > 0 && (!sites || !records))) return MPGEMMFI_ERR_ARG;
-    if (detect_mode & ~(MPGEMMFI_DETECT_TECHNIQUE_MASK | MPGEMMFI_CORRECT | MPGEMMFI_TERM_HMMA_STEP)) return MPGEMMFI_ERR_ARG;
+    if (detect_mode & ~(MPGEMMFI_DETECT_TECHNIQUE_MASK | MPGEMMFI_CORRECT | MPGEMMFI_TERM_HMMA_STEP | MPGEMMFI_TERM_IN_FORMAT)) return MPGEMMFI_ERR_ARG;
     if (((uintptr_t)sites & 15) || ((uintptr_t)records & 7)) return MPGEMMFI_ERR_ALIGN;
     if (n_trials > MPGEMMFI_STATIC_MAX_TRIALS) return MPGEMMFI_ERR_WORKSPACE;   // built-in scratch too small
     DeviceInfo di;

@@ -168,6 +168,16 @@ __global__ void __launch_bounds__(256) element_kernel(CampaignParams p)
                     before = f32_bits(acc_f);
                     after = before ^ s.xor_mask;
                     acc_f = bits_f32(after);
+                } else if (p.detect_mode & MPGEMMFI_TERM_IN_FORMAT) {
+                    // the product as a word of the operand format: rounded to it, flipped there, widened back; Eq. 1-2
+                    // with this re_2 and its flipped version
+                    before = round_to_operand(p.dtype, re2);
+                    after = flip_operand(p.dtype, before, s.xor_mask);
+                    const float re2_n = widen_operand(p.dtype, before);
+                    bool det;
+                    const uint32_t fin = product_check(p.detect_mode, f32_bits(widen_operand(p.dtype, after)), f32_bits(a_site),
+                                                       f32_bits(b_site), det);
+                    acc_f = __fadd_rn(__fsub_rn(acc_f, re2_n), bits_f32(fin));
                 } else {
                     before = f32_bits(re2);
                     after = before ^ s.xor_mask;

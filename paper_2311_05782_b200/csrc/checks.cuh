@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cstdint>
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 #include "../../include/mpgemmfi.h"
@@ -33,6 +34,18 @@ __device__ __forceinline__ float widen_operand(int dtype, uint32_t s)
     if (dtype == MPGEMMFI_BF16) return __uint_as_float(s << 16);
     if (dtype == MPGEMMFI_TF32) return __uint_as_float(s & 0xFFFFE000u);
     return __half2float(__ushort_as_half(static_cast<unsigned short>(s)));
+}
+
+// FP32 value -> storage word of the operand format, round to nearest even (FP16 / BF16: the conversion
+// instructions; TF32: on the 13 dropped bits of the FP32 word, Inf kept, NaN kept a NaN)
+__device__ __forceinline__ uint32_t round_to_operand(int dtype, float v)
+{
+    if (dtype == MPGEMMFI_FP16) return __half_as_ushort(__float2half_rn(v));
+    if (dtype == MPGEMMFI_BF16) return __bfloat16_as_ushort(__float2bfloat16_rn(v));
+    const uint32_t u = __float_as_uint(v);
+    if (((u >> 23) & 0xFFu) == 0xFFu) return (u & 0xFFFFE000u) | ((u & 0x7FFFFFu) ? 0x00400000u : 0u);
+    const uint32_t keep = u >> 13, rest = u & 0x1FFFu;
+    return (keep + ((rest > 0x1000u || (rest == 0x1000u && (keep & 1u))) ? 1u : 0u)) << 13;
 }
 
 __device__ __forceinline__ uint32_t load_operand(int dtype, const void *base, size_t idx)

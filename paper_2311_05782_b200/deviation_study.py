@@ -45,11 +45,17 @@ def log2_quantile(hist: np.ndarray, q: float):
     return e - 127 if e < 255 else float("inf")
 
 
-def run_cell(mpg, synth, torch, workload: str, fmt: int, nbits: int, mode: int, trials: int, seed: int = 1):
-    """One cell of the study; returns the device summary (numpy record) and the derived figures."""
+def run_cell(mpg, synth, torch, workload: str, fmt: int, nbits: int, mode: int, trials: int, seed: int = 1,
+             in_format: bool = False):
+    """One cell of the study; returns the device summary (numpy record) and the derived figures.
+    in_format: the product is held in the operand format when its bits are flipped (MPGEMMFI_TERM_IN_FORMAT; the
+    masks then lie in that format's 16 or 19 bits) instead of in FP32."""
     cfg, M, N, K = WORKLOADS[workload]
     A, Bt = synth.make_operands(cfg, M, N, K, dtype=fmt)
-    sites = synth.make_sites("term", fmt, M, N, K, trials, synth.config_seed(cfg) + 100 * nbits + seed, nbits=nbits)
+    sites = synth.make_sites("term_op" if in_format else "term", fmt, M, N, K, trials,
+                             synth.config_seed(cfg) + 100 * nbits + seed, nbits=nbits)
+    if in_format:
+        mode |= mpg.TERM_IN_FORMAT
     view = np.int32 if fmt == synth.DTYPE_TF32 else np.int16
     a = torch.from_numpy(A.view(view)).cuda()
     b = torch.from_numpy(Bt.view(view)).cuda()
@@ -73,6 +79,8 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--trials", type=int, default=50000)
     ap.add_argument("--json", default=None)
+    ap.add_argument("--product", default="fp32", choices=["fp32", "operand"],
+                    help="format the product is held in when its bits are flipped (default: FP32, the library's default)")
     args = ap.parse_args()
     import torch
 
@@ -86,7 +94,7 @@ def main():
         for fname, fmt in FORMATS.items():
             for nbits in (1, 2, 4):
                 for tname, mode in TECHNIQUES.items():
-                    _, cell = run_cell(mpg, synth, torch, wname, fmt, nbits, mode, args.trials)
+                    _, cell = run_cell(mpg, synth, torch, wname, fmt, nbits, mode, args.trials, in_format=args.product == "operand")
                     results[f"{wname}/{fname}/{nbits}bit/{tname}"] = cell
     print(f"{'cell':46s} {'zero-diff %':>11s} {'median':>7s} {'p80':>5s} {'max':>5s} {'inf':>6s}")
     for k, c in results.items():
@@ -94,7 +102,7 @@ def main():
               f"{str(c['log2_max']):>5s} {c['infinite']:6d}")
     if args.json:
         with open(args.json, "w") as f:
-            json.dump({"trials_per_cell": args.trials, "cells": results}, f, indent=1)
+            json.dump({"trials_per_cell": args.trials, "product": args.product, "cells": results}, f, indent=1)
 
 
 if __name__ == "__main__":

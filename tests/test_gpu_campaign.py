@@ -302,3 +302,37 @@ def test_deviation_study_cell_against_the_oracle(workload, fmt, nbits, mode):
     assert diff[:5].sum() == 0 and diff[6:16].sum() == 0, (got[:16], want[:16])
     assert diff[16:].sum() <= 2 * nan_made and diff[5] <= nan_made
     assert cell["trials"] == trials and abs(cell["zero_diff_pct"] - 100.0 * want[2] / trials) < 1e-9
+
+
+@pytest.mark.parametrize("dtype,name", [(orc.FP16, "c5"), (orc.BF16, "c2"), (orc.TF32, "c4")])
+@pytest.mark.parametrize("nbits", [1, 2, 4])
+def test_campaign_term_trials_with_the_product_in_the_operand_format(dtype, name, nbits):
+    """MPGEMMFI_TERM_IN_FORMAT: the product rounded to the operand format, flipped there, written back by Eq. 1-2.
+    Both sides walk the same sums in the same order: the records agree bit for bit (NaN payloads aside), at the GEMM's
+    k-step and at HMMA granularity, under every technique."""
+    M, N, K = 192, 160, 208
+    A, Bt = synth.make_operands(name, M, N, K, dtype=dtype)
+    sites = synth.make_sites("term_op", dtype, M, N, K, 300, 199 + nbits, nbits=nbits)
+    step = 8 if dtype == orc.TF32 else 16
+    Cclean, *_ = orc.gemm(dtype, A, Bt)
+    for tech in (orc.T_NONE, orc.T_BOUND | orc.CORRECT, orc.T_RMAX | orc.CORRECT, orc.T_RFLIP | orc.CORRECT, orc.T_RMAX):
+        for hmma in (True, False):
+            _, rg = run_gpu_campaign(dtype, A, Bt, sites, tech | mpg.TERM_IN_FORMAT | (mpg.TERM_HMMA_STEP if hmma else 0))
+            ro = orc.campaign(dtype, A, Bt, Cclean, sites, tech | orc.TERM_IN_FORMAT, kstep=step if hmma else None)
+            raw = orc.campaign(dtype, A, Bt, Cclean, sites, (tech & ~orc.CORRECT) | orc.TERM_IN_FORMAT, kstep=step if hmma else None)
+            nan_made = np.isnan(raw["final_bits"].view(np.float32))
+            for f in rg.dtype.names:
+                same = rg[f] == ro[f]
+                if f in ("final_bits", "max_abs_dev"):
+                    same |= nan_made
+                if f == "max_abs_dev":
+                    same |= np.isnan(rg[f]) & np.isnan(ro[f])
+                assert same.all(), (tech, hmma, f, np.nonzero(~same)[0][:5], rg[~same][:2], ro[~same][:2])
+    # it changes what a trial does: an FP16 zero product with a flipped mantissa bit now shows in the sum
+    if dtype == orc.FP16:
+        _, r32 = run_gpu_campaign(dtype, A, Bt, sites, mpg.TERM_HMMA_STEP)
+        _, r16 = run_gpu_campaign(dtype, A, Bt, sites, mpg.TERM_HMMA_STEP | mpg.TERM_IN_FORMAT)
+        assert (r16["status"] & 1).sum() > (r32["status"] & 1).sum()
+    # the GEMM entry point does not take the flag
+    with pytest.raises(mpg.MpgemmfiError):
+        mpg.gemm(dtype, to_dev(A, dtype), to_dev(Bt, dtype), sites[:1], mpg.TERM_IN_FORMAT)
