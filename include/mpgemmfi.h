@@ -368,7 +368,8 @@ int mpgemmfi_campaign_summary(const mpgemmfi_trial_record *records, int n_trials
  *   SINGLE every CTA computes whole 128 x {64,128,256} tiles
  *   PAIR   two CTAs on neighbouring SMs share one 256 x 256 tile and the Bt tile (tcgen05
  *          cta_group::2); falls back to SINGLE when the device cannot host such pairs
- * Process-wide, not thread-safe against concurrent launches. Results are the same fault
+ * Process-wide; read once when a launch is queued (a host thread that changes it while another
+ * queues a launch gives that launch the old or the new value). Results are the same fault
  * semantics either way; individual output values may differ in rounding between policies.
  * Returns MPGEMMFI_OK or MPGEMMFI_ERR_ARG.
  */
@@ -393,7 +394,7 @@ int mpgemmfi_set_tile_policy(int policy);
  * accumulation in increasing k, bit-identical to the uncut tile, and accumulator / term sites meet
  * the same running sum. While the launch runs, C therefore holds intermediate values in those
  * tiles. The hand-over between walkers uses 160 KB of static device memory of the library,
- * tagged per launch. Process-wide, not thread-safe against concurrent launches.
+ * tagged per launch. Process-wide; read once when a launch is queued.
  * Returns MPGEMMFI_OK or MPGEMMFI_ERR_ARG.
  */
 enum {

@@ -1,4 +1,5 @@
 // C ABI of the library: argument checks, tensor-map encoding, kernel launches.
+#include <atomic>
 #include <cstdint>
 #include <cstring>
 #include <cuda.h>
@@ -14,7 +15,7 @@ static_assert(MPGEMMFI_STATIC_MAX_TRIALS == mpg::CAMPAIGN_STATIC_MAX_TRIALS, "he
 
 namespace {
 
-int g_last_cuda_error = 0;
+std::atomic<int> g_last_cuda_error{0};
 
 int cuda_fail(cudaError_t e)
 {
@@ -118,10 +119,12 @@ int encode_output_map16(CUtensorMap *map, void *D, int out_fmt, int M, int N)
     return MPGEMMFI_OK;
 }
 
-int g_tile_policy = MPGEMMFI_TILES_AUTO;
-int g_split_policy = MPGEMMFI_SPLIT_AUTO;
-int g_wait_limit_ms = 4000;
-int g_break_handover = 0;
+// process-wide knobs: each is read once when a launch is queued; atomics, so that a host thread changing one while
+// another queues a launch gives that launch either the old or the new value, never a torn one
+std::atomic<int> g_tile_policy{MPGEMMFI_TILES_AUTO};
+std::atomic<int> g_split_policy{MPGEMMFI_SPLIT_AUTO};
+std::atomic<int> g_wait_limit_ms{4000};
+std::atomic<int> g_break_handover{0};
 
 // Split schedule for `tiles` tiles on `walkers` tile walkers: fills the three schedule fields of p.
 // Off unless there is at least one full round, the left-over tiles number at most half the walkers,
@@ -130,7 +133,8 @@ void choose_split(mpg::GemmParams &p, int walkers)
 {
     p.split_parts = 0; p.full_rounds = 0; p.left_tiles = 0;
     // (a cut tile's unfinished FP32 sums wait in C: not with a 16-bit C)
-    if (g_split_policy == MPGEMMFI_SPLIT_OFF || !p.c_vec_ok || p.out_fmt != MPGEMMFI_OUT_FP32) return;
+    const int policy = g_split_policy.load();
+    if (policy == MPGEMMFI_SPLIT_OFF || !p.c_vec_ok || p.out_fmt != MPGEMMFI_OUT_FP32) return;
     const int rounds = p.num_tiles / walkers, left = p.num_tiles % walkers;
     if (rounds < 1 || left == 0 || left * 16 > mpg::SPLIT_SIGNAL_WORDS) return;
     int parts = walkers / left;
@@ -138,7 +142,7 @@ void choose_split(mpg::GemmParams &p, int walkers)
     if (parts > rounds + 1) parts = rounds + 1;
     while (parts >= 2 && p.num_kt / parts < 4) --parts;
     if (parts < 2) return;
-    if (g_split_policy == MPGEMMFI_SPLIT_AUTO) {
+    if (policy == MPGEMMFI_SPLIT_AUTO) {
         // a cut tile costs its walkers one more pass of accumulators through C (measured: about 5 us); it
         // pays when the k-tiles saved (0.35 us each) outweigh that and are a visible share of the launch
         const int saved = p.num_kt - (p.num_kt + parts - 1) / parts;
@@ -163,10 +167,11 @@ int choose_bn(int M, int N, int num_sms)
 // 256 x 256 tiles on CTA pairs pay off once there are enough of them to occupy most pairs
 bool choose_pair(int dtype, int M, int N, int *max_pairs)
 {
-    if (g_tile_policy == MPGEMMFI_TILES_SINGLE) return false;
+    const int policy = g_tile_policy.load();
+    if (policy == MPGEMMFI_TILES_SINGLE) return false;
     *max_pairs = mpg::gemm_max_resident_pairs(dtype);
     if (*max_pairs <= 0) return false;
-    if (g_tile_policy == MPGEMMFI_TILES_PAIR) return true;
+    if (policy == MPGEMMFI_TILES_PAIR) return true;
     const long long tiles = (long long)((M + 255) / 256) * ((N + 255) / 256);
     return M > 128 && N > 128 && tiles >= *max_pairs / 2;
 }
