@@ -509,7 +509,13 @@ def main():
     achieved = flops / (ms_inj / args.steps * 1e-3) / 1e12
 
     min_bytes = (M * K + N * K) * A.element_size() + M * N * 4 + M * ((N + 31) // 32) * 4
-    if args.config == "c5":
+    if args.config == "c1":
+        # 33.6 MFLOP on four tiles: a single wave, bound by launch and pipeline-fill latency; reported in microseconds
+        us = ms_inj / args.steps * 1e3
+        roofline = {"bound": "latency", "achieved": us, "peak": None, "unit": "us per GEMM", "frac": None, "traffic": None,
+                    "kernel": "gemm_kernel", "flops_per_launch": flops, "min_bytes_per_launch": min_bytes,
+                    "note": "one wave of tiles: neither the tensor pipe nor HBM can be kept busy"}
+    elif args.config == "c5":
         # narrow N: about 52 flop per byte, below the ridge; the GEMM is bound by HBM
         gbs = min_bytes / (ms_inj / args.steps * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -45,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
                     raise subprocess.CalledProcessError(r.returncode, r.args)
     objs = [os.path.join(OBJ_DIR, s[:-3] + ".o") for s in SOURCES]
     if jobs or not os.path.exists(LIB) or os.path.getmtime(LIB) < max(os.path.getmtime(o) for o in objs):
-        subprocess.run([nvcc, *ARCH, "-shared", "-Xcompiler", "-fPIC", "-o", LIB, *objs], check=True)
+        subprocess.run([nvcc, *ARCH, "-shared", "-Xcompiler", "-fPIC", "-o", LIB, *objs, "-ldl"], check=True)
     return LIB
 
 

@@ -4,6 +4,7 @@
 #include <cstring>
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include "../../include/mpgemmfi.h"
 #include "campaign.cuh"
@@ -22,6 +23,15 @@ int cuda_fail(cudaError_t e)
     g_last_cuda_error = (int)e;
     return MPGEMMFI_ERR_CUDA;
 }
+
+// NVTX range over the queueing of one part of a call (a profiler's timeline then shows the clean GEMM and the trial
+// kernels of a campaign apart); a no-op when no tool is attached
+struct Range {
+    explicit Range(const char *name) { nvtxRangePushA(name); }
+    ~Range() { nvtxRangePop(); }
+    Range(const Range &) = delete;
+    Range &operator=(const Range &) = delete;
+};
 
 struct DeviceInfo {
     bool known = false;
@@ -191,6 +201,7 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, void
              const uint32_t *exp_a = nullptr, const uint32_t *exp_bt = nullptr, const float *addend = nullptr,
              int out_fmt = MPGEMMFI_OUT_FP32)
 {
+    Range range("mpgemmfi: gemm");
     int max_pairs = 0;
     const bool pair = choose_pair(dtype, M, N, &max_pairs);
     const int bn = pair ? 256 : choose_bn(M, N, di.num_sms);
@@ -381,6 +392,7 @@ int mpgemmfi_campaign(int dtype, int M, int N, int K, const void *A, const void 
     p.dtype = dtype; p.M = M; p.N = N; p.K = K; p.detect_mode = detect_mode; p.n_trials = n_trials;
     p.A = A; p.Bt = Bt; p.C = C_clean; p.sites = sites; p.records = records;
     mpg::campaign_bind_schedule(p, workspace);
+    Range range("mpgemmfi: campaign trials");
     const cudaError_t e = mpg::launch_campaign_trials(p, di.num_sms, st);
     return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
 }
@@ -411,6 +423,7 @@ int mpgemmfi_campaign_static(int dtype, int M, int N, int K, const void *A, cons
     p.dtype = dtype; p.M = M; p.N = N; p.K = K; p.detect_mode = detect_mode; p.n_trials = n_trials;
     p.A = A; p.Bt = Bt; p.C = C_clean; p.sites = sites; p.records = records;
     mpg::campaign_bind_schedule(p, scratch);
+    Range range("mpgemmfi: campaign trials");
     e = mpg::launch_campaign_trials(p, di.num_sms, st);   // clears the schedule counters first
     return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
 }
