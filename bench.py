@@ -287,9 +287,14 @@ def main():
     local_rank = env_int("LOCAL_RANK", 0)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if env_int("MPGEMMFI_BENCH_ONE_DEVICE", 0):
+        local_rank = 0      # rehearsal of the N > 1 path where there is one GPU: every rank on device 0, gloo instead of nccl
     torch.cuda.set_device(local_rank)
     if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        if env_int("MPGEMMFI_BENCH_ONE_DEVICE", 0):
+            dist.init_process_group("gloo")
+        else:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     mpg.load_library()
 
     w = synth.make_workload(args.config)
@@ -430,7 +435,7 @@ def main():
         torch.cuda.synchronize(dev)
         ms_sh = reduce_max(e0.elapsed_time(e1), world, dev)
         sharded = {"trials": len(w.sites), "ms": ms_sh, "trials_per_s": len(w.sites) / (ms_sh * 1e-3),
-                   "gathered_record_bytes": int(allrec.numel() * 4), "collective": "one all_gather (nccl)"}
+                   "gathered_record_bytes": int(allrec.numel() * 4), "collective": f"one all_gather ({dist.get_backend()})"}
 
     # ---- end to end: pinned host buffers, copies inside the timed region
     hA = torch.from_numpy(w.A.view(view)).pin_memory()

@@ -21,6 +21,8 @@ def _reduce(value: float, world: int, device, op_name: str) -> float:
         return float(value)
     import torch
     import torch.distributed as dist
+    if dist.get_backend() != "nccl":
+        device = "cpu"
     t = torch.tensor([value], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=getattr(dist.ReduceOp, op_name))
     return float(t.item())
@@ -53,13 +55,17 @@ def gather_records(local, counts, group=None):
     if world <= 1:
         return flat
     block = max(counts) * RECORD_BYTES
-    send = torch.zeros(block, dtype=torch.uint8, device=flat.device)
-    send[:flat.numel()] = flat
-    recv = torch.empty(world * block, dtype=torch.uint8, device=flat.device)
+    # the collective runs where the group's backend works: device memory for nccl, host memory for gloo (the records
+    # then travel through the host and come back to the device they were on)
+    home = flat.device
+    coll = home if dist.get_backend(group) == "nccl" else torch.device("cpu")
+    send = torch.zeros(block, dtype=torch.uint8, device=coll)
+    send[:flat.numel()] = flat.to(coll)
+    recv = torch.empty(world * block, dtype=torch.uint8, device=coll)
     dist.all_gather_into_tensor(recv, send, group=group)
-    if all(c == counts[0] for c in counts):
-        return recv
-    return torch.cat([recv[r * block:r * block + counts[r] * RECORD_BYTES] for r in range(world)])
+    if not all(c == counts[0] for c in counts):
+        recv = torch.cat([recv[r * block:r * block + counts[r] * RECORD_BYTES] for r in range(world)])
+    return recv.to(home)
 
 
 def campaign_sharded(dtype, A, Bt, sites, detect_mode, group=None, run_local=None):
