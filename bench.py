@@ -138,12 +138,12 @@ def oracle_sample_run(w, rows, n_sites=1):
     return time.perf_counter() - t0
 
 
-def cpu_baseline(w, budget_s=12.0):
+def cpu_baseline(w, limit_s=12.0):
     import oracle as orc
     orc.build()
     t_small, t_probe = oracle_sample_run(w, 32), oracle_sample_run(w, 160)
     per_row = max((t_probe - t_small) / 128.0, 1e-6)          # the fixed part (widening Bt) is not per-row work
-    rows = int(min(w.M, max(160, (budget_s - t_small) / per_row)))
+    rows = int(min(w.M, max(160, (limit_s - t_small) / per_row)))
     rows = max(32, (rows // 32) * 32)
     t = oracle_sample_run(w, rows)
     flops = 2.0 * rows * w.N * w.K

@@ -56,7 +56,7 @@ constexpr int SITE_CACHE = 64;
 constexpr int MAX_STAGES = 8;
 constexpr int OUT_BUF_BYTES = 16 * 128;                    // staging of one epilogue warp: 16 rows x 128 bytes
 constexpr int OUT_STAGING_BYTES = EPI_WARPS * OUT_BUF_BYTES;
-constexpr int SMEM_BUDGET = 227 * 1024;                    // dynamic shared memory one CTA may have
+constexpr int SMEM_LIMIT = 227 * 1024;                    // dynamic shared memory one CTA may have
 constexpr int CONTROL_RESERVE = 12 * 1024;                 // control block + 1 KB of alignment slack
 
 template <int BN, bool kPair>
@@ -66,7 +66,7 @@ struct Cfg {
     static constexpr int B_BYTES = B_ROWS * 128;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     // the operand ring gets what the output staging and the control block leave
-    static constexpr int STAGES_FIT = (SMEM_BUDGET - CONTROL_RESERVE - OUT_STAGING_BYTES) / STAGE_BYTES;
+    static constexpr int STAGES_FIT = (SMEM_LIMIT - CONTROL_RESERVE - OUT_STAGING_BYTES) / STAGE_BYTES;
     static constexpr int STAGES = STAGES_FIT < MAX_STAGES ? STAGES_FIT : MAX_STAGES;
     static_assert(STAGES >= 3, "operand ring too short");
     static constexpr int TMEM_COLS = 2 * BN;   // two accumulators; 128, 256 or 512 columns
@@ -1196,7 +1196,7 @@ cudaError_t launch_one(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const C
 {
     using C = Cfg<BN, kPair>;
     const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024;
-    static_assert(C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024 <= SMEM_BUDGET, "shared memory over budget");
+    static_assert(C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024 <= SMEM_LIMIT, "shared memory over the limit");
     static bool configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -1232,7 +1232,7 @@ int gemm_max_resident_pairs(int dtype)
     if (cache[dev][tf] == 0) {
         using C = Cfg<256, true>;
         const size_t smem = (size_t)C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024;
-    static_assert(C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024 <= SMEM_BUDGET, "shared memory over budget");
+    static_assert(C::STAGES * C::STAGE_BYTES + OUT_STAGING_BYTES + sizeof(Control) + 1024 <= SMEM_LIMIT, "shared memory over the limit");
         auto kern = tf ? gemm_kernel<256, true, true> : gemm_kernel<256, false, true>;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return 0;
         cudaLaunchConfig_t cfg = {};
