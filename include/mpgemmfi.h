@@ -428,6 +428,16 @@ int mpgemmfi_debug_break_handover(int on);
  */
 int mpgemmfi_debug_launch_slot(uint32_t counter, uint32_t *tag);
 
+/*
+ * Host logic of the tile schedule (no device needed): for `num_tiles` output tiles of `num_kt` k-steps each on
+ * `walkers` tile walkers (CTAs or CTA pairs) under split policy `policy`, writes one 8-word entry per piece of
+ * work, walker by walker in the order the walker runs them: {walker, index, tile, first k-step, end k-step, part,
+ * starts from the sums a previous part left in C (0/1), leaves its sums in C for the next part (0/1)}. At most
+ * max_out entries are written; the return value is the number of entries there are (or MPGEMMFI_ERR_ARG). It assumes
+ * an FP32 C that allows 16-byte accesses, as the split schedule requires.
+ */
+int mpgemmfi_debug_segments(int num_tiles, int num_kt, int walkers, int policy, uint32_t *out, int max_out);
+
 /* k elements between two accumulator boundaries: 64 (FP16, BF16), 32 (TF32); 0 for a bad dtype. */
 int mpgemmfi_kstep(int dtype);
 

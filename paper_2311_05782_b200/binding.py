@@ -48,7 +48,7 @@ _SYMBOLS = [
     "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version", "mpgemmfi_campaign_static",
     "mpgemmfi_set_tile_policy", "mpgemmfi_set_split_policy", "mpgemmfi_campaign_summary", "mpgemmfi_operand_exponents", "mpgemmfi_gemm_ranged",
     "mpgemmfi_gemm_addend", "mpgemmfi_set_wait_limit_ms", "mpgemmfi_debug_break_handover", "mpgemmfi_debug_launch_slot",
-    "mpgemmfi_gemm_out16",
+    "mpgemmfi_gemm_out16", "mpgemmfi_debug_segments",
 ]
 
 
@@ -105,6 +105,8 @@ def load_library():
     L.mpgemmfi_debug_break_handover.argtypes = [i]
     L.mpgemmfi_debug_launch_slot.restype = i
     L.mpgemmfi_debug_launch_slot.argtypes = [C.c_uint32, C.POINTER(C.c_uint32)]
+    L.mpgemmfi_debug_segments.restype = i
+    L.mpgemmfi_debug_segments.argtypes = [i, i, i, i, vp, i]
     L.mpgemmfi_kstep.restype = i
     L.mpgemmfi_kstep.argtypes = [i]
     L.mpgemmfi_flags_bytes.restype = sz
@@ -208,6 +210,18 @@ def mpgemmfi_debug_launch_slot(counter):
     tag = C.c_uint32(0)
     slot = load_library().mpgemmfi_debug_launch_slot(int(counter) & 0xFFFFFFFF, C.byref(tag))
     return slot, tag.value
+
+
+def mpgemmfi_debug_segments(num_tiles, num_kt, walkers, policy):
+    """The tile schedule as the kernel's walkers will run it: uint32 array [n, 8] of
+    (walker, index, tile, kt0, kt1, part, load, save)."""
+    L = load_library()
+    n = L.mpgemmfi_debug_segments(num_tiles, num_kt, walkers, policy, None, 0)
+    if n < 0:
+        raise MpgemmfiError(n, "mpgemmfi_debug_segments")
+    out = np.zeros((n, 8), dtype=np.uint32)
+    L.mpgemmfi_debug_segments(num_tiles, num_kt, walkers, policy, out.ctypes.data_as(C.c_void_p), n)
+    return out
 
 
 def mpgemmfi_kstep(dtype):

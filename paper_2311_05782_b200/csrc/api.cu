@@ -136,14 +136,12 @@ std::atomic<int> g_split_policy{MPGEMMFI_SPLIT_AUTO};
 std::atomic<int> g_wait_limit_ms{4000};
 std::atomic<int> g_break_handover{0};
 
-// Split schedule for `tiles` tiles on `walkers` tile walkers: fills the three schedule fields of p.
-// Off unless there is at least one full round, the left-over tiles number at most half the walkers,
-// every part keeps at least four k-tiles, and (policy AUTO) the launch gets visibly shorter.
-void choose_split(mpg::GemmParams &p, int walkers)
+}  // namespace
+
+void mpg::choose_split_schedule(mpg::GemmParams &p, int walkers, int policy)
 {
     p.split_parts = 0; p.full_rounds = 0; p.left_tiles = 0;
     // (a cut tile's unfinished FP32 sums wait in C: not with a 16-bit C)
-    const int policy = g_split_policy.load();
     if (policy == MPGEMMFI_SPLIT_OFF || !p.c_vec_ok || p.out_fmt != MPGEMMFI_OUT_FP32) return;
     const int rounds = p.num_tiles / walkers, left = p.num_tiles % walkers;
     if (rounds < 1 || left == 0 || left * 16 > mpg::SPLIT_SIGNAL_WORDS) return;
@@ -160,6 +158,8 @@ void choose_split(mpg::GemmParams &p, int walkers)
     }
     p.split_parts = parts; p.full_rounds = rounds; p.left_tiles = left;
 }
+
+namespace {
 
 // widest tile that still gives every SM a tile; narrow outputs get narrow tiles
 int choose_bn(int M, int N, int num_sms)
@@ -243,7 +243,7 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, void
     p.epoch = 0; p.signals = nullptr; p.ready = nullptr;
     p.wait_limit_ns = (uint64_t)g_wait_limit_ms * 1000000ull;
     p.tag_skew = g_break_handover ? 4u : 0u;        // test hook: an expected part number that nobody writes
-    choose_split(p, walkers);
+    mpg::choose_split_schedule(p, walkers, g_split_policy.load());
     int slot = -1;
     if (p.split_parts > 1 || flags) {
         // (the header and the site log of `flags` are cleared by the kernel itself)
@@ -473,6 +473,27 @@ int mpgemmfi_debug_launch_slot(uint32_t counter, uint32_t *epoch)
 {
     if (epoch) *epoch = mpg::gemm_epoch_of(counter);
     return mpg::gemm_slot_of(counter);
+}
+
+int mpgemmfi_debug_segments(int num_tiles, int num_kt, int walkers, int policy, uint32_t *out, int max_out)
+{
+    if (num_tiles <= 0 || num_kt <= 0 || walkers <= 0 || max_out < 0 || (max_out > 0 && !out)) return MPGEMMFI_ERR_ARG;
+    mpg::GemmParams p = {};
+    p.num_tiles = num_tiles; p.num_kt = num_kt; p.c_vec_ok = 1; p.out_fmt = MPGEMMFI_OUT_FP32;
+    mpg::choose_split_schedule(p, walkers, policy);
+    const uint32_t groups = (uint32_t)(num_tiles < walkers ? num_tiles : walkers);
+    int n = 0;
+    for (uint32_t gid = 0; gid < groups; ++gid) {
+        mpg::Segment sg;
+        for (uint32_t i = 0; mpg::get_segment(p, gid, groups, i, sg); ++i, ++n) {
+            if (n < max_out) {
+                uint32_t *o = out + 8 * (size_t)n;
+                o[0] = gid; o[1] = i; o[2] = sg.tile; o[3] = sg.kt0; o[4] = sg.kt1; o[5] = sg.part;
+                o[6] = sg.load ? 1u : 0u; o[7] = sg.save ? 1u : 0u;
+            }
+        }
+    }
+    return n;
 }
 
 int mpgemmfi_kstep(int dtype)

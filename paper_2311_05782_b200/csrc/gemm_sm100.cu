@@ -326,43 +326,6 @@ __device__ __forceinline__ uint32_t tile_number(const GemmParams &p, uint32_t tm
     return band * (uint32_t)p.group_m * (uint32_t)p.tiles_n + tn * rows + (tm - band * (uint32_t)p.group_m);
 }
 
-// One piece of work of a tile walker: k-tiles [kt0, kt1) of one output tile. `load`: the
-// accumulators of k-tiles [0, kt0) come from C (left there by the walker of the previous part);
-// `save`: the tile is not finished here, the raw accumulators go to C for the next part.
-struct Segment {
-    uint32_t tile, kt0, kt1, part;
-    bool load, save;
-};
-
-// i-th segment of walker `gid`. Plain schedule (split_parts <= 1): tiles gid, gid + groups, ...,
-// each whole. Split schedule: `full_rounds` whole tiles dealt out the same way, and the
-// `left_tiles` tiles of the last round cut into `split_parts` equal runs of k-tiles; part g of
-// left-over tile j belongs to walker g * left_tiles + j, which runs it after its g-th whole tile
-// (the last part: after all of them), so that part g is finished long before part g + 1 starts.
-__device__ __forceinline__ bool get_segment(const GemmParams &p, uint32_t gid, uint32_t groups, uint32_t i, Segment &sg)
-{
-    const uint32_t nkt = (uint32_t)p.num_kt;
-    if (p.split_parts <= 1) {
-        sg.tile = gid + i * groups;
-        sg.kt0 = 0; sg.kt1 = nkt; sg.part = 0; sg.load = false; sg.save = false;
-        return sg.tile < (uint32_t)p.num_tiles;
-    }
-    const uint32_t left = (uint32_t)p.left_tiles, parts = (uint32_t)p.split_parts, rounds = (uint32_t)p.full_rounds;
-    const uint32_t g = gid / left;
-    const bool has_part = g < parts;
-    const uint32_t pos = g + 1 < parts ? g : rounds;
-    if (i >= rounds + (has_part ? 1u : 0u)) return false;
-    if (has_part && i == pos) {
-        sg.tile = groups * rounds + gid % left;
-        sg.kt0 = g * nkt / parts; sg.kt1 = (g + 1) * nkt / parts; sg.part = g;
-        sg.load = g > 0; sg.save = g + 1 < parts;
-        return true;
-    }
-    sg.tile = gid + ((has_part && i > pos) ? i - 1 : i) * groups;
-    sg.kt0 = 0; sg.kt1 = nkt; sg.part = 0; sg.load = false; sg.save = false;
-    return true;
-}
-
 // Do the accumulators of this segment start from memory (the previous part's sums left in C, or the
 // addend of D = A x B + C at a tile's first k-tile) rather than from the first MMA's overwrite?
 __device__ __forceinline__ bool starts_from_memory(const GemmParams &p, const Segment &sg)

@@ -47,6 +47,43 @@ struct GemmParams {
     uint32_t tag_skew;
 };
 
+// One piece of work of a tile walker: k-tiles [kt0, kt1) of one output tile. `load`: the
+// accumulators of k-tiles [0, kt0) come from C (left there by the walker of the previous part);
+// `save`: the tile is not finished here, the raw accumulators go to C for the next part.
+struct Segment {
+    uint32_t tile, kt0, kt1, part;
+    bool load, save;
+};
+
+// i-th segment of walker `gid`. Plain schedule (split_parts <= 1): tiles gid, gid + groups, ...,
+// each whole. Split schedule: `full_rounds` whole tiles dealt out the same way, and the
+// `left_tiles` tiles of the last round cut into `split_parts` equal runs of k-tiles; part g of
+// left-over tile j belongs to walker g * left_tiles + j, which runs it after its g-th whole tile
+// (the last part: after all of them), so that part g is finished long before part g + 1 starts.
+__host__ __device__ inline bool get_segment(const GemmParams &p, uint32_t gid, uint32_t groups, uint32_t i, Segment &sg)
+{
+    const uint32_t nkt = (uint32_t)p.num_kt;
+    if (p.split_parts <= 1) {
+        sg.tile = gid + i * groups;
+        sg.kt0 = 0; sg.kt1 = nkt; sg.part = 0; sg.load = false; sg.save = false;
+        return sg.tile < (uint32_t)p.num_tiles;
+    }
+    const uint32_t left = (uint32_t)p.left_tiles, parts = (uint32_t)p.split_parts, rounds = (uint32_t)p.full_rounds;
+    const uint32_t g = gid / left;
+    const bool has_part = g < parts;
+    const uint32_t pos = g + 1 < parts ? g : rounds;
+    if (i >= rounds + (has_part ? 1u : 0u)) return false;
+    if (has_part && i == pos) {
+        sg.tile = groups * rounds + gid % left;
+        sg.kt0 = g * nkt / parts; sg.kt1 = (g + 1) * nkt / parts; sg.part = g;
+        sg.load = g > 0; sg.save = g + 1 < parts;
+        return true;
+    }
+    sg.tile = gid + ((has_part && i > pos) ? i - 1 : i) * groups;
+    sg.kt0 = 0; sg.kt1 = nkt; sg.part = 0; sg.load = false; sg.save = false;
+    return true;
+}
+
 // hand-over words one launch can use: 16 per left-over tile, fewer left-over tiles than walkers
 constexpr int SPLIT_MAX_WALKERS = 160;
 constexpr int SPLIT_SIGNAL_WORDS = SPLIT_MAX_WALKERS * 16;
@@ -76,6 +113,12 @@ inline uint32_t gemm_epoch_of(uint32_t counter) { return (counter & 0x1FFFFFFFu)
 // tm_c covers C and is used for the stores of finished tiles when p.c_vec_ok is set (otherwise its contents do
 // not matter): FP32 output: box 32 columns x 16 rows, 128-byte swizzle; 16-bit output: box 32 columns x 32 rows,
 // 64-byte swizzle.
+// Split schedule for `tiles` tiles of `num_kt` k-tiles on `walkers` tile walkers under `policy` (MPGEMMFI_SPLIT_*): fills
+// split_parts / full_rounds / left_tiles of p (split_parts 0: every tile whole). Off unless there is at least one full
+// round, the left-over tiles number at most half the walkers, every part keeps at least four k-tiles, C allows 16-byte
+// accesses and is FP32, and (policy AUTO) the launch gets visibly shorter. Host logic, no device needed.
+void choose_split_schedule(GemmParams &p, int walkers, int policy);
+
 cudaError_t launch_gemm(int bn, bool pair, const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_c,
                         const GemmParams &p, int grid, cudaStream_t stream);
 

@@ -73,3 +73,54 @@ def test_launch_slots_and_tags():
     # two launches that share a slot never share a tag unless 2^29 launches lie between them
     assert mpg.mpgemmfi_debug_launch_slot(5)[1] != mpg.mpgemmfi_debug_launch_slot(21)[1]
     assert mpg.mpgemmfi_debug_launch_slot(5)[0] == mpg.mpgemmfi_debug_launch_slot(21)[0]
+
+
+def test_tile_schedule_covers_every_k_step_once_and_orders_the_parts():
+    """The schedule the kernel's tile walkers follow, enumerated on the host for many shapes and all three policies:
+    every k-step of every tile is computed exactly once; a cut tile's parts are consecutive runs of k-steps, the first
+    starting fresh and leaving its sums, the last loading and finishing; and the walker of part g has a LOWER index than
+    the walker of part g + 1 and runs its part no later in its own order than the next walker runs the following one --
+    the order of dispatch the hand-over's bounded wait relies on."""
+    rng = np.random.default_rng(5)
+    shapes = [(256, 64, 74), (81, 9, 74), (104, 8, 74), (168, 9, 74), (156, 8, 148), (1024, 16, 74), (100, 16, 74), (75, 64, 74),
+              (73, 64, 74), (148, 3, 74), (6272, 9, 148)]
+    shapes += [(int(rng.integers(1, 700)), int(rng.integers(1, 200)), int(rng.choice([74, 148, 132, 66]))) for _ in range(60)]
+    engaged = 0
+    for num_tiles, num_kt, walkers in shapes:
+        for policy in (mpg.SPLIT_AUTO, mpg.SPLIT_OFF, mpg.SPLIT_ON):
+            seg = mpg.mpgemmfi_debug_segments(num_tiles, num_kt, walkers, policy)
+            cover = np.zeros((num_tiles, num_kt), dtype=np.int32)
+            for w, i, t, k0, k1, part, load, save in seg:
+                assert t < num_tiles and k0 < k1 <= num_kt
+                cover[t, k0:k1] += 1
+                assert bool(load) == (k0 > 0) and bool(save) == (k1 < num_kt)
+            assert (cover == 1).all(), (num_tiles, num_kt, walkers, policy)
+            # per walker: indices 0, 1, 2, ... without gaps
+            for w in np.unique(seg[:, 0]):
+                idx = seg[seg[:, 0] == w][:, 1]
+                assert list(idx) == list(range(len(idx)))
+            cut = seg[(seg[:, 6] == 1) | (seg[:, 7] == 1)]
+            if policy == mpg.SPLIT_OFF:
+                assert len(cut) == 0
+            if len(cut):
+                engaged += 1
+                for t in np.unique(cut[:, 2]):
+                    parts = cut[cut[:, 2] == t]
+                    parts = parts[np.argsort(parts[:, 5])]
+                    assert list(parts[:, 5]) == list(range(len(parts))) and 2 <= len(parts) <= 4
+                    assert parts[0, 3] == 0 and parts[-1, 4] == num_kt and (parts[1:, 3] == parts[:-1, 4]).all()
+                    assert (parts[:, 4] - parts[:, 3] >= 4).all()                  # no part shorter than four k-steps
+                    assert (parts[1:, 0] > parts[:-1, 0]).all()                     # producer has the lower walker index
+                    assert (parts[1:, 1] >= parts[:-1, 1]).all()                    # ... and runs its part no later
+                # a walker that hands a part on never waits for anybody before it: its part's predecessors are lower walkers
+                # that run theirs first
+                first = cut[cut[:, 5] == 0]
+                assert (first[:, 1] == 0).all()
+    assert engaged >= 10                          # the cut schedule did engage on a fair number of the shapes
+    # the benchmark's c2 (256 tiles of 64 k-steps on 74 pairs): 34 left-over tiles cut in two under AUTO
+    seg = mpg.mpgemmfi_debug_segments(256, 64, 74, mpg.SPLIT_AUTO)
+    assert ((seg[:, 7] == 1).sum(), (seg[:, 6] == 1).sum()) == (34, 34)
+    # c3a (1024 tiles of 16 k-steps): too short to pay, left whole
+    seg = mpg.mpgemmfi_debug_segments(1024, 16, 74, mpg.SPLIT_AUTO)
+    assert not seg[:, 6].any() and not seg[:, 7].any()
+    assert mpg.load_library().mpgemmfi_debug_segments(0, 1, 1, 0, None, 0) == -1
