@@ -69,6 +69,8 @@ struct Cfg {
     static constexpr int STAGES_FIT = (SMEM_LIMIT - CONTROL_RESERVE - OUT_STAGING_BYTES) / STAGE_BYTES;
     static constexpr int STAGES = STAGES_FIT < MAX_STAGES ? STAGES_FIT : MAX_STAGES;
     static_assert(STAGES >= 3, "operand ring too short");
+    // (the last tile's epilogue parks 4 KB per piece in the ring: 8 warps x up to 4 pieces)
+    static_assert(STAGES * STAGE_BYTES >= EPI_WARPS * 4 * 4096, "operand ring smaller than the last tile's staging");
     static constexpr int TMEM_COLS = 2 * BN;   // two accumulators; 128, 256 or 512 columns
     static_assert(BN == 64 || BN == 128 || BN == 256, "BN must be 64, 128 or 256");
     static_assert(!kPair || BN == 256, "pair tiles are 256 x 256");
@@ -888,6 +890,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 }
             }
             set_tile(sg.tile);
+            // the walker's last piece of work: when its accumulators are complete the operand ring is free (see
+            // store_piece_tail)
+            bool last_seg;
+            {
+                Segment nx;
+                last_seg = !get_segment(p, gid, groups, lt + 1, nx);
+            }
             const uint32_t tmem_acc = tmem_base + as * BN;
             bool tile_has_out = false;
             if (has_sites) {
@@ -977,6 +986,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                         tma_store_2d(&tm_c, smem_u32(my_out), (int)c0, (int)r0);
                         bulk_commit_group();
                     }
+                }
+            };
+            // The same for the walker's LAST tile. Nothing overlaps that tile's epilogue, so its latency is the launch's
+            // tail; and once its accumulators are complete (acc_full: every MMA of this CTA, or pair, has read its
+            // operands) the operand ring is free. Every piece gets 4 KB of it to itself: all 32 threads park their rows
+            // at once and both 16-row stores leave without any wait for an earlier store to have read the staging.
+            auto store_piece_tail = [&](uint32_t (&v)[32], uint32_t c0, int piece) {
+                const uint32_t buf = smem_u32(smem) + (uint32_t)(warp - 4) * (4u * 4096u) + (uint32_t)piece * 4096u;
+                const uint32_t mine = buf + (uint32_t)lane * 128u;
+#pragma unroll
+                for (int jj = 0; jj < 8; ++jj)
+                    st_shared_v4(mine + ((uint32_t)(jj ^ (lane & 7)) << 4), v[4 * jj], v[4 * jj + 1], v[4 * jj + 2], v[4 * jj + 3]);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0 && c0 < (uint32_t)p.N) {
+                    if (row0 < (uint32_t)p.M) tma_store_2d(&tm_c, buf, (int)c0, (int)row0);
+                    if (row0 + 16 < (uint32_t)p.M) tma_store_2d(&tm_c, buf + 2048u, (int)c0, (int)(row0 + 16));
+                    bulk_commit_group();
                 }
             };
             // 16-bit output: the checked FP32 values are rounded once (to nearest even) and the whole 32 x 32 piece, now
@@ -1086,6 +1113,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     }
                     if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 1);
                     if (p.out_fmt != MPGEMMFI_OUT_FP32) store_piece16(v, c0);
+                    else if (p.c_vec_ok && last_seg) store_piece_tail(v, c0, i);
                     else if (p.c_vec_ok) store_piece_tma(v, c0);
                     else store_piece(v, c0);
                     return fw;
