@@ -1008,20 +1008,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             };
             // 16-bit output: the checked FP32 values are rounded once (to nearest even) and the whole 32 x 32 piece, now
             // 64 bytes a row, fits the staging: all 32 threads park their rows at once and the piece leaves as ONE store.
-            auto store_piece16 = [&](uint32_t (&v)[32], uint32_t c0) {
+            auto store_piece16 = [&](uint32_t (&v)[32], uint32_t c0, int piece) {
                 uint32_t h[16];
 #pragma unroll
                 for (int jj = 0; jj < 16; ++jj) h[jj] = pack_out16(p.out_fmt, v[2 * jj], v[2 * jj + 1]);
                 if (p.c_vec_ok) {
-                    if (lane == 0) bulk_wait_read_all();
-                    __syncwarp();
+                    // the walker's last tile: a buffer of the free operand ring per piece, no wait (see store_piece_tail)
+                    const uint32_t buf = last_seg ? smem_u32(smem) + (uint32_t)(warp - 4) * (4u * 2048u) + (uint32_t)piece * 2048u
+                                                  : smem_u32(my_out);
+                    if (!last_seg) {
+                        if (lane == 0) bulk_wait_read_all();
+                        __syncwarp();
+                    }
+                    const uint32_t mine = buf + (park16_addr - smem_u32(my_out));
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
-                        st_shared_v4(park16_addr ^ (uint32_t)(c << 4), h[4 * c], h[4 * c + 1], h[4 * c + 2], h[4 * c + 3]);
+                        st_shared_v4(mine ^ (uint32_t)(c << 4), h[4 * c], h[4 * c + 1], h[4 * c + 2], h[4 * c + 3]);
                     fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0 && row0 < (uint32_t)p.M && c0 < (uint32_t)p.N) {
-                        tma_store_2d(&tm_c, smem_u32(my_out), (int)c0, (int)row0);
+                        tma_store_2d(&tm_c, buf, (int)c0, (int)row0);
                         bulk_commit_group();
                     }
                 } else if (row_ok) {
@@ -1112,7 +1118,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                         if (c0 + 32 > (uint32_t)p.N) fw &= c0 < (uint32_t)p.N ? (1u << ((uint32_t)p.N - c0)) - 1u : 0u;
                     }
                     if (tile_has_out && row_ok) apply_out_sites(tc, row, c0, v, 1);
-                    if (p.out_fmt != MPGEMMFI_OUT_FP32) store_piece16(v, c0);
+                    if (p.out_fmt != MPGEMMFI_OUT_FP32) store_piece16(v, c0, i);
                     else if (p.c_vec_ok && last_seg) store_piece_tail(v, c0, i);
                     else if (p.c_vec_ok) store_piece_tma(v, c0);
                     else store_piece(v, c0);
