@@ -69,8 +69,8 @@ struct Cfg {
     static constexpr int STAGES_FIT = (SMEM_LIMIT - CONTROL_RESERVE - OUT_STAGING_BYTES) / STAGE_BYTES;
     static constexpr int STAGES = STAGES_FIT < MAX_STAGES ? STAGES_FIT : MAX_STAGES;
     static_assert(STAGES >= 3, "operand ring too short");
-    // (the last tile's epilogue parks 4 KB per piece in the ring: 8 warps x up to 4 pieces)
-    static_assert(STAGES * STAGE_BYTES >= EPI_WARPS * 4 * 4096, "operand ring smaller than the last tile's staging");
+    // (the last tile's epilogue parks 4 KB per 32-column piece in the ring: 8 warps x BN / 64 pieces each)
+    static_assert(STAGES * STAGE_BYTES >= EPI_WARPS * (BN / 64) * 4096, "operand ring smaller than the last tile's staging");
     static constexpr int TMEM_COLS = 2 * BN;   // two accumulators; 128, 256 or 512 columns
     static_assert(BN == 64 || BN == 128 || BN == 256, "BN must be 64, 128 or 256");
     static_assert(!kPair || BN == 256, "pair tiles are 256 x 256");
@@ -993,7 +993,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             // operands) the operand ring is free. Every piece gets 4 KB of it to itself: all 32 threads park their rows
             // at once and both 16-row stores leave without any wait for an earlier store to have read the staging.
             auto store_piece_tail = [&](uint32_t (&v)[32], uint32_t c0, int piece) {
-                const uint32_t buf = smem_u32(smem) + (uint32_t)(warp - 4) * (4u * 4096u) + (uint32_t)piece * 4096u;
+                const uint32_t buf = smem_u32(smem) + ((uint32_t)(warp - 4) * (uint32_t)MY_PIECES + (uint32_t)piece) * 4096u;
                 const uint32_t mine = buf + (uint32_t)lane * 128u;
 #pragma unroll
                 for (int jj = 0; jj < 8; ++jj)
@@ -1014,7 +1014,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 for (int jj = 0; jj < 16; ++jj) h[jj] = pack_out16(p.out_fmt, v[2 * jj], v[2 * jj + 1]);
                 if (p.c_vec_ok) {
                     // the walker's last tile: a buffer of the free operand ring per piece, no wait (see store_piece_tail)
-                    const uint32_t buf = last_seg ? smem_u32(smem) + (uint32_t)(warp - 4) * (4u * 2048u) + (uint32_t)piece * 2048u
+                    const uint32_t buf = last_seg ? smem_u32(smem) + ((uint32_t)(warp - 4) * (uint32_t)MY_PIECES + (uint32_t)piece) * 2048u
                                                   : smem_u32(my_out);
                     if (!last_seg) {
                         if (lane == 0) bulk_wait_read_all();
