@@ -161,15 +161,19 @@ def quick_config(name, mpg, synth, torch, dev, flush, peaks, steps=40, out16=Fal
     view = np.int32 if dtype == synth.DTYPE_TF32 else np.int16
     A = torch.from_numpy(w.A.view(view)).to(dev)
     Bt = torch.from_numpy(w.Bt.view(view)).to(dev)
-    sites = torch.from_numpy(w.sites.view(np.int32).reshape(-1, 8)).to(dev)
+    host_sites = torch.from_numpy(w.sites.view(np.int32).reshape(-1, 8).copy()).pin_memory()
+    sites = host_sites.to(dev)
     C = torch.empty((M, N), dtype=torch.float16 if out16 else torch.float32, device=dev)
     flags = torch.empty(mpg.mpgemmfi_flags_bytes(M, N, 1) // 4, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream(dev)
     sh = stream.cuda_stream
     n = len(w.sites)
 
-    def step(i, inject):
-        sp, nf, md, fl = (sites.data_ptr() + 32 * (i % n), 1, mode, flags.data_ptr()) if inject else (None, 0, 0, None)
+    def step(i, kind):
+        # kind: "host" = the step's site handed over in host memory (it travels in the launch parameters),
+        # "device" = the same site read from the table in device memory, "off" = no injection, no check
+        table = host_sites if kind == "host" else sites
+        sp, nf, md, fl = (table.data_ptr() + 32 * (i % n), 1, mode, flags.data_ptr()) if kind != "off" else (None, 0, 0, None)
         if out16:
             rc = mpg.mpgemmfi_gemm_out16(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), None, mpg.OUT_FP16, C.data_ptr(), sp, nf,
                                          md, fl, sh)
@@ -178,24 +182,25 @@ def quick_config(name, mpg, synth, torch, dev, flush, peaks, steps=40, out16=Fal
         if rc != 0:
             raise mpg.MpgemmfiError(rc, "mpgemmfi_gemm")
 
+    kinds = ("host", "device", "off")
     for i in range(3):
-        for inject in (True, False):
-            flush.zero_(); step(i, inject)
+        for kind in kinds:
+            flush.zero_(); step(i, kind)
     torch.cuda.synchronize(dev)
     ev = []
     for i in range(steps):
-        for inject in (True, False):
+        for kind in kinds:
             flush.zero_()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream); step(i, inject); e1.record(stream)
-            ev.append((inject, e0, e1))
+            e0.record(stream); step(i, kind); e1.record(stream)
+            ev.append((kind, e0, e1))
     torch.cuda.synchronize(dev)
-    t_on = statistics.median(e0.elapsed_time(e1) for inj, e0, e1 in ev if inj) * 1e-3
-    t_off = statistics.median(e0.elapsed_time(e1) for inj, e0, e1 in ev if not inj) * 1e-3
+    t_on, t_dev, t_off = (statistics.median(e0.elapsed_time(e1) for k, e0, e1 in ev if k == kind) * 1e-3 for kind in kinds)
     if int(flags[0].item()) & mpg.STATUS_WAIT_LIMIT:
         raise SystemExit(f"device wait limit hit on {name}")
     flops = 2.0 * M * N * K
-    out = {"us_per_gemm": t_on * 1e6, "tflops": flops / t_on / 1e12, "injected_over_plain_time": t_on / t_off,
+    out = {"us_per_gemm": t_on * 1e6, "us_per_gemm_device_table": t_dev * 1e6, "tflops": flops / t_on / 1e12,
+           "injected_over_plain_time": t_on / t_off,
            "dtype": DTYPE_NAMES[dtype], "output": "fp16" if out16 else "fp32", "steps": steps}
     es = A.element_size()
     min_bytes = (M * K + N * K) * es + M * N * C.element_size() + M * ((N + 31) // 32) * 4
@@ -314,9 +319,12 @@ def main():
     n_my = len(my_sites)
     flops = 2.0 * M * N * K
 
+    # the step's one site is handed over in (pinned) host memory: it travels in the launch parameters
+    sites_host = torch.from_numpy(my_sites.view(np.int32).reshape(-1, 8).copy()).pin_memory()
+
     def gemm_step(i, inject=True):
         if inject:
-            sp = sites_dev.data_ptr() + 32 * (i % n_my)
+            sp = sites_host.data_ptr() + 32 * (i % n_my)
             rc = mpg.mpgemmfi_gemm(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), C.data_ptr(), sp, 1, mode,
                                    flags.data_ptr(), sh)
         else:
@@ -440,16 +448,14 @@ def main():
     # ---- end to end: pinned host buffers, copies inside the timed region
     hA = torch.from_numpy(w.A.view(view)).pin_memory()
     hB = torch.from_numpy(w.Bt.view(view)).pin_memory()
-    hS = torch.from_numpy(my_sites.view(np.int32).reshape(-1, 8)).pin_memory()
+    hS = sites_host
     hC = torch.empty((M, N), dtype=torch.float32).pin_memory()
     hF = torch.empty(flags.numel(), dtype=torch.int32).pin_memory()
-    site1 = torch.empty((1, 8), dtype=torch.int32, device=dev)
 
     def e2e_step(i):
         A.copy_(hA, non_blocking=True)
         Bt.copy_(hB, non_blocking=True)
-        site1.copy_(hS[i % n_my:i % n_my + 1], non_blocking=True)
-        rc = mpg.mpgemmfi_gemm(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), C.data_ptr(), site1.data_ptr(), 1, mode,
+        rc = mpg.mpgemmfi_gemm(dtype, M, N, K, A.data_ptr(), Bt.data_ptr(), C.data_ptr(), hS.data_ptr() + 32 * (i % n_my), 1, mode,
                                flags.data_ptr(), sh)
         if rc != 0:
             raise mpg.MpgemmfiError(rc, "mpgemmfi_gemm")
@@ -466,21 +472,21 @@ def main():
     # the previous step's result (the link is full duplex). Every step still copies all of its inputs up and all of its
     # results down; timed from an event before the first step to an event after the last copy of both streams.
     streams2 = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
-    dbuf = [(A, Bt, C, flags, site1, hC, hF)]
-    dbuf.append((torch.empty_like(A), torch.empty_like(Bt), torch.empty_like(C), torch.empty_like(flags), torch.empty_like(site1),
+    dbuf = [(A, Bt, C, flags, hC, hF)]
+    dbuf.append((torch.empty_like(A), torch.empty_like(Bt), torch.empty_like(C), torch.empty_like(flags),
                  torch.empty((M, N), dtype=torch.float32).pin_memory(), torch.empty(flags.numel(), dtype=torch.int32).pin_memory()))
     flush2 = [flush, torch.empty_like(flush)]
 
     def e2e_pipelined(n_steps, first):
         for i in range(n_steps):
             k = i % 2
-            dA, dB, dC, dF, dS, oC, oF = dbuf[k]
+            dA, dB, dC, dF, oC, oF = dbuf[k]
             with torch.cuda.stream(streams2[k]):
                 flush2[k].zero_()
                 dA.copy_(hA, non_blocking=True)
                 dB.copy_(hB, non_blocking=True)
-                dS.copy_(hS[(first + i) % n_my:(first + i) % n_my + 1], non_blocking=True)
-                rc = mpg.mpgemmfi_gemm(dtype, M, N, K, dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), dS.data_ptr(), 1, mode,
+                rc = mpg.mpgemmfi_gemm(dtype, M, N, K, dA.data_ptr(), dB.data_ptr(), dC.data_ptr(),
+                                       hS.data_ptr() + 32 * ((first + i) % n_my), 1, mode,
                                        dF.data_ptr(), streams2[k].cuda_stream)
                 if rc != 0:
                     raise mpg.MpgemmfiError(rc, "mpgemmfi_gemm")
@@ -505,9 +511,9 @@ def main():
     torch.cuda.synchronize(dev)
     ms_e2e_pipe = reduce_max(ev0.elapsed_time(ev1), world, dev)
     e2e_value = reduce_sum(flops * e2e_steps, world, dev) / (ms_e2e_pipe * 1e-3) / 1e12
-    if int(dbuf[1][6][0].item()) & mpg.STATUS_WAIT_LIMIT:
+    if int(dbuf[1][5][0].item()) & mpg.STATUS_WAIT_LIMIT:
         raise SystemExit("device wait limit hit during the end-to-end steps")
-    h2d = hA.numel() * hA.element_size() + hB.numel() * hB.element_size() + 32
+    h2d = hA.numel() * hA.element_size() + hB.numel() * hB.element_size()      # (the 32-byte site rides in the launch)
     d2h = hC.numel() * 4 + hF.numel() * 4
 
     peaks, peak_src = load_peaks()
@@ -585,6 +591,8 @@ def main():
                        "timing": "sum of per-step CUDA-event intervals on the launching stream",
                        "clocks_sampling": "nvidia-smi every 20 ms over the timed steps, continued over identical untimed "
                                           "steps until 0.4 s of load have been seen",
+                       "site_table": "the step's site is handed over in host memory and travels in the kernel's launch "
+                                     "parameters (all_configs.*.us_per_gemm_device_table: the same read from device memory)",
                        "trials_per_rank": n_my},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

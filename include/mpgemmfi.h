@@ -146,6 +146,7 @@ enum {
 };
 
 #define MPGEMMFI_MAX_FAULTS 4096      /* sites per mpgemmfi_gemm call */
+#define MPGEMMFI_INLINE_FAULTS 8      /* sites a table in HOST memory may hold (it travels in the launch parameters) */
 #define MPGEMMFI_HEADER_WORDS 16
 
 /* status word of the flags header */
@@ -212,6 +213,14 @@ typedef struct {
  *   A, Bt, C     device pointers, layouts above; C is written in full.
  *   fault_sites  device pointer to n_faults entries (may be NULL when n_faults = 0);
  *                0 <= n_faults <= MPGEMMFI_MAX_FAULTS.
+ *                Alternatively a pointer to ordinary or pinned HOST memory holding at most
+ *                MPGEMMFI_INLINE_FAULTS entries (the single fault of one trial, Section IV-A): the
+ *                entries are copied during the call and travel in the kernel's launch parameters,
+ *                so the caller may reuse the memory at once and the kernel reads no table from
+ *                device memory (a table that is cold in the caches delays every CTA's start by
+ *                a few microseconds). Which kind a pointer is, is asked of the CUDA runtime;
+ *                managed memory counts as device memory. A host table with more entries: ERR_ARG.
+ *                Results are identical either way. The same holds for every mpgemmfi_gemm_* below.
  *   flags_out    device pointer to mpgemmfi_flags_bytes(M, N, n_faults) bytes, 16-byte
  *                aligned, written in full; may be NULL only when n_faults = 0 and the
  *                technique is NONE (plain GEMM, nothing to report).

@@ -9,7 +9,7 @@ from .binding import (  # noqa: F401
     FP16, BF16, TF32,
     SITE_A, SITE_B, SITE_ACC, SITE_OUT, SITE_TERM,
     DETECT_NONE, DETECT_BOUNDCHECK, DETECT_RANGE_MAX, DETECT_RANGE_FLIP, CORRECT, TERM_HMMA_STEP, OUTPUT_RANGE, TERM_IN_FORMAT,
-    STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT, MAX_FAULTS, HEADER_WORDS, STATIC_MAX_TRIALS,
+    STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT, MAX_FAULTS, INLINE_FAULTS, HEADER_WORDS, STATIC_MAX_TRIALS,
     TILES_AUTO, TILES_SINGLE, TILES_PAIR, mpgemmfi_set_tile_policy,
     SPLIT_AUTO, SPLIT_OFF, SPLIT_ON, mpgemmfi_set_split_policy,
     SITE_DTYPE, SITE_LOG_DTYPE, RECORD_DTYPE, SUMMARY_DTYPE,

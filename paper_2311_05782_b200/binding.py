@@ -22,6 +22,7 @@ OUTPUT_RANGE = 64
 TERM_IN_FORMAT = 128
 STATUS_SITE_SKIPPED, STATUS_WAIT_LIMIT = 1, 2
 MAX_FAULTS = 4096
+INLINE_FAULTS = 8
 STATIC_MAX_TRIALS = 65536
 TILES_AUTO, TILES_SINGLE, TILES_PAIR = 0, 1, 2
 SPLIT_AUTO, SPLIT_OFF, SPLIT_ON = 0, 1, 2
@@ -277,8 +278,20 @@ def _check_operand(t, dtype, name):
         raise ValueError(f"{name}: expected a contiguous 2-D CUDA tensor of dtype in {ok} (storage {want})")
 
 
-def _sites_tensor(sites, device):
-    """numpy structured array (or None) -> int32 CUDA tensor [n, 8]; tensors pass through."""
+class _HostSites:
+    """A small site table kept in host memory (it travels in the launch parameters); quacks like a tensor here."""
+
+    def __init__(self, arr):
+        self.arr = arr
+
+    def data_ptr(self):
+        return self.arr.ctypes.data
+
+
+def _sites_tensor(sites, device, inline=True):
+    """numpy structured array (or None) -> the table to pass and its length. Up to INLINE_FAULTS entries stay in
+    host memory (inline=False: copied to the device like a longer table); a longer table becomes an int32 CUDA
+    tensor [n, 8]; CUDA tensors pass through."""
     torch = _torch()
     if sites is None:
         return None, 0
@@ -287,6 +300,12 @@ def _sites_tensor(sites, device):
         assert s.dtype.itemsize == 32
         if len(s) == 0:
             return None, 0
+        if inline and len(s) <= INLINE_FAULTS:
+            host = np.empty(len(s) * 8 + 4, dtype=np.int32)          # room to start on a 16-byte boundary
+            off = (-host.ctypes.data % 16) // 4
+            host = host[off:off + len(s) * 8]
+            host[:] = s.view(np.int32).reshape(-1)
+            return _HostSites(host), len(s)
         t = torch.from_numpy(s.view(np.int32).reshape(len(s), 8)).to(device)
         return t, len(s)
     assert sites.is_cuda and sites.is_contiguous() and sites.dtype == torch.int32 and sites.shape[-1] == 8
@@ -294,11 +313,13 @@ def _sites_tensor(sites, device):
 
 
 def gemm(dtype, A, Bt, sites=None, detect_mode=DETECT_NONE, C_out=None, flags_out=None, stream=None, addend=None,
-         out_format=OUT_FP32):
+         out_format=OUT_FP32, inline_sites=True):
     """Fault-injected GEMM on CUDA tensors. Returns (C, flags) where flags is the raw uint32 buffer
     (as an int32 tensor) laid out as documented in include/mpgemmfi.h; see split_flags().
     addend: optional M x N float32 CUDA tensor, the C_in of D = A x B + C_in (it may be C_out itself).
-    out_format: OUT_FP16 / OUT_BF16 give an M x N float16 / bfloat16 result (mpgemmfi_gemm_out16)."""
+    out_format: OUT_FP16 / OUT_BF16 give an M x N float16 / bfloat16 result (mpgemmfi_gemm_out16).
+    sites: numpy structured array (up to INLINE_FAULTS entries are handed over in host memory unless
+    inline_sites=False; more are copied to the device) or an int32 CUDA tensor [n, 8]."""
     torch = _torch()
     _check_operand(A, dtype, "A")
     _check_operand(Bt, dtype, "Bt")
@@ -306,7 +327,7 @@ def gemm(dtype, A, Bt, sites=None, detect_mode=DETECT_NONE, C_out=None, flags_ou
     N, K2 = Bt.shape
     if K != K2:
         raise ValueError("A and Bt disagree on K")
-    st, n_faults = _sites_tensor(sites, A.device)
+    st, n_faults = _sites_tensor(sites, A.device, inline_sites)
     out_dtype = {OUT_FP32: torch.float32, OUT_FP16: torch.float16, OUT_BF16: torch.bfloat16}[out_format]
     if C_out is None:
         C_out = torch.empty((M, N), dtype=out_dtype, device=A.device)
@@ -376,7 +397,7 @@ def campaign(dtype, A, Bt, sites, detect_mode=DETECT_NONE, C_clean=None, records
     _check_operand(Bt, dtype, "Bt")
     M, K = A.shape
     N, _ = Bt.shape
-    st, n_trials = _sites_tensor(sites, A.device)
+    st, n_trials = _sites_tensor(sites, A.device, inline=False)      # the campaign reads its table on the device
     if C_clean is None:
         C_clean = torch.empty((M, N), dtype=torch.float32, device=A.device)
     if records is None:

@@ -234,6 +234,20 @@ int run_gemm(int dtype, int M, int N, int K, const void *A, const void *Bt, void
         if (rc) return rc;
     }
     p.A = A; p.Bt = Bt; p.C = static_cast<float *>(C); p.sites = sites; p.flags = flags;
+    p.sites_inline = 0;
+    memset(p.inline_sites, 0, sizeof(p.inline_sites));
+    if (n_faults > 0) {
+        // a table in host memory rides in the launch parameters
+        cudaPointerAttributes at;
+        const cudaError_t ea = cudaPointerGetAttributes(&at, sites);
+        if (ea != cudaSuccess) return cuda_fail(ea);
+        if (at.type == cudaMemoryTypeUnregistered || at.type == cudaMemoryTypeHost) {
+            if (n_faults > mpg::GEMM_INLINE_SITES) return MPGEMMFI_ERR_ARG;
+            memcpy(p.inline_sites, sites, (size_t)n_faults * sizeof(mpgemmfi_site));
+            p.sites_inline = 1;
+            p.sites = nullptr;
+        }
+    }
     p.exp_a = exp_a; p.exp_b = exp_bt;
     p.addend = addend;
     p.addend_vec_ok = (N % 4 == 0) && (((uintptr_t)addend & 15) == 0);

@@ -53,6 +53,7 @@ constexpr int BM = 128;
 constexpr int NUM_THREADS = 384;     // 4 control warps + 8 epilogue warps
 constexpr int EPI_WARPS = 8;
 constexpr int SITE_CACHE = 64;
+constexpr int SINGLE_SITE_WARP = 3;       // the warp with no other role, see build_site_list
 constexpr int MAX_STAGES = 8;
 constexpr int OUT_BUF_BYTES = 16 * 128;                    // staging of one epilogue warp: 16 rows x 128 bytes
 constexpr int OUT_STAGING_BYTES = EPI_WARPS * OUT_BUF_BYTES;
@@ -110,11 +111,18 @@ __device__ __forceinline__ bool in_tile_rows(const TileCtx &c, uint32_t row) { r
 __device__ __forceinline__ bool in_tile_cols(const TileCtx &c, uint32_t col) { return col - c.n0 < c.bn; }
 __device__ __forceinline__ bool in_own_b(const TileCtx &c, uint32_t col) { return col - c.b0 < c.b_rows; }
 
+// entry i of the site table: from the launch parameters when the table travels there, else from device memory
+__device__ __forceinline__ mpgemmfi_site table_site(const GemmParams &p, int i)
+{
+    if (p.sites_inline) return p.inline_sites[i & (GEMM_INLINE_SITES - 1)];
+    return load_site(p.sites, i);
+}
+
 // entry i of the CTA's site list: from shared memory for the first SITE_CACHE entries
 __device__ __forceinline__ mpgemmfi_site listed_site(const TileCtx &c, uint32_t i)
 {
     if (i < (uint32_t)SITE_CACHE) return c.ctl->site_cache[i];
-    return load_site(c.p->sites, c.ctl->site_idx[i]);
+    return table_site(*c.p, c.ctl->site_idx[i]);
 }
 
 // smallest k-tile >= kt_from in which this tile has an operand site (warp-wide)
@@ -365,6 +373,27 @@ __device__ bool site_touches_group(const mpgemmfi_site &s, const GemmParams &p, 
     return walker_has_tile(p, tile_number(p, s.row / TM, s.col / BN), gid, groups);
 }
 
+// The same question asked by a whole warp about ONE site (the same `s` in every lane): the tiles of an operand
+// site's row / column of tiles are shared out over the lanes, 32 per round, and a round with a hit ends the search.
+// (One thread alone runs a division chain per tile: 3 us for the 16 tiles of a 4096-wide row, far more for the
+// thousands of tile rows of a tall matrix.)
+template <int TM, int BN>
+__device__ bool site_touches_group_warp(const mpgemmfi_site &s, const GemmParams &p, uint32_t gid, uint32_t groups, int lane)
+{
+    if (s.kind == MPGEMMFI_SITE_A || s.kind == MPGEMMFI_SITE_B) {
+        const bool is_a = s.kind == MPGEMMFI_SITE_A;
+        const uint32_t fixed = is_a ? s.row / TM : s.col / BN;
+        const uint32_t count = is_a ? (uint32_t)p.tiles_n : (uint32_t)p.tiles_m;
+        for (uint32_t base = 0; base < count; base += 32) {
+            const uint32_t i = base + (uint32_t)lane;
+            const bool hit = i < count && walker_has_tile(p, is_a ? tile_number(p, fixed, i) : tile_number(p, i, fixed), gid, groups);
+            if (__any_sync(0xFFFFFFFFu, hit)) return true;
+        }
+        return false;
+    }
+    return walker_has_tile(p, tile_number(p, s.row / TM, s.col / BN), gid, groups);
+}
+
 // Hand-over of a tile part between walkers: one word per epilogue warp of the walker.
 __device__ __forceinline__ void signal_store_release(uint32_t *ptr, uint32_t v)
 {
@@ -481,9 +510,12 @@ __device__ __forceinline__ SiteSlice site_slice(int n, int warp)
 // reports invalid entries (skipped) and the applied count. Each warp compacts a contiguous slice
 // of the table with ballots, so the list keeps table order. `first` is the entry this thread
 // examines in its slice's first round, loaded by the caller ahead of time.
+// A table of one entry -- the single fault of a trial (Section IV-A), the usual case -- is handled by warp
+// SINGLE_SITE_WARP alone (every lane holds the entry in `first`), with no compaction and no CTA-wide barrier, next
+// to the other warps' set-up; it also waits for CTA 0's cleared log where this CTA will write to it.
 template <int TM, int BN>
 __device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid, uint32_t groups,
-                                const mpgemmfi_site &first)
+                                const mpgemmfi_site &first, uint64_t wait_ns)
 {
     constexpr int WARPS = NUM_THREADS / 32;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -492,13 +524,32 @@ __device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid,
         if (tid == 0) ctl->site_count = 0;
         return;
     }
+    if (n == 1) {
+        if (warp != SINGLE_SITE_WARP) return;
+        const bool ok = site_valid(first, p.dtype, p.M, p.N, p.K);
+        const bool mine = ok && site_touches_group_warp<TM, BN>(first, p, gid, groups, lane);
+        if (lane == 0) {
+            ctl->site_count = mine ? 1u : 0u;
+            if (mine) { ctl->site_cache[0] = first; ctl->site_idx[0] = 0; }
+            if (blockIdx.x == 0) {
+                if (!ok) write_log(p, 0, 0u, 0u, 0u, 2u);
+                if (p.flags) {
+                    if (ok) atomicAdd(&p.flags[3], 1u);
+                    else { atomicAdd(&p.flags[4], 1u); atomicOr(&p.flags[0], MPGEMMFI_STATUS_SITE_SKIPPED); }
+                }
+            } else if (mine && p.flags) {
+                signal_wait(p.ready, p.epoch, &ctl->abort_flag, wait_ns);
+            }
+        }
+        return;
+    }
     const SiteSlice sl = site_slice(n, warp);
     uint32_t cnt = 0, n_valid = 0, n_bad = 0, first_vote = 0;
     for (int base = sl.beg; base < sl.end; base += 32) {
         const int i = base + lane;
         bool ok = false, mine = false;
         if (i < sl.end) {
-            const mpgemmfi_site s = base == sl.beg ? first : load_site(p.sites, i);
+            const mpgemmfi_site s = base == sl.beg ? first : table_site(p, i);
             ok = site_valid(s, p.dtype, p.M, p.N, p.K);
             mine = ok && site_touches_group<TM, BN>(s, p, gid, groups);
             if (!ok && blockIdx.x == 0) write_log(p, i, 0u, 0u, 0u, 2u);
@@ -531,7 +582,7 @@ __device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid,
         uint32_t vote = first_vote;
         if (base != sl.beg) {
             if (i < sl.end) {
-                s = load_site(p.sites, i);
+                s = table_site(p, i);
                 mine = site_valid(s, p.dtype, p.M, p.N, p.K) && site_touches_group<TM, BN>(s, p, gid, groups);
             }
             vote = __ballot_sync(0xFFFFFFFFu, mine);
@@ -564,7 +615,7 @@ __device__ __forceinline__ uint32_t pack_out16(int out_fmt, uint32_t lo_bits, ui
 template <int BN, bool kTF32, bool kPair>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-            const __grid_constant__ CUtensorMap tm_c, const GemmParams p)
+            const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ GemmParams p)
 {
     using C = Cfg<BN, kPair>;
     constexpr int KT = kTF32 ? 32 : 64;      // elements per 128-byte row
@@ -587,10 +638,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
 
     // this thread's first entry of the site table: requested now, needed only after the set-up below
     mpgemmfi_site first_site = {};
-    if (p.n_faults > 0) {
+    if (p.n_faults == 1) {
+        if (warp == SINGLE_SITE_WARP) first_site = table_site(p, 0);
+    } else if (p.n_faults > 0) {
         const SiteSlice sl = site_slice(p.n_faults, warp);
-        if (sl.beg + lane < sl.end) first_site = load_site(p.sites, sl.beg + lane);
+        if (sl.beg + lane < sl.end) first_site = table_site(p, sl.beg + lane);
     }
+    // (set by the thread that may be the first to poll it, see build_site_list; everybody else meets it after a barrier)
+    if (threadIdx.x == SINGLE_SITE_WARP * 32) ctl->abort_flag = 0;
 
     if (blockIdx.x == 0 && p.flags) {
         // header and site log start at zero: cleared here rather than by a memset in front of every launch
@@ -609,7 +664,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         mbar_init(smem_u32(&ctl->pause_full), 1);
         mbar_init(smem_u32(&ctl->pause_done), EPI_ARRIVALS);
         for (int s = 0; s < 2; ++s) mbar_init(smem_u32(&ctl->acc_loaded[s]), EPI_ARRIVALS);
-        ctl->abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tm_a);
         tma_prefetch_desc(&tm_b);
@@ -619,9 +673,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         if constexpr (kPair) { tmem_alloc_pair(smem_u32(&ctl->tmem_base), C::TMEM_COLS); tmem_relinquish_pair(); }
         else { tmem_alloc(smem_u32(&ctl->tmem_base), C::TMEM_COLS); tmem_relinquish(); }
     }
-    build_site_list<TM, BN>(p, ctl, gid, groups, first_site);
+    build_site_list<TM, BN>(p, ctl, gid, groups, first_site, wait_ns);
     // a CTA with sites writes log entries as it goes: not before CTA 0 has cleared the log
-    if (threadIdx.x == 0 && blockIdx.x != 0 && p.flags && ctl->site_count != 0) signal_wait(p.ready, p.epoch, abort_flag, wait_ns);
+    // (a one-entry table: waited for inside build_site_list)
+    if (threadIdx.x == 0 && blockIdx.x != 0 && p.flags && p.n_faults > 1 && ctl->site_count != 0)
+        signal_wait(p.ready, p.epoch, abort_flag, wait_ns);
     tc_fence_before_sync();
     if constexpr (kPair) cluster_sync_all(); else __syncthreads();
     tc_fence_after_sync();

@@ -9,6 +9,9 @@
 
 namespace mpg {
 
+// a site table of at most this many entries may travel in the launch parameters instead of device memory
+constexpr int GEMM_INLINE_SITES = MPGEMMFI_INLINE_FAULTS;
+
 struct GemmParams {
     int dtype, M, N, K;
     int detect_mode, n_faults;
@@ -20,7 +23,11 @@ struct GemmParams {
     const void *A;
     const void *Bt;
     float *C;
-    const mpgemmfi_site *sites;
+    const mpgemmfi_site *sites;     // the table in device memory; unused when sites_inline is set
+    // The table given by value (n_faults <= GEMM_INLINE_SITES): the kernel then reads it from its parameters and
+    // never waits for a (cold) line of device memory before its first operand copy.
+    int sites_inline;
+    mpgemmfi_site inline_sites[GEMM_INLINE_SITES];
     uint32_t *flags;
     // output-level range check (null when not requested): row exponent maxima of A and Bt, ceil(log2 K)
     const uint32_t *exp_a;

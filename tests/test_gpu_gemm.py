@@ -215,6 +215,50 @@ def test_config_tables_in_one_gemm(name, shape, trials):
     check_gemm_against_oracle(w.dtype, w.A, w.Bt, w.sites, w.detect_mode, max_fragile=1)
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_host_table_in_the_launch_parameters_equals_the_device_table(dtype):
+    """A table of up to INLINE_FAULTS entries in host memory travels in the launch parameters; the same table in
+    device memory gives the same C and the same flags buffer bit for bit, on every entry point. The host-table
+    results are also checked against the oracle (every other test that passes a short numpy table goes that way)."""
+    kt = synth.kstep(dtype)
+    M, N, K = 520, 392, 5 * kt
+    A, Bt = rand_operands(dtype, M, N, K, 23)
+    hi = 31 if dtype == orc.TF32 else 15
+    full = np.concatenate([
+        site(orc.KIND_A, 300, 0, 2 * kt + 1, 1 << (hi - 1)), site(orc.KIND_B, 0, 391, 7, 1 << (hi - 2)),
+        site(orc.KIND_ACC, 519, 3, 3 * kt, 1 << 30), site(orc.KIND_TERM, 128, 256, 4 * kt + 3, 1 << 29),
+        site(orc.KIND_OUT, 0, 0, 0, 1 << 30), site(orc.KIND_OUT, 9999, 0, 0, 1),      # the last one is out of range
+        site(orc.KIND_OUT, 257, 131, 0, 1 << 27), site(orc.KIND_A, 300, 0, 2 * kt + 1, 1 << (hi - 3))])
+    assert len(full) == mpg.INLINE_FAULTS
+    a, b = to_dev(A, dtype), to_dev(Bt, dtype)
+    cin = torch.from_numpy(np.random.default_rng(24).standard_normal((M, N)).astype(np.float32)).cuda()
+    for n in (1, 5, 8):
+        sites = full[:n]
+        for mode in (orc.T_BOUND | orc.CORRECT, orc.T_RMAX):
+            check_gemm_against_oracle(dtype, A, Bt, sites, mode, max_fragile=1)
+            for kw in ({}, {"addend": cin}, {"out_format": mpg.OUT_BF16}):
+                c_h, f_h = mpg.gemm(dtype, a, b, sites, mode, inline_sites=True, **kw)
+                c_d, f_d = mpg.gemm(dtype, a, b, sites, mode, inline_sites=False, **kw)
+                torch.cuda.synchronize()
+                fh, fd = f_h.cpu().numpy(), f_d.cpu().numpy()
+                assert np.array_equal(fh, fd), (n, mode, kw.keys(), np.nonzero(fh != fd)[0][:8])
+                assert torch.equal(c_h.view(torch.int32 if c_h.dtype == torch.float32 else torch.int16),
+                                   c_d.view(torch.int32 if c_d.dtype == torch.float32 else torch.int16))
+                if n >= 6:
+                    assert fh.view(np.uint32)[4] == 1          # the out-of-range entry was skipped, not applied
+    # a host table beyond the limit is refused before anything is launched
+    long = np.ascontiguousarray(np.concatenate([full, full[:1]]))
+    c = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    f = torch.empty(mpg.mpgemmfi_flags_bytes(M, N, len(long)) // 4, dtype=torch.int32, device="cuda")
+    host = np.zeros(len(long) * 8 + 4, dtype=np.int32)
+    off = (-host.ctypes.data % 16) // 4
+    host[off:off + len(long) * 8] = long.view(np.int32).reshape(-1)
+    rc = mpg.mpgemmfi_gemm(dtype, M, N, K, a.data_ptr(), b.data_ptr(), c.data_ptr(), host.ctypes.data + 4 * off, len(long),
+                           orc.T_BOUND, f.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    assert rc == -1
+    torch.cuda.synchronize()
+
+
 def test_maximum_site_count():
     w = synth.make_workload("c5", 1024, 64, 192, trials=mpg.MAX_FAULTS, mix="out")
     check_gemm_against_oracle(w.dtype, w.A, w.Bt, w.sites, w.detect_mode, max_fragile=2)
