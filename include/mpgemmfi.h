@@ -432,6 +432,14 @@ int mpgemmfi_set_wait_limit_ms(int ms);
 int mpgemmfi_debug_break_handover(int on);
 
 /*
+ * Measurement aid (no counterpart in the paper): queues a kernel of one thread that does nothing on
+ * `stream`. Timed like a GEMM (event, launch, event) it gives what launching and completing any kernel
+ * costs on the system by itself -- several microseconds, which is most of the time of a GEMM of one
+ * wave of tiles and a few percent of a 4096^3 one. Errors: ERR_CUDA.
+ */
+int mpgemmfi_null_launch(mpgemmfi_stream stream);
+
+/*
  * Host logic of the launch slots (no device needed): returns the slot (0..15) that the launch with
  * counter value `counter` uses and stores its tag (29 bits, never 0) in *tag (if non-NULL).
  */

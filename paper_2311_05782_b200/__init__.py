@@ -20,6 +20,6 @@ from .binding import (  # noqa: F401
     gemm, campaign, split_flags, mpgemmfi_campaign_summary, campaign_summary,
     mpgemmfi_operand_exponents, mpgemmfi_gemm_ranged, mpgemmfi_gemm_addend,
     mpgemmfi_set_wait_limit_ms, mpgemmfi_debug_break_handover, mpgemmfi_debug_launch_slot,
-    mpgemmfi_gemm_out16, OUT_FP32, OUT_FP16, OUT_BF16, mpgemmfi_debug_segments,
+    mpgemmfi_gemm_out16, OUT_FP32, OUT_FP16, OUT_BF16, mpgemmfi_debug_segments, mpgemmfi_null_launch,
 )
 from .sharding import campaign_sharded, shard_range  # noqa: F401,E402

@@ -49,7 +49,7 @@ _SYMBOLS = [
     "mpgemmfi_strerror", "mpgemmfi_last_cuda_error", "mpgemmfi_version", "mpgemmfi_campaign_static",
     "mpgemmfi_set_tile_policy", "mpgemmfi_set_split_policy", "mpgemmfi_campaign_summary", "mpgemmfi_operand_exponents", "mpgemmfi_gemm_ranged",
     "mpgemmfi_gemm_addend", "mpgemmfi_set_wait_limit_ms", "mpgemmfi_debug_break_handover", "mpgemmfi_debug_launch_slot",
-    "mpgemmfi_gemm_out16", "mpgemmfi_debug_segments",
+    "mpgemmfi_gemm_out16", "mpgemmfi_debug_segments", "mpgemmfi_null_launch",
 ]
 
 
@@ -102,6 +102,8 @@ def load_library():
     L.mpgemmfi_set_split_policy.argtypes = [i]
     L.mpgemmfi_set_wait_limit_ms.restype = i
     L.mpgemmfi_set_wait_limit_ms.argtypes = [i]
+    L.mpgemmfi_null_launch.restype = i
+    L.mpgemmfi_null_launch.argtypes = [vp]
     L.mpgemmfi_debug_break_handover.restype = i
     L.mpgemmfi_debug_break_handover.argtypes = [i]
     L.mpgemmfi_debug_launch_slot.restype = i
@@ -199,6 +201,11 @@ def mpgemmfi_set_split_policy(policy):
 def mpgemmfi_set_wait_limit_ms(ms):
     """How long a device-side wait of the GEMM kernel may last before the launch gives up (1..60000 ms, default 4000)."""
     return load_library().mpgemmfi_set_wait_limit_ms(ms)
+
+
+def mpgemmfi_null_launch(stream):
+    """Queue a kernel that does nothing (what a launch costs by itself when timed like a GEMM)."""
+    return load_library().mpgemmfi_null_launch(stream)
 
 
 def mpgemmfi_debug_break_handover(on):

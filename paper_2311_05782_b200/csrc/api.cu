@@ -483,6 +483,12 @@ int mpgemmfi_debug_break_handover(int on)
     return MPGEMMFI_OK;
 }
 
+int mpgemmfi_null_launch(mpgemmfi_stream stream)
+{
+    const cudaError_t e = mpg::launch_null(static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? MPGEMMFI_OK : cuda_fail(e);
+}
+
 int mpgemmfi_debug_launch_slot(uint32_t counter, uint32_t *epoch)
 {
     if (epoch) *epoch = mpg::gemm_epoch_of(counter);

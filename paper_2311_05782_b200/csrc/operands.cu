@@ -38,7 +38,15 @@ __global__ void __launch_bounds__(256) exponent_max_kernel(int dtype, int rows, 
     }
 }
 
+__global__ void null_kernel() {}
+
 }  // namespace
+
+cudaError_t launch_null(cudaStream_t stream)
+{
+    null_kernel<<<1, 1, 0, stream>>>();
+    return cudaGetLastError();
+}
 
 cudaError_t launch_operand_exponents(int dtype, int rows, int K, const void *X, uint32_t *out, int num_sms,
                                      cudaStream_t stream)

@@ -10,4 +10,7 @@ namespace mpg {
 cudaError_t launch_operand_exponents(int dtype, int rows, int K, const void *X, uint32_t *out, int num_sms,
                                      cudaStream_t stream);
 
+// a kernel of one thread that does nothing (what a launch costs by itself)
+cudaError_t launch_null(cudaStream_t stream);
+
 }  // namespace mpg
