@@ -90,7 +90,11 @@ struct alignas(16) Control {
     uint32_t abort_flag;
     uint32_t site_count;
     uint32_t pad;
-    uint32_t scan[NUM_THREADS / 32];
+    // The CTA's list holds its sites by class, each class in table order: operand sites (A, B) in
+    // [0, class_end[0]), accumulator and term sites in [class_end[0], class_end[1]), output sites in
+    // [class_end[1], site_count): every role walks only the entries it can do something with.
+    uint32_t class_end[2];
+    uint32_t scan[3][NUM_THREADS / 32];
     uint16_t site_idx[MPGEMMFI_MAX_FAULTS];
     mpgemmfi_site site_cache[SITE_CACHE];     // the first entries of the CTA's list, so that scans stay on chip
 };
@@ -118,6 +122,12 @@ __device__ __forceinline__ mpgemmfi_site table_site(const GemmParams &p, int i)
     return load_site(p.sites, i);
 }
 
+// class of a site kind in the CTA's list (see Control::class_end)
+__device__ __forceinline__ int site_class(uint32_t kind)
+{
+    return (kind == MPGEMMFI_SITE_A || kind == MPGEMMFI_SITE_B) ? 0 : (kind == MPGEMMFI_SITE_OUT ? 2 : 1);
+}
+
 // entry i of the CTA's site list: from shared memory for the first SITE_CACHE entries
 __device__ __forceinline__ mpgemmfi_site listed_site(const TileCtx &c, uint32_t i)
 {
@@ -136,7 +146,7 @@ __device__ uint32_t scan_next_operand(const TileCtx &c, uint32_t kt_from, int la
         return (hit && (s.k >> sh) >= kt_from) ? s.k >> sh : NONE;
     }
     uint32_t best = NONE;
-    for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
+    for (uint32_t i = lane; i < c.ctl->class_end[0]; i += 32) {
         const mpgemmfi_site s = listed_site(c, i);
         const bool hit = (s.kind == MPGEMMFI_SITE_A && in_own_rows(c, s.row)) ||
                          (s.kind == MPGEMMFI_SITE_B && in_own_b(c, s.col));
@@ -157,7 +167,7 @@ __device__ uint32_t scan_next_boundary(const TileCtx &c, uint32_t b_from, int la
         return NONE;
     }
     uint32_t best = NONE;
-    for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
+    for (uint32_t i = c.ctl->class_end[0] + (uint32_t)lane; i < c.ctl->class_end[1]; i += 32) {
         const mpgemmfi_site s = listed_site(c, i);
         if ((s.kind == MPGEMMFI_SITE_ACC || s.kind == MPGEMMFI_SITE_TERM) && in_tile_rows(c, s.row) &&
             in_tile_cols(c, s.col)) {
@@ -175,7 +185,7 @@ __device__ bool scan_has_out(const TileCtx &c, int lane)
         return s.kind == MPGEMMFI_SITE_OUT && in_own_rows(c, s.row) && in_tile_cols(c, s.col);
     }
     bool any = false;
-    for (uint32_t i = lane; i < c.ctl->site_count; i += 32) {
+    for (uint32_t i = c.ctl->class_end[1] + (uint32_t)lane; i < c.ctl->site_count; i += 32) {
         const mpgemmfi_site s = listed_site(c, i);
         any |= s.kind == MPGEMMFI_SITE_OUT && in_own_rows(c, s.row) && in_tile_cols(c, s.col);
     }
@@ -200,36 +210,89 @@ __device__ __forceinline__ uint32_t swizzled_offset(uint32_t r, uint32_t kb)
     return r * 128u + ((((kb >> 4) ^ (r & 7u)) << 4) | (kb & 15u));
 }
 
-// One thread: XOR the operand sites of k-tile `kt` into the staged A / Bt tiles, table order.
-__device__ void apply_operand_sites(const TileCtx &c, uint32_t kt, uint8_t *smem_a, uint8_t *smem_b)
+// One thread: XOR operand site `s` (entry `idx` of the table, known to lie in k-tile `kt` of this CTA's staged rows)
+// into the staged tile and log it where this CTA is the one that reports the site.
+__device__ __forceinline__ void flip_staged_operand(const TileCtx &c, const mpgemmfi_site &s, uint32_t idx, uint8_t *tile,
+                                                    uint32_t r, bool log_here)
 {
     const GemmParams &p = *c.p;
     const uint32_t sh = kshift_of(p.dtype);
     const uint32_t es = (uint32_t)esize_of(p.dtype);
-    for (uint32_t i = 0; i < c.ctl->site_count; ++i) {
-        const uint32_t idx = c.ctl->site_idx[i];
-        const mpgemmfi_site s = listed_site(c, i);
-        uint8_t *tile;
-        uint32_t r;
-        bool log_here;
-        if (s.kind == MPGEMMFI_SITE_A && in_own_rows(c, s.row)) { tile = smem_a; r = s.row - c.m0; log_here = c.n0 == 0; }
-        else if (s.kind == MPGEMMFI_SITE_B && in_own_b(c, s.col)) { tile = smem_b; r = s.col - c.b0; log_here = c.tile_m0 == 0; }
-        else continue;
-        if ((s.k >> sh) != kt) continue;
-        uint8_t *ptr = tile + swizzled_offset(r, (s.k & ((1u << sh) - 1u)) * es);
-        uint32_t before, after;
-        if (es == 2) {
-            unsigned short *w = reinterpret_cast<unsigned short *>(ptr);
-            before = *w;
-            after = flip_operand(p.dtype, before, s.xor_mask);
-            *w = (unsigned short)after;
-        } else {
-            uint32_t *w = reinterpret_cast<uint32_t *>(ptr);
-            before = *w & 0xFFFFE000u;
-            after = flip_operand(p.dtype, before, s.xor_mask);
-            *w = after;
+    uint8_t *ptr = tile + swizzled_offset(r, (s.k & ((1u << sh) - 1u)) * es);
+    uint32_t before, after;
+    if (es == 2) {
+        unsigned short *w = reinterpret_cast<unsigned short *>(ptr);
+        before = *w;
+        after = flip_operand(p.dtype, before, s.xor_mask);
+        *w = (unsigned short)after;
+    } else {
+        uint32_t *w = reinterpret_cast<uint32_t *>(ptr);
+        before = *w & 0xFFFFE000u;
+        after = flip_operand(p.dtype, before, s.xor_mask);
+        *w = after;
+    }
+    if (log_here) write_log(p, idx, before, after, after, 1u);
+}
+
+// which staged tile and row of it operand site s touches in k-tile kt of this CTA (tile == nullptr: none)
+__device__ __forceinline__ void staged_place(const TileCtx &c, const mpgemmfi_site &s, uint32_t kt, uint8_t *smem_a, uint8_t *smem_b,
+                                             uint8_t *&tile, uint32_t &r, bool &log_here)
+{
+    tile = nullptr; r = 0; log_here = false;
+    if ((s.k >> kshift_of(c.p->dtype)) != kt) return;
+    if (s.kind == MPGEMMFI_SITE_A && in_own_rows(c, s.row)) { tile = smem_a; r = s.row - c.m0; log_here = c.n0 == 0; }
+    else if (s.kind == MPGEMMFI_SITE_B && in_own_b(c, s.col)) { tile = smem_b; r = s.col - c.b0; log_here = c.tile_m0 == 0; }
+}
+
+// The whole warp: XOR the operand sites of k-tile `kt` into the staged A / Bt tiles. A list of one entry (the usual
+// case) is handled by lane 0 alone. Otherwise the lanes look through the operand entries of the CTA's list 32 at a
+// time; the entries that hit this k-tile are applied one after the other in table order (two flips of one word log
+// their before / after words in that order), each by the lane that holds it. A lane that has written fences its
+// writes towards the tensor core's (asynchronous) reads.
+__device__ __noinline__ void apply_operand_sites_many(TileCtx c, uint32_t kt, uint8_t *smem_a, uint8_t *smem_b, int lane);
+
+__device__ __forceinline__ void apply_operand_sites(const TileCtx &c, uint32_t kt, uint8_t *smem_a, uint8_t *smem_b, int lane)
+{
+    uint8_t *tile;
+    uint32_t r;
+    bool log_here;
+    if (c.ctl->site_count == 1) {
+        if (lane == 0) {
+            const mpgemmfi_site s = c.ctl->site_cache[0];
+            staged_place(c, s, kt, smem_a, smem_b, tile, r, log_here);
+            if (tile) { flip_staged_operand(c, s, c.ctl->site_idx[0], tile, r, log_here); fence_proxy_async_smem(); }
         }
-        if (log_here) write_log(p, idx, before, after, after, 1u);
+        __syncwarp();
+        return;
+    }
+    apply_operand_sites_many(c, kt, smem_a, smem_b, lane);
+}
+
+// (kept out of line, like the long form of build_site_list: the code of the one-site case stays short)
+__device__ __noinline__ void apply_operand_sites_many(TileCtx c, uint32_t kt, uint8_t *smem_a, uint8_t *smem_b, int lane)
+{
+    uint8_t *tile;
+    uint32_t r;
+    bool log_here;
+    const uint32_t n_op = c.ctl->class_end[0];
+    for (uint32_t base = 0; base < n_op; base += 32) {
+        const uint32_t i = base + (uint32_t)lane;
+        mpgemmfi_site s = {};
+        tile = nullptr; r = 0; log_here = false;
+        if (i < n_op) {
+            s = listed_site(c, i);
+            staged_place(c, s, kt, smem_a, smem_b, tile, r, log_here);
+        }
+        uint32_t vote = __ballot_sync(0xFFFFFFFFu, tile != nullptr);
+        while (vote) {
+            const int turn = __ffs(vote) - 1;
+            vote &= vote - 1u;
+            if (lane == turn) {
+                flip_staged_operand(c, s, c.ctl->site_idx[i], tile, r, log_here);
+                fence_proxy_async_smem();
+            }
+            __syncwarp();
+        }
     }
 }
 
@@ -238,7 +301,7 @@ __device__ uint32_t faulty_operand(const TileCtx &c, bool is_a, uint32_t rc, uin
 {
     const GemmParams &p = *c.p;
     uint32_t w = load_operand(p.dtype, is_a ? p.A : p.Bt, (size_t)rc * p.K + k);
-    for (uint32_t i = 0; i < c.ctl->site_count; ++i) {
+    for (uint32_t i = 0; i < c.ctl->class_end[0]; ++i) {
         const mpgemmfi_site s = listed_site(c, i);
         if (s.k != k) continue;
         if (is_a ? (s.kind == MPGEMMFI_SITE_A && s.row == rc) : (s.kind == MPGEMMFI_SITE_B && s.col == rc))
@@ -252,7 +315,7 @@ __device__ uint32_t faulty_operand(const TileCtx &c, bool is_a, uint32_t rc, uin
 __device__ void apply_boundary_sites(const TileCtx &c, uint32_t b, uint32_t tmem_acc, int q, int h, int lane)
 {
     const GemmParams &p = *c.p;
-    for (uint32_t i = 0; i < c.ctl->site_count; ++i) {
+    for (uint32_t i = c.ctl->class_end[0]; i < c.ctl->class_end[1]; ++i) {
         const uint32_t idx = c.ctl->site_idx[i];
         const mpgemmfi_site s = listed_site(c, i);
         if (!(s.kind == MPGEMMFI_SITE_ACC || s.kind == MPGEMMFI_SITE_TERM)) continue;
@@ -294,7 +357,7 @@ template <int W>
 __device__ void apply_out_sites(const TileCtx &c, uint32_t row, uint32_t c0, uint32_t (&v)[W], int pass)
 {
     const GemmParams &p = *c.p;
-    for (uint32_t i = 0; i < c.ctl->site_count; ++i) {
+    for (uint32_t i = c.ctl->class_end[1]; i < c.ctl->site_count; ++i) {
         const uint32_t idx = c.ctl->site_idx[i];
         const mpgemmfi_site s = listed_site(c, i);
         if (s.kind != MPGEMMFI_SITE_OUT || s.row != row || s.col - c0 >= (uint32_t)W) continue;
@@ -514,14 +577,16 @@ __device__ __forceinline__ SiteSlice site_slice(int n, int warp)
 // SINGLE_SITE_WARP alone (every lane holds the entry in `first`), with no compaction and no CTA-wide barrier, next
 // to the other warps' set-up; it also waits for CTA 0's cleared log where this CTA will write to it.
 template <int TM, int BN>
+__device__ __noinline__ void build_site_list_many(const GemmParams &p, Control *ctl, uint32_t gid, uint32_t groups, mpgemmfi_site first);
+
+template <int TM, int BN>
 __device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid, uint32_t groups,
                                 const mpgemmfi_site &first, uint64_t wait_ns)
 {
-    constexpr int WARPS = NUM_THREADS / 32;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n = p.n_faults;
     if (n == 0) {
-        if (tid == 0) ctl->site_count = 0;
+        if (tid == 0) { ctl->site_count = 0; ctl->class_end[0] = 0; ctl->class_end[1] = 0; }
         return;
     }
     if (n == 1) {
@@ -530,6 +595,8 @@ __device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid,
         const bool mine = ok && site_touches_group_warp<TM, BN>(first, p, gid, groups, lane);
         if (lane == 0) {
             ctl->site_count = mine ? 1u : 0u;
+            ctl->class_end[0] = (mine && site_class(first.kind) == 0) ? 1u : 0u;
+            ctl->class_end[1] = (mine && site_class(first.kind) <= 1) ? 1u : 0u;
             if (mine) { ctl->site_cache[0] = first; ctl->site_idx[0] = 0; }
             if (blockIdx.x == 0) {
                 if (!ok) write_log(p, 0, 0u, 0u, 0u, 2u);
@@ -543,22 +610,36 @@ __device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid,
         }
         return;
     }
+    build_site_list_many<TM, BN>(p, ctl, gid, groups, first);
+}
+
+template <int TM, int BN>
+__device__ __noinline__ void build_site_list_many(const GemmParams &p, Control *ctl, uint32_t gid, uint32_t groups, mpgemmfi_site first)
+{
+    constexpr int WARPS = NUM_THREADS / 32;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n = p.n_faults;
     const SiteSlice sl = site_slice(n, warp);
-    uint32_t cnt = 0, n_valid = 0, n_bad = 0, first_vote = 0;
+    uint32_t cnt[3] = {0, 0, 0}, n_valid = 0, n_bad = 0, first_vote = 0;
     for (int base = sl.beg; base < sl.end; base += 32) {
         const int i = base + lane;
         bool ok = false, mine = false;
+        int cls = 2;
         if (i < sl.end) {
             const mpgemmfi_site s = base == sl.beg ? first : table_site(p, i);
             ok = site_valid(s, p.dtype, p.M, p.N, p.K);
             mine = ok && site_touches_group<TM, BN>(s, p, gid, groups);
+            cls = site_class(s.kind);
             if (!ok && blockIdx.x == 0) write_log(p, i, 0u, 0u, 0u, 2u);
             n_valid += ok ? 1u : 0u;
             n_bad += ok ? 0u : 1u;
         }
         const uint32_t vote = __ballot_sync(0xFFFFFFFFu, mine);
+        const uint32_t v0 = __ballot_sync(0xFFFFFFFFu, mine && cls == 0), v1 = __ballot_sync(0xFFFFFFFFu, mine && cls == 1);
         if (base == sl.beg) first_vote = vote;
-        cnt += __popc(vote);
+        cnt[0] += __popc(v0);
+        cnt[1] += __popc(v1);
+        cnt[2] += __popc(vote) - __popc(v0) - __popc(v1);
     }
     if (blockIdx.x == 0 && p.flags) {
         n_valid = __reduce_add_sync(0xFFFFFFFFu, n_valid);
@@ -566,35 +647,51 @@ __device__ void build_site_list(const GemmParams &p, Control *ctl, uint32_t gid,
         if (lane == 0 && n_valid) atomicAdd(&p.flags[3], n_valid);
         if (lane == 0 && n_bad) { atomicAdd(&p.flags[4], n_bad); atomicOr(&p.flags[0], MPGEMMFI_STATUS_SITE_SKIPPED); }
     }
-    if (lane == 0) ctl->scan[warp] = cnt;
+    if (lane == 0) { ctl->scan[0][warp] = cnt[0]; ctl->scan[1][warp] = cnt[1]; ctl->scan[2][warp] = cnt[2]; }
     __syncthreads();
-    uint32_t off = 0, total = 0;
-    for (int w = 0; w < WARPS; ++w) {
-        const uint32_t x = ctl->scan[w];
-        if (w < warp) off += x;
-        total += x;
+    // where this warp's entries of each class go: after the classes before it and, inside the class, after the
+    // entries of the warps before it (their slices of the table come first)
+    uint32_t off[3], total[3];
+#pragma unroll
+    for (int c = 0; c < 3; ++c) {
+        off[c] = 0; total[c] = 0;
+        for (int w = 0; w < WARPS; ++w) {
+            const uint32_t x = ctl->scan[c][w];
+            if (w < warp) off[c] += x;
+            total[c] += x;
+        }
     }
-    if (tid == 0) ctl->site_count = total;
+    off[1] += total[0];
+    off[2] += total[0] + total[1];
+    if (tid == 0) {
+        ctl->class_end[0] = total[0];
+        ctl->class_end[1] = total[0] + total[1];
+        ctl->site_count = total[0] + total[1] + total[2];
+    }
     for (int base = sl.beg; base < sl.end; base += 32) {
         const int i = base + lane;
         bool mine = false;
         mpgemmfi_site s = first;
-        uint32_t vote = first_vote;
         if (base != sl.beg) {
             if (i < sl.end) {
                 s = table_site(p, i);
                 mine = site_valid(s, p.dtype, p.M, p.N, p.K) && site_touches_group<TM, BN>(s, p, gid, groups);
             }
-            vote = __ballot_sync(0xFFFFFFFFu, mine);
         } else {
-            mine = (vote >> lane) & 1u;
+            mine = (first_vote >> lane) & 1u;
         }
-        if (mine) {
-            const uint32_t pos = off + __popc(vote & ((1u << lane) - 1u));
-            if (pos < (uint32_t)SITE_CACHE) ctl->site_cache[pos] = s;
-            ctl->site_idx[pos] = (uint16_t)i;
+        const int cls = site_class(s.kind);
+        const uint32_t lower = (1u << lane) - 1u;
+#pragma unroll
+        for (int c = 0; c < 3; ++c) {
+            const uint32_t vc = __ballot_sync(0xFFFFFFFFu, mine && cls == c);
+            if (mine && cls == c) {
+                const uint32_t pos = off[c] + __popc(vc & lower);
+                if (pos < (uint32_t)SITE_CACHE) ctl->site_cache[pos] = s;
+                ctl->site_idx[pos] = (uint16_t)i;
+            }
+            off[c] += __popc(vc);
         }
-        off += __popc(vote);
     }
 }
 
@@ -763,9 +860,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ctl->full[stage]), (own_phase >> stage) & 1u, abort_flag, wait_ns));
                     if (!ok) break;
                     own_phase ^= 1u << stage;
-                    if (lane == 0) {
+                    {
                         uint8_t *sa = smem + stage * C::STAGE_BYTES;
-                        apply_operand_sites(tc, kt, sa, sa + C::A_BYTES);
+                        apply_operand_sites(tc, kt, sa, sa + C::A_BYTES, lane);
+                    }
+                    if (lane == 0) {
                         fence_proxy_async_smem();
                         mbar_arrive_cluster(lead_full0 + stage * (uint32_t)sizeof(uint64_t));
                     }
@@ -839,10 +938,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 tc_fence_after_sync();
                 uint8_t *sa = smem + stage * C::STAGE_BYTES;
                 if (kt == next_op) {
-                    if (lane == 0) {
-                        apply_operand_sites(tc, kt, sa, sa + C::A_BYTES);
-                        fence_proxy_async_smem();
-                    }
+                    apply_operand_sites(tc, kt, sa, sa + C::A_BYTES, lane);
+                    if (lane == 0) fence_proxy_async_smem();
                     __syncwarp();
                 }
                 if (lane == 0) {
