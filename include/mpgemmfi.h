@@ -223,7 +223,7 @@ typedef struct {
  *                Results are identical either way. The same holds for every mpgemmfi_gemm_* below.
  *                The call is tuned for short tables (the paper's one fault per run): the time grows
  *                roughly linearly up to about 64 entries and faster beyond (a 4096^3 GEMM: 0.1 ms
- *                with one site, 0.15 ms with 64 operand sites, 5 ms with 1024); many independent
+ *                with one site, 0.13 ms with 64 operand sites, 0.6 ms with 1024); many independent
  *                faults are the business of mpgemmfi_campaign.
  *   flags_out    device pointer to mpgemmfi_flags_bytes(M, N, n_faults) bytes, 16-byte
  *                aligned, written in full; may be NULL only when n_faults = 0 and the
