@@ -55,7 +55,7 @@ WORKLOAD_TEXT = {
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMM kernel, from the ncu capture summarised
 # under profiles/ (the capture names the kernel source it was taken on); None for a config without a capture of the
 # present kernel
-KERNEL_TRAFFIC_BYTES = {"c2": 152.7e6, "c3a": 266.0e6}
+KERNEL_TRAFFIC_BYTES = {"c2": 151.2e6, "c3a": 266.6e6}
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 
 
