@@ -259,6 +259,23 @@ def test_host_table_in_the_launch_parameters_equals_the_device_table(dtype):
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("name,shape,mix,trials", [
+    ("c5", (384, 192, 256), "mixed", 700),
+    ("c2", (520, 392, 320), "operand", 600),
+    ("c5", (384, 192, 256), "term_op", 300),
+    ("c4", (300, 264, 160), "acc", 500),
+])
+def test_long_tables_on_few_tiles(name, shape, mix, trials):
+    """Hundreds of sites on a handful of tiles: every CTA's list is longer than its shared-memory cache and holds
+    operand, accumulator / term and output sites side by side (the list is kept by class, each class in table
+    order); many sites share rows, columns and k-steps. Everything against the oracle: values, flags, header, log."""
+    M, N, K = shape
+    w = synth.make_workload(name, M, N, K, trials=trials, mix=mix)
+    extra = synth.make_workload(name, M, N, K, trials=trials // 3, mix="out").sites
+    sites = np.concatenate([w.sites, extra]) if mix != "mixed" else w.sites
+    check_gemm_against_oracle(w.dtype, w.A, w.Bt, sites, w.detect_mode, max_fragile=3)
+
+
 def test_maximum_site_count():
     w = synth.make_workload("c5", 1024, 64, 192, trials=mpg.MAX_FAULTS, mix="out")
     check_gemm_against_oracle(w.dtype, w.A, w.Bt, w.sites, w.detect_mode, max_fragile=2)
